@@ -1,0 +1,173 @@
+/*
+ * treekv.h -- C ABI of the TreeKV cache library for NVIDIA B200 (sm_100a).
+ *
+ * TreeKV (arXiv 2501.04987) keeps a key/value cache of fixed size c per
+ * attention head.  Each step appends the new token, attends over the cache
+ * (Section 3.1: a = SoftMax(q K^T / sqrt(d)), o = a V), accumulates for every
+ * cached token the attention weight it received (Algorithm 1: S <- S + a,
+ * C <- C + 1, importance = S / C), and once the cache is longer than c evicts
+ * the lower-scored member of the adjacent pair {idx, idx+1}, where idx cycles
+ * 1..c (Section 4.1 "Eviction Scope").  Old context thins out like a binary
+ * tree; recent context stays dense.
+ *
+ * Conventions shared by every entry point
+ *   - One treekv_ctx is one attention layer for `batch` sequences.  A layer
+ *     stack is an array of contexts driven in layer order.
+ *   - "dev" pointers are device memory, "host" pointers are host memory.  The
+ *     caller owns every buffer it passes, including the workspace, for the
+ *     life of the context.  The library allocates no device memory, never
+ *     frees caller memory and never synchronises the stream unless an entry
+ *     point says so: a call only enqueues work on `stream` (a cudaStream_t
+ *     passed as void*, NULL = the default stream).
+ *   - Tensors are contiguous, 16-byte aligned, element type = the context's
+ *     dtype (fp32 or bf16).  q and k arrive with any position encoding already
+ *     applied; the library is position-agnostic and records for every cached
+ *     token its 0-based stream index.
+ *   - Grouped-query attention: query head h uses KV head h / (n_heads /
+ *     n_kv_heads); the weight a cached token receives in a step is the mean
+ *     over the query heads of its group (equal to Algorithm 1 when the group
+ *     size is 1).
+ *   - Errors are returned, never thrown or trapped.  Argument and state errors
+ *     are detected before anything is enqueued.  Asynchronous CUDA errors
+ *     surface on a later call or in treekv_get_stats.
+ */
+#ifndef TREEKV_H
+#define TREEKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct treekv_ctx treekv_ctx; /* opaque, host-side; owned by the library */
+
+typedef enum {
+    TREEKV_OK = 0,
+    TREEKV_ERR_INVALID_ARG = 1, /* null pointer, misaligned buffer, length out of range */
+    TREEKV_ERR_BAD_STATE = 2,   /* call not valid in the context's current state */
+    TREEKV_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+    TREEKV_ERR_UNSUPPORTED = 4, /* shape or dtype outside what the kernels cover */
+    TREEKV_ERR_CUDA = 5,        /* a CUDA runtime call failed; see treekv_stats.last_cuda_error */
+    TREEKV_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up; the context must be reset */
+} treekv_status;
+
+typedef enum { TREEKV_F32 = 0, TREEKV_BF16 = 1 } treekv_dtype;
+
+/* Eviction rule.  SCORES is Algorithm 1.  KEEP_LEFT is the ablation of Section 5.4 (always keep the
+ * left token of the scope).  EVICT_LEFT is what an exact tie does under Algorithm 1's strict '>'.
+ * The two score-free rules make the retained set a function of the schedule alone. */
+typedef enum { TREEKV_RULE_SCORES = 0, TREEKV_RULE_KEEP_LEFT = 1, TREEKV_RULE_EVICT_LEFT = 2 } treekv_rule;
+
+/* Options for treekv_set_option. */
+typedef enum {
+    TREEKV_OPT_DECODE_SPLIT = 0, /* thread blocks per (sequence, KV head) in decode: 0 = automatic, else 1,2,4,8 */
+    TREEKV_OPT_PREFILL_PATH = 1  /* 0 = automatic, 1 = CUDA-core kernel, 2 = tcgen05 tensor-core kernel (bf16, head_dim 128) */
+} treekv_option;
+
+typedef struct {
+    uint64_t evictions;       /* pair evictions performed, summed over sequences (not over heads) */
+    uint64_t near_ties;       /* pair decisions whose relative score gap was below 1e-4, summed over heads */
+    uint64_t kernel_launches; /* kernels this context has enqueued since creation or reset */
+    uint32_t device_error;    /* 0, or the code a kernel left when it refused to continue */
+    int32_t last_cuda_error;  /* last cudaError_t seen by the library, 0 if none */
+} treekv_stats;
+
+/*
+ * Bytes of device workspace a context of this shape needs (0 if the shape is unsupported).
+ * The workspace holds, per (sequence, KV head): K and V slabs of 2*budget + max_chunk rows, the score sums
+ * S and the stream positions of the cached tokens; plus per-call scratch for chunked prefill (partial
+ * column sums, staging rows for compaction) and staging buffers for the *_host entry points.
+ * max_chunk = 0 makes a decode-only context.
+ */
+size_t treekv_workspace_bytes(int budget, int n_heads, int n_kv_heads, int head_dim, treekv_dtype dtype,
+                              int batch, int max_chunk);
+
+/*
+ * Create a layer context (Algorithm 1, initialisation: empty cache, idx = 1).
+ *   budget      cache size c, 2..65536                n_heads / n_kv_heads   query / KV heads, n_heads % n_kv_heads == 0,
+ *   head_dim    64 or 128                                                    group size in {1,2,4,8}
+ *   batch       1..1024 sequences                     max_chunk              longest prefill chunk, 0..8192
+ *   dev_workspace  device memory, 256-byte aligned, at least treekv_workspace_bytes(...) bytes; owned by the caller and
+ *                  used by the context until treekv_destroy
+ * Enqueues the initialisation of the workspace on `stream`.  On error *out is NULL.
+ */
+treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_heads, int head_dim,
+                            treekv_dtype dtype, int batch, int max_chunk, void* dev_workspace,
+                            size_t workspace_bytes, void* stream);
+
+/*
+ * One decode step for every active sequence (Algorithm 1, one iteration of the loop; Section 3.1 for the
+ * attention): append k,v; attend over the cache including the new token; add the weights to S; if the cache
+ * is longer than c, evict one member of the scope and advance idx.
+ *   dev_q, dev_out  [batch][n_heads][head_dim]        dev_k, dev_v  [batch][n_kv_heads][head_dim]
+ *   host_active     [batch] bytes, nonzero = take the step; NULL = all sequences.  Read before returning.
+ * Inactive sequences are untouched and their rows of dev_out are not written.
+ */
+treekv_status treekv_decode_step(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v,
+                                 void* dev_out, const uint8_t* host_active, void* stream);
+
+/*
+ * One chunk of chunked prefill (the paper's prefill is one-shot; this applies Algorithm 1 to a chunk at a
+ * time): append chunk_lens[b] tokens to sequence b; chunk row i attends to every cached token and to chunk
+ * rows <= i; S gains the column sums of the chunk's probability matrix and C advances by the chunk; then
+ * Algorithm 1's eviction branch is repeated with those scores until the cache is back to c.
+ *   dev_q, dev_out  [batch][chunk_stride][n_heads][head_dim]
+ *   dev_k, dev_v    [batch][chunk_stride][n_kv_heads][head_dim]
+ *   host_chunk_lens [batch] int32 in 0..min(chunk_stride, max_chunk) (0 = sequence not in this call); NULL = all
+ *                   chunk_stride.  Read before returning.
+ * Rows of dev_out beyond a sequence's chunk length are not written.
+ */
+treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v,
+                                   void* dev_out, const int32_t* host_chunk_lens, int chunk_stride,
+                                   void* stream);
+
+/*
+ * The same two calls with HOST tensors (pageable or pinned): inputs are copied to staging buffers inside the
+ * workspace, the step runs, and the output is copied back, all enqueued on `stream`.  host_out is valid once
+ * the stream has been synchronised.  Shapes as above.
+ */
+treekv_status treekv_decode_step_host(treekv_ctx* ctx, const void* host_q, const void* host_k, const void* host_v,
+                                      void* host_out, const uint8_t* host_active, void* stream);
+treekv_status treekv_prefill_chunk_host(treekv_ctx* ctx, const void* host_q, const void* host_k,
+                                        const void* host_v, void* host_out, const int32_t* host_chunk_lens,
+                                        int chunk_stride, void* stream);
+
+/*
+ * Stream positions of the retained tokens (what Figures 1 and 3 draw), in cache order, i.e. strictly increasing.
+ *   dev_pos    [batch][n_kv_heads][budget] int32, unused tail filled with -1
+ *   dev_count  [batch][n_kv_heads] int32, number of retained tokens (= min(tokens seen, budget))
+ */
+treekv_status treekv_retained_positions(treekv_ctx* ctx, int32_t* dev_pos, int32_t* dev_count, void* stream);
+
+/*
+ * Importance score S / C (Algorithm 1, "Importance Scores") of every retained token, in cache order.
+ *   dev_sbar   [batch][n_kv_heads][budget] float, unused tail filled with 0
+ */
+treekv_status treekv_scores(treekv_ctx* ctx, float* dev_sbar, void* stream);
+
+/* Counters and error words.  Synchronises `stream` to read the device-side counters. */
+treekv_status treekv_get_stats(treekv_ctx* ctx, treekv_stats* host_out, void* stream);
+
+/* Tokens seen so far by sequence b according to the host-side record (-1 on bad arguments). */
+int64_t treekv_tokens_seen(const treekv_ctx* ctx, int b);
+
+treekv_status treekv_set_rule(treekv_ctx* ctx, treekv_rule rule);
+treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value);
+
+/* Back to the empty cache (idx = 1, nothing seen).  Enqueued on `stream`. */
+treekv_status treekv_reset(treekv_ctx* ctx, void* stream);
+
+/* Frees the host-side context.  The workspace stays the caller's. */
+void treekv_destroy(treekv_ctx* ctx);
+
+const char* treekv_status_string(treekv_status s);
+
+/* Library version, "major.minor". */
+const char* treekv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TREEKV_H */

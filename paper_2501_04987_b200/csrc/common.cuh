@@ -1,0 +1,140 @@
+// Shared declarations of the TreeKV CUDA library: cache geometry, parameter blocks, small device helpers.
+//
+// Cache geometry ("cycle coordinates").  Algorithm 1 of the TreeKV paper evicts from the scope {idx, idx+1}
+// with idx cycling 1..c.  During one cycle of c evictions the scopes are the disjoint pairs (2p, 2p+1),
+// p = 0..c-1 (0-based), of the sequence [cache at cycle start | tokens appended during the cycle].  Each unit
+// (sequence, KV head) therefore owns a slab of R = 2c + max_chunk rows whose physical row index is the index
+// in that sequence: the survivor of pair p is moved to row p and nothing else ever moves.  With i evictions
+// done in the current cycle (i = idx - 1) and L cached tokens the live rows are
+//     [0, i)  and  [2i, L + i)            (both in stream order, the first entirely older than the second)
+// and the next token is appended at row L + i.  While the cache is still filling, i = 0 and the live rows
+// are [0, L).  "Live index" lambda in [0, L) maps to the physical row  lambda < i ? lambda : lambda + i.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/treekv.h"
+
+namespace treekv {
+
+constexpr int kMaxBatch = 1024;
+constexpr float kNearTieRel = 1e-4f;
+constexpr float kLog2e = 1.4426950408889634f;
+
+// device counters, one block per context
+struct DevStats {
+    unsigned long long near_ties;
+    unsigned int error;
+    unsigned int pad;
+};
+
+// geometry + slab pointers, passed by value to every kernel
+struct CacheView {
+    void* K;          // [units][R][d]
+    void* V;          // [units][R][d]
+    float* S;         // [units][R]   sum of attention received
+    int32_t* pos;     // [units][R]   0-based stream index of the token in the row
+    int32_t* n_seen;  // [units]      tokens fed so far (kept per unit so a kernel only reads what it alone writes)
+    DevStats* stats;
+    int c;            // budget
+    int R;            // rows per slab
+    int Hq, Hkv, B, d;
+    int rule;
+};
+
+struct ActiveMask {
+    uint32_t w[kMaxBatch / 32];
+    __host__ __device__ bool test(int b) const { return (w[b >> 5] >> (b & 31)) & 1u; }
+};
+
+// cache state derived from the number of tokens seen
+struct UnitState {
+    int L;  // cached tokens
+    int i;  // evictions done in the current cycle (idx - 1)
+};
+__host__ __device__ inline UnitState unit_state(long long n_seen, int c) {
+    UnitState s;
+    if (n_seen <= c) { s.L = (int)n_seen; s.i = 0; }
+    else { s.L = c; s.i = (int)((n_seen - c) % c); }
+    return s;
+}
+__host__ __device__ inline int phys_row(int lambda, int i) { return lambda < i ? lambda : lambda + i; }
+
+// One segment of a chunk's eviction: E pairs (2(i+p), 2(i+p)+1) -> row i+p, then, if the cycle wraps with
+// tokens still above budget, `rebase` rows [2c, 2c+rebase) move down to [c, c+rebase).
+struct EvictSegment {
+    int i;       // cycle position at segment start
+    int len;     // live rows at segment start
+    int E;       // evictions in this segment
+    int rebase;  // rows moved down after a wrap
+    int nseg;    // total number of segments for this chunk
+};
+__host__ __device__ inline EvictSegment evict_segment(long long n_seen_before, int m, int c, int seg) {
+    UnitState st = unit_state(n_seen_before, c);
+    EvictSegment cur;
+    cur.i = st.i; cur.len = st.L + m; cur.E = 0; cur.rebase = 0; cur.nseg = 0;
+    int i = st.i, len = st.L + m;
+    int s = 0;
+    while (len > c) {
+        const int E = len - c < c - i ? len - c : c - i;
+        const int len2 = len - E;
+        int i2 = i + E, rebase = 0;
+        if (i2 == c) { i2 = 0; if (len2 > c) rebase = len2 - c; }
+        if (s == seg) { cur.i = i; cur.len = len; cur.E = E; cur.rebase = rebase; }
+        i = i2; len = len2; ++s;
+    }
+    cur.nseg = s;
+    if (seg >= s) { cur.E = 0; cur.rebase = 0; }
+    return cur;
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kVec = 4;  // elements per 16-byte load
+    __device__ static void unpack(const uint4& u, float (&f)[4]) {
+        f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+    }
+    __device__ static float to_float(float x) { return x; }
+    __device__ static float from_float(float x) { return x; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kVec = 8;
+    __device__ static void unpack(const uint4& u, float (&f)[8]) {
+        f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
+        f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
+        f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
+        f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
+    }
+    __device__ static float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+    __device__ static __nv_bfloat16 from_float(float x) { return __float2bfloat16_rn(x); }
+};
+
+// 128-bit read-only load that bypasses L1 allocation; only for rows no thread writes while they are being read
+__device__ inline uint4 ld_stream(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+__device__ inline uint4 ld_plain(const void* p) { return *reinterpret_cast<const uint4*>(p); }
+
+// Algorithm 1's comparison on the averaged scores; returns true when the right member of the pair is evicted.
+// Also reports whether the decision was a near-tie (relative gap below kNearTieRel).
+__device__ inline bool pair_evicts_right(float S_l, int C_l, float S_r, int C_r, int rule, bool* near_tie) {
+    *near_tie = false;
+    if (rule == TREEKV_RULE_KEEP_LEFT) return true;
+    if (rule == TREEKV_RULE_EVICT_LEFT) return false;
+    const float a = __fdiv_rn(S_l, (float)C_l);
+    const float b = __fdiv_rn(S_r, (float)C_r);
+    const float mx = fmaxf(fabsf(a), fabsf(b));
+    *near_tie = !(fabsf(a - b) >= kNearTieRel * mx);
+    return a > b;  // strict: ties and NaN evict the left (older) slot
+}
+
+// ---- launchers implemented in the .cu files
+size_t decode_smem_bytes(int G, int D, int c, int split);
+cudaError_t launch_decode(const CacheView& cv, treekv_dtype dt, const void* q, const void* k, const void* v, void* out,
+                          const ActiveMask& active, int split, cudaStream_t stream);
+
+}  // namespace treekv

@@ -1,0 +1,340 @@
+// Decode step of TreeKV (Algorithm 1, one loop iteration; attention of Section 3.1) as ONE kernel launch.
+//
+// A thread-block cluster of `split` CTAs owns one unit (sequence, KV head).  Each CTA streams its share of
+// the c+1 live rows of K with 128-bit loads, keeps the logits of all G query heads of the group in shared
+// memory, and the cluster agrees on the softmax statistics through distributed shared memory.  Every CTA
+// then turns its logits into normalised probabilities, adds their group mean to S, streams its share of V
+// and the cluster sums the partial outputs.  Finally CTA 0 plays Algorithm 1's eviction branch: compare the
+// averaged scores of rows (2i, 2i+1), move the survivor to row i, advance the token count.  K and V are read
+// exactly once per step; nothing but the survivor row is ever moved.
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace treekv {
+
+constexpr int kDecodeThreads = 256;
+constexpr int kDecodeWarps = kDecodeThreads / 32;
+
+template <int N>
+__device__ inline void block_reduce(float (&v)[N], float* scratch /*[kDecodeWarps][N]*/, bool is_max) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int h = 0; h < N; ++h) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float x = __shfl_xor_sync(0xffffffffu, v[h], o);
+            v[h] = is_max ? fmaxf(v[h], x) : v[h] + x;
+        }
+    }
+    __syncthreads();  // scratch may still be read from a previous use
+    if (lane == 0) {
+#pragma unroll
+        for (int h = 0; h < N; ++h) scratch[warp * N + h] = v[h];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int h = 0; h < N; ++h) {
+        float r = scratch[h];
+        for (int w = 1; w < kDecodeWarps; ++w) r = is_max ? fmaxf(r, scratch[w * N + h]) : r + scratch[w * N + h];
+        v[h] = r;
+    }
+}
+
+template <typename T, int D, int G, int U>
+__global__ void __launch_bounds__(kDecodeThreads)
+decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in, const T* __restrict__ v_in,
+              T* __restrict__ out, ActiveMask active, int rows_cap) {
+    constexpr int VEC = Elem<T>::kVec;
+    constexpr int LPR = D / VEC;   // lanes per row
+    constexpr int RPW = 32 / LPR;  // rows per warp-wide load
+    constexpr int CHUNKS = D * (int)sizeof(T) / 16;
+    static_assert(LPR >= 1 && LPR <= 32 && (32 % LPR) == 0, "row must map onto a warp");
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int nsplit = (int)cluster.num_blocks();
+    const int kh = blockIdx.y, b = blockIdx.z;
+    if (!active.test(b)) return;  // the whole cluster shares b
+
+    const int unit = b * cv.Hkv + kh;
+    const int N = cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv.c);
+    const int n = st.L + 1;  // live rows including the token appended by this step
+    const int i_cyc = st.i;
+    const int per = (n + nsplit - 1) / nsplit;
+    const int lo = min(rank * per, n), hi = min(lo + per, n);
+    const int nrows = hi - lo;
+
+    T* Kc = reinterpret_cast<T*>(cv.K) + (size_t)unit * cv.R * D;
+    T* Vc = reinterpret_cast<T*>(cv.V) + (size_t)unit * cv.R * D;
+    float* Sc = cv.S + (size_t)unit * cv.R;
+    int32_t* Pc = cv.pos + (size_t)unit * cv.R;
+    const T* k_new = k_in + (size_t)unit * D;
+    const T* v_new = v_in + (size_t)unit * D;
+    const int new_row = st.L + i_cyc;  // physical row of the appended token
+
+    extern __shared__ __align__(16) float smem[];
+    float* sl = smem;                          // [G][rows_cap] logits -> probabilities
+    float* red = sl + (size_t)G * rows_cap;    // [kDecodeWarps][G]
+    float* cl_stats = red + kDecodeWarps * G;  // [2G] this CTA's (max, sum), read by the cluster
+    float* o_part = cl_stats + 2 * G;          // [G][D] this CTA's partial output, read by the cluster
+    float* o_warp = o_part + G * D;            // [kDecodeWarps][G][D]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, rsub = lane / LPR;
+
+    // ---- append (Algorithm 1: K <- K u {k}, V <- V u {v}).  This step itself reads the new token from
+    //      k_in / v_in, so the slab row is not read back before the cluster barrier below.
+    if (hi == n && nrows > 0 && warp == 0) {
+        for (int e = lane; e < CHUNKS; e += 32) {
+            reinterpret_cast<uint4*>(Kc + (size_t)new_row * D)[e] = ld_plain(reinterpret_cast<const uint4*>(k_new) + e);
+            reinterpret_cast<uint4*>(Vc + (size_t)new_row * D)[e] = ld_plain(reinterpret_cast<const uint4*>(v_new) + e);
+        }
+    }
+
+    // ---- q of the group, this lane's channel slice, pre-scaled by log2(e)/sqrt(d)
+    float qr[G][VEC];
+    {
+        const float scale = kLog2e * rsqrtf((float)D);
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            const uint4 u = ld_plain(reinterpret_cast<const uint4*>(q + ((size_t)b * cv.Hq + kh * G + h) * D) + sub);
+            Elem<T>::unpack(u, qr[h]);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) qr[h][e] *= scale;
+        }
+    }
+
+    // ---- K phase: logits (in log2 units) of this CTA's rows
+    float mx[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) mx[h] = -INFINITY;
+    for (int base = lo + warp * RPW * U; base < hi; base += kDecodeWarps * RPW * U) {
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int lam = base + u * RPW + rsub;
+            raw[u] = make_uint4(0, 0, 0, 0);
+            if (lam < hi) {
+                if (lam == n - 1) raw[u] = ld_plain(reinterpret_cast<const uint4*>(k_new) + sub);
+                else raw[u] = ld_stream(reinterpret_cast<const uint4*>(Kc + (size_t)phys_row(lam, i_cyc) * D) + sub);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int lam = base + u * RPW + rsub;
+            float f[VEC];
+            Elem<T>::unpack(raw[u], f);
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                float a = 0.f;
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) a = fmaf(qr[h][e], f[e], a);
+#pragma unroll
+                for (int o = LPR / 2; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+                if (lam < hi) {
+                    mx[h] = fmaxf(mx[h], a);
+                    if (sub == 0) sl[h * rows_cap + (lam - lo)] = a;
+                }
+            }
+        }
+    }
+    block_reduce<G>(mx, red, true);  // includes the barrier that publishes sl
+
+    // ---- e = 2^(s - max), local sum
+    float sum[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) sum[h] = 0.f;
+    for (int j = tid; j < nrows; j += kDecodeThreads) {
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            const float e = exp2f(sl[h * rows_cap + j] - mx[h]);
+            sl[h * rows_cap + j] = e;
+            sum[h] += e;
+        }
+    }
+    block_reduce<G>(sum, red, false);
+    if (tid < G) { cl_stats[tid] = mx[tid]; cl_stats[G + tid] = sum[tid]; }
+
+    cluster.sync();  // (A) every CTA's statistics are visible
+
+    // ---- global softmax statistics through distributed shared memory; factor that normalises this CTA's e
+    float fac[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+        float M = -INFINITY;
+        for (int r = 0; r < nsplit; ++r) M = fmaxf(M, cluster.map_shared_rank(cl_stats, r)[h]);
+        float Lsum = 0.f;
+        for (int r = 0; r < nsplit; ++r) {
+            const float* rs = cluster.map_shared_rank(cl_stats, r);
+            const float mr = rs[h];
+            Lsum += (mr == -INFINITY) ? 0.f : rs[G + h] * exp2f(mr - M);
+        }
+        fac[h] = (mx[h] == -INFINITY) ? 0.f : exp2f(mx[h] - M) / Lsum;
+    }
+
+    // ---- normalised probabilities; score update (Algorithm 1: S <- (S u {0}) + a, group mean)
+    for (int j = tid; j < nrows; j += kDecodeThreads) {
+        float ps = 0.f;
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            const float p = sl[h * rows_cap + j] * fac[h];
+            sl[h * rows_cap + j] = p;
+            ps += p;
+        }
+        const int lam = lo + j;
+        const int ph = phys_row(lam, i_cyc);
+        const float s_old = (lam == n - 1) ? 0.f : Sc[ph];
+        Sc[ph] = s_old + ps * (1.0f / G);
+        if (lam == n - 1) Pc[ph] = N;
+    }
+    __syncthreads();
+
+    // ---- V phase: o = sum_j p_j v_j over this CTA's rows
+    float acc[G][VEC];
+#pragma unroll
+    for (int h = 0; h < G; ++h)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[h][e] = 0.f;
+    for (int base = lo + warp * RPW * U; base < hi; base += kDecodeWarps * RPW * U) {
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int lam = base + u * RPW + rsub;
+            raw[u] = make_uint4(0, 0, 0, 0);
+            if (lam < hi) {
+                if (lam == n - 1) raw[u] = ld_plain(reinterpret_cast<const uint4*>(v_new) + sub);
+                else raw[u] = ld_stream(reinterpret_cast<const uint4*>(Vc + (size_t)phys_row(lam, i_cyc) * D) + sub);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int lam = base + u * RPW + rsub;
+            if (lam < hi) {
+                float f[VEC];
+                Elem<T>::unpack(raw[u], f);
+#pragma unroll
+                for (int h = 0; h < G; ++h) {
+                    const float p = sl[h * rows_cap + (lam - lo)];
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) acc[h][e] = fmaf(p, f[e], acc[h][e]);
+                }
+            }
+        }
+    }
+    // rows handled by the same lane slice within the warp
+#pragma unroll
+    for (int h = 0; h < G; ++h)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e)
+#pragma unroll
+            for (int o = 16; o >= LPR; o >>= 1) acc[h][e] += __shfl_xor_sync(0xffffffffu, acc[h][e], o);
+    if (rsub == 0) {
+#pragma unroll
+        for (int h = 0; h < G; ++h)
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) o_warp[(warp * G + h) * D + sub * VEC + e] = acc[h][e];
+    }
+    __syncthreads();
+    for (int t = tid; t < G * D; t += kDecodeThreads) {
+        float r = 0.f;
+        for (int w = 0; w < kDecodeWarps; ++w) r += o_warp[w * G * D + t];
+        o_part[t] = r;
+    }
+
+    cluster.sync();  // (B) partial outputs, the appended row and every S update of the unit are complete
+
+    if (rank == 0) {
+        for (int t = tid; t < G * D; t += kDecodeThreads) {
+            float r = 0.f;
+            for (int rr = 0; rr < nsplit; ++rr) r += cluster.map_shared_rank(o_part, rr)[t];
+            out[((size_t)b * cv.Hq + kh * G) * D + t] = Elem<T>::from_float(r);
+        }
+        // ---- Algorithm 1, "length > c" branch: scope {idx, idx+1} = physical rows (2i, 2i+1)
+        if (warp == 0) {
+            const int N1 = N + 1;
+            if (N1 > cv.c) {
+                const int l = 2 * i_cyc, r = l + 1;
+                int evict_right = 0;
+                if (lane == 0) {
+                    bool near_tie = false;
+                    evict_right = pair_evicts_right(__ldcg(Sc + l), N1 - __ldcg(Pc + l), __ldcg(Sc + r), N1 - __ldcg(Pc + r),
+                                                    cv.rule, &near_tie) ? 1 : 0;
+                    if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
+                }
+                evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
+                const int src = evict_right ? l : r, dst = i_cyc;
+                if (src != dst) {
+                    for (int e = lane; e < CHUNKS; e += 32) {
+                        const uint4 kk = __ldcg(reinterpret_cast<const uint4*>(Kc + (size_t)src * D) + e);
+                        const uint4 vv = __ldcg(reinterpret_cast<const uint4*>(Vc + (size_t)src * D) + e);
+                        reinterpret_cast<uint4*>(Kc + (size_t)dst * D)[e] = kk;
+                        reinterpret_cast<uint4*>(Vc + (size_t)dst * D)[e] = vv;
+                    }
+                    if (lane == 0) { Sc[dst] = __ldcg(Sc + src); Pc[dst] = __ldcg(Pc + src); }
+                }
+            }
+            if (lane == 0) cv.n_seen[unit] = N1;
+        }
+    }
+    cluster.sync();  // (C) keep shared memory alive until CTA 0 has read it
+}
+
+size_t decode_smem_bytes(int G, int D, int c, int split) {
+    const int rows_cap = (c + 1 + split - 1) / split;
+    return sizeof(float) * ((size_t)G * rows_cap + kDecodeWarps * G + 2 * G + (size_t)G * D + (size_t)kDecodeWarps * G * D);
+}
+
+template <typename T, int D, int G>
+static cudaError_t launch_decode_t(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+                                   const ActiveMask& active, int split, cudaStream_t stream) {
+    constexpr int U = 4;
+    auto kern = decode_kernel<T, D, G, U>;
+    const int rows_cap = (cv.c + 1 + split - 1) / split;
+    const size_t smem = decode_smem_bytes(G, D, cv.c, split);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(split, cv.Hkv, cv.B);
+    cfg.blockDim = dim3(kDecodeThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = split;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, cv, reinterpret_cast<const T*>(q), reinterpret_cast<const T*>(k),
+                              reinterpret_cast<const T*>(v), reinterpret_cast<T*>(out), active, rows_cap);
+}
+
+template <typename T, int D>
+static cudaError_t launch_decode_g(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+                                   const ActiveMask& active, int split, cudaStream_t stream) {
+    switch (cv.Hq / cv.Hkv) {
+        case 1: return launch_decode_t<T, D, 1>(cv, q, k, v, out, active, split, stream);
+        case 2: return launch_decode_t<T, D, 2>(cv, q, k, v, out, active, split, stream);
+        case 4: return launch_decode_t<T, D, 4>(cv, q, k, v, out, active, split, stream);
+        case 8: return launch_decode_t<T, D, 8>(cv, q, k, v, out, active, split, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_decode(const CacheView& cv, treekv_dtype dt, const void* q, const void* k, const void* v, void* out,
+                          const ActiveMask& active, int split, cudaStream_t stream) {
+    if (dt == TREEKV_F32) {
+        if (cv.d == 64) return launch_decode_g<float, 64>(cv, q, k, v, out, active, split, stream);
+        if (cv.d == 128) return launch_decode_g<float, 128>(cv, q, k, v, out, active, split, stream);
+    } else {
+        if (cv.d == 64) return launch_decode_g<__nv_bfloat16, 64>(cv, q, k, v, out, active, split, stream);
+        if (cv.d == 128) return launch_decode_g<__nv_bfloat16, 128>(cv, q, k, v, out, active, split, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace treekv
