@@ -1,0 +1,356 @@
+// C ABI of the TreeKV library: context bookkeeping, argument checks, workspace carving, launch sequencing.
+// Every step of the path runs in the kernels of decode.cu, prefill_*.cu and state.cu; this file only decides
+// what to enqueue.
+#include <new>
+#include <string.h>
+
+#include "common.cuh"
+
+using namespace treekv;
+
+struct treekv_ctx {
+    CacheView cv;
+    PrefillScratch ps;
+    treekv_dtype dt;
+    int max_chunk;
+    int G;
+    size_t elem;
+    // staging for the *_host entry points
+    void *st_q, *st_k, *st_v, *st_out;
+    // options
+    int opt_decode_split;
+    int opt_prefill_path;
+    // host-side record
+    int64_t n_seen[kMaxBatch];
+    uint64_t evictions;
+    uint64_t launches;
+    int last_cuda_error;
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr size_t kSmemLimit = 227 * 1024;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+    size_t K, V, S, pos, n_seen, stats, colsum, stage_K, stage_V, stage_S, stage_pos, st_q, st_k, st_v, st_out, total;
+    int R, QT, n_max;
+};
+
+bool shape_ok(int budget, int n_heads, int n_kv_heads, int head_dim, treekv_dtype dt, int batch, int max_chunk) {
+    if (budget < 2 || budget > 65536) return false;
+    if (n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads) return false;
+    const int G = n_heads / n_kv_heads;
+    if (!(G == 1 || G == 2 || G == 4 || G == 8)) return false;
+    if (!(head_dim == 64 || head_dim == 128)) return false;
+    if (!(dt == TREEKV_F32 || dt == TREEKV_BF16)) return false;
+    if (batch < 1 || batch > kMaxBatch) return false;
+    if (max_chunk < 0 || max_chunk > 8192) return false;
+    if (n_kv_heads > 65535 || (long long)batch * n_kv_heads > 65535) return false;  // grid.y of the per-unit kernels
+    if (decode_smem_bytes(G, head_dim, budget, 8) > kSmemLimit) return false;
+    if (max_chunk > 0 && prefill_simt_smem_bytes(G, head_dim, budget + max_chunk) > kSmemLimit) return false;
+    return true;
+}
+
+Layout make_layout(int budget, int n_heads, int n_kv_heads, int head_dim, treekv_dtype dt, int batch, int max_chunk) {
+    Layout L;
+    const size_t e = dt == TREEKV_F32 ? 4 : 2;
+    const size_t units = (size_t)batch * n_kv_heads;
+    const int G = n_heads / n_kv_heads;
+    L.R = 2 * budget + max_chunk;
+    L.QT = max_chunk > 0 ? (max_chunk * G + kQTileRows - 1) / kQTileRows : 0;
+    L.n_max = budget + max_chunk;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    L.K = take(units * L.R * head_dim * e);
+    L.V = take(units * L.R * head_dim * e);
+    L.S = take(units * L.R * 4);
+    L.pos = take(units * L.R * 4);
+    L.n_seen = take(units * 4);
+    L.stats = take(sizeof(DevStats));
+    L.colsum = take(units * L.QT * L.n_max * 4);
+    L.stage_K = take(units * max_chunk * head_dim * e);
+    L.stage_V = take(units * max_chunk * head_dim * e);
+    L.stage_S = take(units * max_chunk * 4);
+    L.stage_pos = take(units * max_chunk * 4);
+    const size_t mc = max_chunk > 0 ? max_chunk : 1;
+    L.st_q = take((size_t)batch * mc * n_heads * head_dim * e);
+    L.st_k = take((size_t)batch * mc * n_kv_heads * head_dim * e);
+    L.st_v = take((size_t)batch * mc * n_kv_heads * head_dim * e);
+    L.st_out = take((size_t)batch * mc * n_heads * head_dim * e);
+    L.total = off;
+    return L;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+treekv_status cuda_fail(treekv_ctx* ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda_error = (int)e;
+    return TREEKV_ERR_CUDA;
+}
+
+int pick_decode_split(const treekv_ctx* ctx) {
+    const int c = ctx->cv.c, units = ctx->cv.B * ctx->cv.Hkv;
+    int s = ctx->opt_decode_split;
+    if (s == 0) {
+        s = 1;
+        while (s < 8 && units * s < 444 && (c + 1) / (2 * s) >= 128) s *= 2;
+    }
+    while (s < 8 && decode_smem_bytes(ctx->G, ctx->cv.d, c, s) > kSmemLimit) s *= 2;
+    return s;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t treekv_workspace_bytes(int budget, int n_heads, int n_kv_heads, int head_dim, treekv_dtype dtype, int batch,
+                              int max_chunk) {
+    if (!shape_ok(budget, n_heads, n_kv_heads, head_dim, dtype, batch, max_chunk)) return 0;
+    return make_layout(budget, n_heads, n_kv_heads, head_dim, dtype, batch, max_chunk).total;
+}
+
+treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_heads, int head_dim, treekv_dtype dtype,
+                            int batch, int max_chunk, void* dev_workspace, size_t workspace_bytes, void* stream) {
+    if (!out) return TREEKV_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!shape_ok(budget, n_heads, n_kv_heads, head_dim, dtype, batch, max_chunk)) return TREEKV_ERR_UNSUPPORTED;
+    const Layout L = make_layout(budget, n_heads, n_kv_heads, head_dim, dtype, batch, max_chunk);
+    if (!dev_workspace || (reinterpret_cast<uintptr_t>(dev_workspace) % kAlign) != 0 || workspace_bytes < L.total)
+        return TREEKV_ERR_WORKSPACE;
+    treekv_ctx* ctx = new (std::nothrow) treekv_ctx;
+    if (!ctx) return TREEKV_ERR_INVALID_ARG;
+    memset(ctx, 0, sizeof(*ctx));
+    char* base = static_cast<char*>(dev_workspace);
+    ctx->cv.K = base + L.K;
+    ctx->cv.V = base + L.V;
+    ctx->cv.S = reinterpret_cast<float*>(base + L.S);
+    ctx->cv.pos = reinterpret_cast<int32_t*>(base + L.pos);
+    ctx->cv.n_seen = reinterpret_cast<int32_t*>(base + L.n_seen);
+    ctx->cv.stats = reinterpret_cast<DevStats*>(base + L.stats);
+    ctx->cv.c = budget; ctx->cv.R = L.R; ctx->cv.Hq = n_heads; ctx->cv.Hkv = n_kv_heads; ctx->cv.B = batch;
+    ctx->cv.d = head_dim; ctx->cv.rule = TREEKV_RULE_SCORES;
+    ctx->ps.colsum = reinterpret_cast<float*>(base + L.colsum);
+    ctx->ps.stage_K = base + L.stage_K;
+    ctx->ps.stage_V = base + L.stage_V;
+    ctx->ps.stage_S = reinterpret_cast<float*>(base + L.stage_S);
+    ctx->ps.stage_pos = reinterpret_cast<int32_t*>(base + L.stage_pos);
+    ctx->ps.QT = L.QT; ctx->ps.n_max = L.n_max; ctx->ps.max_chunk = max_chunk;
+    ctx->st_q = base + L.st_q; ctx->st_k = base + L.st_k; ctx->st_v = base + L.st_v; ctx->st_out = base + L.st_out;
+    ctx->dt = dtype; ctx->max_chunk = max_chunk; ctx->G = n_heads / n_kv_heads;
+    ctx->elem = dtype == TREEKV_F32 ? 4 : 2;
+    const cudaError_t e = launch_init_state(ctx->cv, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { delete ctx; return TREEKV_ERR_CUDA; }
+    ctx->launches = 1;
+    *out = ctx;
+    return TREEKV_OK;
+}
+
+treekv_status treekv_reset(treekv_ctx* ctx, void* stream) {
+    if (!ctx) return TREEKV_ERR_INVALID_ARG;
+    const cudaError_t e = launch_init_state(ctx->cv, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    memset(ctx->n_seen, 0, sizeof(ctx->n_seen));
+    ctx->evictions = 0;
+    ctx->launches = 1;
+    return TREEKV_OK;
+}
+
+void treekv_destroy(treekv_ctx* ctx) { delete ctx; }
+
+treekv_status treekv_decode_step(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v, void* dev_out,
+                                 const uint8_t* host_active, void* stream) {
+    if (!ctx || !dev_q || !dev_k || !dev_v || !dev_out) return TREEKV_ERR_INVALID_ARG;
+    if (!aligned16(dev_q) || !aligned16(dev_k) || !aligned16(dev_v) || !aligned16(dev_out)) return TREEKV_ERR_INVALID_ARG;
+    ActiveMask mask;
+    memset(&mask, 0, sizeof(mask));
+    int n_active = 0;
+    for (int b = 0; b < ctx->cv.B; ++b) {
+        if (!host_active || host_active[b]) {
+            if (ctx->n_seen[b] >= 0x7fffffff - 1) return TREEKV_ERR_BAD_STATE;
+            mask.w[b >> 5] |= 1u << (b & 31);
+            ++n_active;
+        }
+    }
+    if (n_active == 0) return TREEKV_OK;
+    const cudaError_t e = launch_decode(ctx->cv, ctx->dt, dev_q, dev_k, dev_v, dev_out, mask, pick_decode_split(ctx),
+                                        static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    for (int b = 0; b < ctx->cv.B; ++b) {
+        if (mask.test(b)) {
+            ctx->n_seen[b] += 1;
+            if (ctx->n_seen[b] > ctx->cv.c) ctx->evictions += 1;
+        }
+    }
+    return TREEKV_OK;
+}
+
+treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v, void* dev_out,
+                                   const int32_t* host_chunk_lens, int chunk_stride, void* stream) {
+    if (!ctx || !dev_q || !dev_k || !dev_v || !dev_out) return TREEKV_ERR_INVALID_ARG;
+    if (!aligned16(dev_q) || !aligned16(dev_k) || !aligned16(dev_v) || !aligned16(dev_out)) return TREEKV_ERR_INVALID_ARG;
+    if (ctx->max_chunk == 0) return TREEKV_ERR_BAD_STATE;  // decode-only context
+    if (chunk_stride < 1) return TREEKV_ERR_INVALID_ARG;
+    ChunkLens lens;
+    memset(&lens, 0, sizeof(lens));
+    int max_m = 0, max_seg = 0;
+    for (int b = 0; b < ctx->cv.B; ++b) {
+        const int m = host_chunk_lens ? host_chunk_lens[b] : chunk_stride;
+        if (m < 0 || m > chunk_stride || m > ctx->max_chunk) return TREEKV_ERR_INVALID_ARG;
+        if (ctx->n_seen[b] + m >= 0x7fffffff - 1) return TREEKV_ERR_BAD_STATE;
+        lens.m[b] = (uint16_t)m;
+        if (m > max_m) max_m = m;
+        if (m > 0) {
+            const int ns = evict_segment(ctx->n_seen[b], m, ctx->cv.c, 0).nseg;
+            if (ns > max_seg) max_seg = ns;
+        }
+    }
+    if (max_m == 0) return TREEKV_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, chunk_stride, max_m, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = launch_prefill_simt(ctx->cv, ctx->dt, ctx->ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = launch_chunk_scores(ctx->cv, ctx->ps, lens, max_m, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 3;
+    for (int seg = 0; seg < max_seg; ++seg) {
+        int max_items = 0;
+        for (int b = 0; b < ctx->cv.B; ++b) {
+            if (!lens.m[b]) continue;
+            const EvictSegment sg = evict_segment(ctx->n_seen[b], lens.m[b], ctx->cv.c, seg);
+            if (sg.E + sg.rebase > max_items) max_items = sg.E + sg.rebase;
+        }
+        e = launch_chunk_evict(ctx->cv, ctx->dt, ctx->ps, lens, seg, max_items, s);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 2;
+    }
+    e = launch_chunk_finalize(ctx->cv, lens, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    for (int b = 0; b < ctx->cv.B; ++b) {
+        const int64_t before = ctx->n_seen[b];
+        ctx->n_seen[b] += lens.m[b];
+        const int64_t ev_before = before > ctx->cv.c ? before - ctx->cv.c : 0;
+        const int64_t ev_after = ctx->n_seen[b] > ctx->cv.c ? ctx->n_seen[b] - ctx->cv.c : 0;
+        ctx->evictions += (uint64_t)(ev_after - ev_before);
+    }
+    return TREEKV_OK;
+}
+
+treekv_status treekv_decode_step_host(treekv_ctx* ctx, const void* host_q, const void* host_k, const void* host_v,
+                                      void* host_out, const uint8_t* host_active, void* stream) {
+    if (!ctx || !host_q || !host_k || !host_v || !host_out) return TREEKV_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t qb = (size_t)ctx->cv.B * ctx->cv.Hq * ctx->cv.d * ctx->elem;
+    const size_t kb = (size_t)ctx->cv.B * ctx->cv.Hkv * ctx->cv.d * ctx->elem;
+    cudaError_t e = cudaMemcpyAsync(ctx->st_q, host_q, qb, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->st_k, host_k, kb, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->st_v, host_v, kb, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    const treekv_status st = treekv_decode_step(ctx, ctx->st_q, ctx->st_k, ctx->st_v, ctx->st_out, host_active, stream);
+    if (st != TREEKV_OK) return st;
+    e = cudaMemcpyAsync(host_out, ctx->st_out, qb, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return TREEKV_OK;
+}
+
+treekv_status treekv_prefill_chunk_host(treekv_ctx* ctx, const void* host_q, const void* host_k, const void* host_v,
+                                        void* host_out, const int32_t* host_chunk_lens, int chunk_stride, void* stream) {
+    if (!ctx || !host_q || !host_k || !host_v || !host_out) return TREEKV_ERR_INVALID_ARG;
+    if (ctx->max_chunk == 0) return TREEKV_ERR_BAD_STATE;
+    if (chunk_stride < 1 || chunk_stride > ctx->max_chunk) return TREEKV_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t qb = (size_t)ctx->cv.B * chunk_stride * ctx->cv.Hq * ctx->cv.d * ctx->elem;
+    const size_t kb = (size_t)ctx->cv.B * chunk_stride * ctx->cv.Hkv * ctx->cv.d * ctx->elem;
+    cudaError_t e = cudaMemcpyAsync(ctx->st_q, host_q, qb, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->st_k, host_k, kb, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->st_v, host_v, kb, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    const treekv_status st =
+        treekv_prefill_chunk(ctx, ctx->st_q, ctx->st_k, ctx->st_v, ctx->st_out, host_chunk_lens, chunk_stride, stream);
+    if (st != TREEKV_OK) return st;
+    e = cudaMemcpyAsync(host_out, ctx->st_out, qb, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return TREEKV_OK;
+}
+
+treekv_status treekv_retained_positions(treekv_ctx* ctx, int32_t* dev_pos, int32_t* dev_count, void* stream) {
+    if (!ctx || !dev_pos || !dev_count) return TREEKV_ERR_INVALID_ARG;
+    const cudaError_t e = launch_retained_positions(ctx->cv, dev_pos, dev_count, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return TREEKV_OK;
+}
+
+treekv_status treekv_scores(treekv_ctx* ctx, float* dev_sbar, void* stream) {
+    if (!ctx || !dev_sbar) return TREEKV_ERR_INVALID_ARG;
+    const cudaError_t e = launch_scores(ctx->cv, dev_sbar, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return TREEKV_OK;
+}
+
+treekv_status treekv_get_stats(treekv_ctx* ctx, treekv_stats* host_out, void* stream) {
+    if (!ctx || !host_out) return TREEKV_ERR_INVALID_ARG;
+    DevStats ds;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(&ds, ctx->cv.stats, sizeof(ds), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    host_out->evictions = ctx->evictions;
+    host_out->near_ties = ds.near_ties;
+    host_out->kernel_launches = ctx->launches;
+    host_out->device_error = ds.error;
+    host_out->last_cuda_error = ctx->last_cuda_error;
+    return ds.error ? TREEKV_ERR_TIMEOUT : TREEKV_OK;
+}
+
+int64_t treekv_tokens_seen(const treekv_ctx* ctx, int b) {
+    if (!ctx || b < 0 || b >= ctx->cv.B) return -1;
+    return ctx->n_seen[b];
+}
+
+treekv_status treekv_set_rule(treekv_ctx* ctx, treekv_rule rule) {
+    if (!ctx) return TREEKV_ERR_INVALID_ARG;
+    if (rule != TREEKV_RULE_SCORES && rule != TREEKV_RULE_KEEP_LEFT && rule != TREEKV_RULE_EVICT_LEFT)
+        return TREEKV_ERR_INVALID_ARG;
+    ctx->cv.rule = (int)rule;
+    return TREEKV_OK;
+}
+
+treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value) {
+    if (!ctx) return TREEKV_ERR_INVALID_ARG;
+    switch (opt) {
+        case TREEKV_OPT_DECODE_SPLIT:
+            if (!(value == 0 || value == 1 || value == 2 || value == 4 || value == 8)) return TREEKV_ERR_INVALID_ARG;
+            if (value && decode_smem_bytes(ctx->G, ctx->cv.d, ctx->cv.c, value) > kSmemLimit) return TREEKV_ERR_UNSUPPORTED;
+            ctx->opt_decode_split = value;
+            return TREEKV_OK;
+        case TREEKV_OPT_PREFILL_PATH:
+            if (value < 0 || value > 2) return TREEKV_ERR_INVALID_ARG;
+            if (value == 2) return TREEKV_ERR_UNSUPPORTED;
+            ctx->opt_prefill_path = value;
+            return TREEKV_OK;
+    }
+    return TREEKV_ERR_INVALID_ARG;
+}
+
+const char* treekv_status_string(treekv_status s) {
+    switch (s) {
+        case TREEKV_OK: return "ok";
+        case TREEKV_ERR_INVALID_ARG: return "invalid argument";
+        case TREEKV_ERR_BAD_STATE: return "call not valid in this state";
+        case TREEKV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case TREEKV_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case TREEKV_ERR_CUDA: return "CUDA runtime error";
+        case TREEKV_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+const char* treekv_version(void) { return "0.1"; }
+
+}  // extern "C"

@@ -132,9 +132,43 @@ __device__ inline bool pair_evicts_right(float S_l, int C_l, float S_r, int C_r,
     return a > b;  // strict: ties and NaN evict the left (older) slot
 }
 
-// ---- launchers implemented in the .cu files
+// chunk length of every sequence in a prefill call (0 = not in the call), passed by value
+struct ChunkLens {
+    uint16_t m[kMaxBatch];
+};
+
+// per-call scratch of chunked prefill, carved from the context's workspace
+struct PrefillScratch {
+    float* colsum;    // [units][QT][n_max] partial column sums of the chunk's probability matrix, one slice per
+                      // tile of 128 query rows (row = token * G + head), indexed by live index
+    void* stage_K;    // [units][max_chunk][d] rows in flight during compaction
+    void* stage_V;    // [units][max_chunk][d]
+    float* stage_S;   // [units][max_chunk]
+    int32_t* stage_pos;  // [units][max_chunk]
+    int QT;           // tiles per unit: ceil(G * max_chunk / 128)
+    int n_max;        // c + max_chunk
+    int max_chunk;
+};
+constexpr int kQTileRows = 128;  // query rows (token x head-in-group) per prefill tile
+
+// ---- launchers implemented in the .cu files (each enqueues on `stream` and returns the launch status)
 size_t decode_smem_bytes(int G, int D, int c, int split);
 cudaError_t launch_decode(const CacheView& cv, treekv_dtype dt, const void* q, const void* k, const void* v, void* out,
                           const ActiveMask& active, int split, cudaStream_t stream);
+
+cudaError_t launch_init_state(const CacheView& cv, cudaStream_t stream);
+cudaError_t launch_retained_positions(const CacheView& cv, int32_t* pos_out, int32_t* count_out, cudaStream_t stream);
+cudaError_t launch_scores(const CacheView& cv, float* sbar_out, cudaStream_t stream);
+cudaError_t launch_chunk_append(const CacheView& cv, treekv_dtype dt, const void* k, const void* v, const ChunkLens& lens,
+                                int chunk_stride, int max_m, cudaStream_t stream);
+cudaError_t launch_chunk_scores(const CacheView& cv, const PrefillScratch& ps, const ChunkLens& lens, int max_m,
+                                cudaStream_t stream);
+cudaError_t launch_chunk_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
+                               int seg, int max_items, cudaStream_t stream);  // gather + scatter: two launches
+cudaError_t launch_chunk_finalize(const CacheView& cv, const ChunkLens& lens, cudaStream_t stream);
+
+size_t prefill_simt_smem_bytes(int G, int D, int n_max);
+cudaError_t launch_prefill_simt(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const void* q, void* out,
+                                const ChunkLens& lens, int chunk_stride, int max_m, cudaStream_t stream);
 
 }  // namespace treekv

@@ -10,38 +10,11 @@
 #include <cooperative_groups.h>
 
 #include "common.cuh"
+#include "simt_attend.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace treekv {
-
-constexpr int kDecodeThreads = 256;
-constexpr int kDecodeWarps = kDecodeThreads / 32;
-
-template <int N>
-__device__ inline void block_reduce(float (&v)[N], float* scratch /*[kDecodeWarps][N]*/, bool is_max) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int h = 0; h < N; ++h) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float x = __shfl_xor_sync(0xffffffffu, v[h], o);
-            v[h] = is_max ? fmaxf(v[h], x) : v[h] + x;
-        }
-    }
-    __syncthreads();  // scratch may still be read from a previous use
-    if (lane == 0) {
-#pragma unroll
-        for (int h = 0; h < N; ++h) scratch[warp * N + h] = v[h];
-    }
-    __syncthreads();
-#pragma unroll
-    for (int h = 0; h < N; ++h) {
-        float r = scratch[h];
-        for (int w = 1; w < kDecodeWarps; ++w) r = is_max ? fmaxf(r, scratch[w * N + h]) : r + scratch[w * N + h];
-        v[h] = r;
-    }
-}
 
 template <typename T, int D, int G, int U>
 __global__ void __launch_bounds__(kDecodeThreads)
@@ -110,38 +83,7 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
 
     // ---- K phase: logits (in log2 units) of this CTA's rows
     float mx[G];
-#pragma unroll
-    for (int h = 0; h < G; ++h) mx[h] = -INFINITY;
-    for (int base = lo + warp * RPW * U; base < hi; base += kDecodeWarps * RPW * U) {
-        uint4 raw[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int lam = base + u * RPW + rsub;
-            raw[u] = make_uint4(0, 0, 0, 0);
-            if (lam < hi) {
-                if (lam == n - 1) raw[u] = ld_plain(reinterpret_cast<const uint4*>(k_new) + sub);
-                else raw[u] = ld_stream(reinterpret_cast<const uint4*>(Kc + (size_t)phys_row(lam, i_cyc) * D) + sub);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int lam = base + u * RPW + rsub;
-            float f[VEC];
-            Elem<T>::unpack(raw[u], f);
-#pragma unroll
-            for (int h = 0; h < G; ++h) {
-                float a = 0.f;
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) a = fmaf(qr[h][e], f[e], a);
-#pragma unroll
-                for (int o = LPR / 2; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-                if (lam < hi) {
-                    mx[h] = fmaxf(mx[h], a);
-                    if (sub == 0) sl[h * rows_cap + (lam - lo)] = a;
-                }
-            }
-        }
-    }
+    k_phase<T, D, G, U>(Kc, lo, hi, i_cyc, n - 1, k_new, qr, sl, rows_cap, mx);
     block_reduce<G>(mx, red, true);  // includes the barrier that publishes sl
 
     // ---- e = 2^(s - max), local sum
@@ -194,56 +136,7 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
     __syncthreads();
 
     // ---- V phase: o = sum_j p_j v_j over this CTA's rows
-    float acc[G][VEC];
-#pragma unroll
-    for (int h = 0; h < G; ++h)
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) acc[h][e] = 0.f;
-    for (int base = lo + warp * RPW * U; base < hi; base += kDecodeWarps * RPW * U) {
-        uint4 raw[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int lam = base + u * RPW + rsub;
-            raw[u] = make_uint4(0, 0, 0, 0);
-            if (lam < hi) {
-                if (lam == n - 1) raw[u] = ld_plain(reinterpret_cast<const uint4*>(v_new) + sub);
-                else raw[u] = ld_stream(reinterpret_cast<const uint4*>(Vc + (size_t)phys_row(lam, i_cyc) * D) + sub);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int lam = base + u * RPW + rsub;
-            if (lam < hi) {
-                float f[VEC];
-                Elem<T>::unpack(raw[u], f);
-#pragma unroll
-                for (int h = 0; h < G; ++h) {
-                    const float p = sl[h * rows_cap + (lam - lo)];
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) acc[h][e] = fmaf(p, f[e], acc[h][e]);
-                }
-            }
-        }
-    }
-    // rows handled by the same lane slice within the warp
-#pragma unroll
-    for (int h = 0; h < G; ++h)
-#pragma unroll
-        for (int e = 0; e < VEC; ++e)
-#pragma unroll
-            for (int o = 16; o >= LPR; o >>= 1) acc[h][e] += __shfl_xor_sync(0xffffffffu, acc[h][e], o);
-    if (rsub == 0) {
-#pragma unroll
-        for (int h = 0; h < G; ++h)
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) o_warp[(warp * G + h) * D + sub * VEC + e] = acc[h][e];
-    }
-    __syncthreads();
-    for (int t = tid; t < G * D; t += kDecodeThreads) {
-        float r = 0.f;
-        for (int w = 0; w < kDecodeWarps; ++w) r += o_warp[w * G * D + t];
-        o_part[t] = r;
-    }
+    v_phase<T, D, G, U>(Vc, lo, hi, i_cyc, n - 1, v_new, sl, rows_cap, o_warp, o_part);
 
     cluster.sync();  // (B) partial outputs, the appended row and every S update of the unit are complete
 

@@ -1,0 +1,216 @@
+// Cache-state kernels of the TreeKV library: initialisation, read-outs in cache order, and the per-chunk
+// steps around prefill attention: append, score update (Algorithm 1: S <- S + a, summed over the chunk),
+// repeated pair eviction with frozen scores, compaction.
+#include "common.cuh"
+
+namespace treekv {
+
+// ---------------------------------------------------------------------------------------------------------
+__global__ void init_state_kernel(CacheView cv) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < cv.B * cv.Hkv) cv.n_seen[t] = 0;
+    if (t == 0) { cv.stats->near_ties = 0ull; cv.stats->error = 0u; cv.stats->pad = 0u; }
+}
+cudaError_t launch_init_state(const CacheView& cv, cudaStream_t stream) {
+    const int units = cv.B * cv.Hkv;
+    init_state_kernel<<<(units + 255) / 256, 256, 0, stream>>>(cv);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Retained positions / averaged scores in cache order (live index order).
+__global__ void retained_positions_kernel(CacheView cv, int32_t* pos_out, int32_t* count_out) {
+    const int unit = blockIdx.x;
+    const int N = cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv.c);
+    const int32_t* Pc = cv.pos + (size_t)unit * cv.R;
+    for (int lam = threadIdx.x; lam < cv.c; lam += blockDim.x)
+        pos_out[(size_t)unit * cv.c + lam] = lam < st.L ? Pc[phys_row(lam, st.i)] : -1;
+    if (threadIdx.x == 0) count_out[unit] = st.L;
+}
+cudaError_t launch_retained_positions(const CacheView& cv, int32_t* pos_out, int32_t* count_out, cudaStream_t stream) {
+    retained_positions_kernel<<<cv.B * cv.Hkv, 256, 0, stream>>>(cv, pos_out, count_out);
+    return cudaGetLastError();
+}
+
+__global__ void scores_kernel(CacheView cv, float* sbar_out) {
+    const int unit = blockIdx.x;
+    const int N = cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv.c);
+    const int32_t* Pc = cv.pos + (size_t)unit * cv.R;
+    const float* Sc = cv.S + (size_t)unit * cv.R;
+    for (int lam = threadIdx.x; lam < cv.c; lam += blockDim.x) {
+        float r = 0.f;
+        if (lam < st.L) {
+            const int ph = phys_row(lam, st.i);
+            r = __fdiv_rn(Sc[ph], (float)(N - Pc[ph]));  // Algorithm 1: S-bar = S / C with C = tokens seen - position
+        }
+        sbar_out[(size_t)unit * cv.c + lam] = r;
+    }
+}
+cudaError_t launch_scores(const CacheView& cv, float* sbar_out, cudaStream_t stream) {
+    scores_kernel<<<cv.B * cv.Hkv, 256, 0, stream>>>(cv, sbar_out);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Chunk append: chunk token t of sequence b goes to physical row L + i + t of every KV head's slab.
+// One warp per (token, unit); k,v are [B][chunk_stride][Hkv][d].
+template <typename T>
+__global__ void chunk_append_kernel(CacheView cv, const T* __restrict__ k, const T* __restrict__ v, ChunkLens lens,
+                                    int chunk_stride) {
+    const int unit = blockIdx.y;
+    const int b = unit / cv.Hkv, kh = unit % cv.Hkv;
+    const int m = lens.m[b];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (t >= m) return;
+    const int N = cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv.c);
+    const int row = st.L + st.i + t;
+    const int chunks = cv.d * (int)sizeof(T) / 16;
+    const uint4* ks = reinterpret_cast<const uint4*>(k + (((size_t)b * chunk_stride + t) * cv.Hkv + kh) * cv.d);
+    const uint4* vs = reinterpret_cast<const uint4*>(v + (((size_t)b * chunk_stride + t) * cv.Hkv + kh) * cv.d);
+    uint4* kd = reinterpret_cast<uint4*>(reinterpret_cast<T*>(cv.K) + ((size_t)unit * cv.R + row) * cv.d);
+    uint4* vd = reinterpret_cast<uint4*>(reinterpret_cast<T*>(cv.V) + ((size_t)unit * cv.R + row) * cv.d);
+    for (int e = lane; e < chunks; e += 32) { kd[e] = ks[e]; vd[e] = vs[e]; }
+    if (lane == 0) {
+        cv.pos[(size_t)unit * cv.R + row] = N + t;
+        cv.S[(size_t)unit * cv.R + row] = 0.f;
+    }
+}
+cudaError_t launch_chunk_append(const CacheView& cv, treekv_dtype dt, const void* k, const void* v, const ChunkLens& lens,
+                                int chunk_stride, int max_m, cudaStream_t stream) {
+    dim3 grid((max_m + 7) / 8, cv.B * cv.Hkv);
+    if (dt == TREEKV_F32)
+        chunk_append_kernel<float><<<grid, 256, 0, stream>>>(cv, (const float*)k, (const float*)v, lens, chunk_stride);
+    else
+        chunk_append_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(cv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
+                                                                      lens, chunk_stride);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Chunk score update: S[row(lam)] += (sum over query tiles of the partial column sums) / G, tiles added in
+// a fixed order so the result does not depend on scheduling.
+__global__ void chunk_scores_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
+    const int unit = blockIdx.y;
+    const int b = unit / cv.Hkv;
+    const int m = lens.m[b];
+    if (m == 0) return;
+    const int G = cv.Hq / cv.Hkv;
+    const int N = cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv.c);
+    const int n = st.L + m;
+    const int lam = blockIdx.x * blockDim.x + threadIdx.x;
+    if (lam >= n) return;
+    const int qt = (m * G + kQTileRows - 1) / kQTileRows;
+    const float* part = ps.colsum + (size_t)unit * ps.QT * ps.n_max + lam;
+    float s = 0.f;
+    for (int t = 0; t < qt; ++t) s += part[(size_t)t * ps.n_max];
+    float* Sp = cv.S + (size_t)unit * cv.R + phys_row(lam, st.i);
+    *Sp = *Sp + s * (1.0f / (float)G);  // chunk rows were zeroed by the append
+}
+cudaError_t launch_chunk_scores(const CacheView& cv, const PrefillScratch& ps, const ChunkLens& lens, int max_m,
+                                cudaStream_t stream) {
+    const int n_up = cv.c + max_m;
+    dim3 grid((n_up + 255) / 256, cv.B * cv.Hkv);
+    chunk_scores_kernel<<<grid, 256, 0, stream>>>(cv, ps, lens);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Chunk eviction, one segment (see EvictSegment).  Algorithm 1's "length > c" branch repeated with frozen
+// averaged scores: between two wraps of idx the scopes are disjoint, so all pairs of a segment are decided
+// at once.  The survivor of pair p must land on row i+p, which can be a source row of an earlier pair, so the
+// move goes through staging rows: gather (decide + copy out), then scatter (copy in) as a second launch.
+template <typename T>
+__global__ void chunk_evict_gather_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int seg) {
+    const int unit = blockIdx.y;
+    const int b = unit / cv.Hkv;
+    const int m = lens.m[b];
+    if (m == 0) return;
+    const int N = cv.n_seen[unit];
+    const EvictSegment sg = evict_segment(N, m, cv.c, seg);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int item = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (item >= sg.E + sg.rebase) return;
+    const int N1 = N + m;
+    T* Kc = reinterpret_cast<T*>(cv.K) + (size_t)unit * cv.R * cv.d;
+    T* Vc = reinterpret_cast<T*>(cv.V) + (size_t)unit * cv.R * cv.d;
+    const float* Sc = cv.S + (size_t)unit * cv.R;
+    const int32_t* Pc = cv.pos + (size_t)unit * cv.R;
+    int src;
+    if (item < sg.E) {
+        const int l = 2 * (sg.i + item), r = l + 1;
+        int evict_right = 0;
+        if (lane == 0) {
+            bool near_tie = false;
+            evict_right = pair_evicts_right(Sc[l], N1 - Pc[l], Sc[r], N1 - Pc[r], cv.rule, &near_tie) ? 1 : 0;
+            if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
+        }
+        evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
+        src = evict_right ? l : r;
+    } else {
+        src = 2 * cv.c + (item - sg.E);
+    }
+    const int chunks = cv.d * (int)sizeof(T) / 16;
+    const size_t so = ((size_t)unit * ps.max_chunk + item);
+    uint4* kd = reinterpret_cast<uint4*>(reinterpret_cast<T*>(ps.stage_K) + so * cv.d);
+    uint4* vd = reinterpret_cast<uint4*>(reinterpret_cast<T*>(ps.stage_V) + so * cv.d);
+    const uint4* ks = reinterpret_cast<const uint4*>(Kc + (size_t)src * cv.d);
+    const uint4* vs = reinterpret_cast<const uint4*>(Vc + (size_t)src * cv.d);
+    for (int e = lane; e < chunks; e += 32) { kd[e] = ks[e]; vd[e] = vs[e]; }
+    if (lane == 0) { ps.stage_S[so] = Sc[src]; ps.stage_pos[so] = Pc[src]; }
+}
+
+template <typename T>
+__global__ void chunk_evict_scatter_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int seg) {
+    const int unit = blockIdx.y;
+    const int b = unit / cv.Hkv;
+    const int m = lens.m[b];
+    if (m == 0) return;
+    const int N = cv.n_seen[unit];
+    const EvictSegment sg = evict_segment(N, m, cv.c, seg);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int item = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (item >= sg.E + sg.rebase) return;
+    const int dst = item < sg.E ? sg.i + item : cv.c + (item - sg.E);
+    const int chunks = cv.d * (int)sizeof(T) / 16;
+    const size_t so = ((size_t)unit * ps.max_chunk + item);
+    const uint4* ks = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ps.stage_K) + so * cv.d);
+    const uint4* vs = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ps.stage_V) + so * cv.d);
+    uint4* kd = reinterpret_cast<uint4*>(reinterpret_cast<T*>(cv.K) + ((size_t)unit * cv.R + dst) * cv.d);
+    uint4* vd = reinterpret_cast<uint4*>(reinterpret_cast<T*>(cv.V) + ((size_t)unit * cv.R + dst) * cv.d);
+    for (int e = lane; e < chunks; e += 32) { kd[e] = ks[e]; vd[e] = vs[e]; }
+    if (lane == 0) {
+        cv.S[(size_t)unit * cv.R + dst] = ps.stage_S[so];
+        cv.pos[(size_t)unit * cv.R + dst] = ps.stage_pos[so];
+    }
+}
+
+cudaError_t launch_chunk_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
+                               int seg, int max_items, cudaStream_t stream) {
+    if (max_items <= 0) return cudaSuccess;
+    dim3 grid((max_items + 7) / 8, cv.B * cv.Hkv);
+    if (dt == TREEKV_F32) {
+        chunk_evict_gather_kernel<float><<<grid, 256, 0, stream>>>(cv, ps, lens, seg);
+        chunk_evict_scatter_kernel<float><<<grid, 256, 0, stream>>>(cv, ps, lens, seg);
+    } else {
+        chunk_evict_gather_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(cv, ps, lens, seg);
+        chunk_evict_scatter_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(cv, ps, lens, seg);
+    }
+    return cudaGetLastError();
+}
+
+__global__ void chunk_finalize_kernel(CacheView cv, ChunkLens lens) {
+    const int unit = blockIdx.x * blockDim.x + threadIdx.x;
+    if (unit < cv.B * cv.Hkv) cv.n_seen[unit] += lens.m[unit / cv.Hkv];
+}
+cudaError_t launch_chunk_finalize(const CacheView& cv, const ChunkLens& lens, cudaStream_t stream) {
+    const int units = cv.B * cv.Hkv;
+    chunk_finalize_kernel<<<(units + 255) / 256, 256, 0, stream>>>(cv, lens);
+    return cudaGetLastError();
+}
+
+}  // namespace treekv
