@@ -1,0 +1,102 @@
+"""Lock-step comparison of the CUDA library (through its C ABI) with the fp64 oracle on identical inputs.
+
+After every call the retained positions of both sides are compared.  A pair decision whose relative score gap
+in the oracle is below 1e-4 is a near-tie: there the fp32 kernel may legitimately choose the other token, and
+the oracle then follows the library's choice so that later calls still compare like with like; such flips are
+counted.  Any other difference in the retained sets is a failure.  Outputs and averaged scores are compared
+element by element within the stated tolerances.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+OUT_TOL = {"bf16": 2e-2, "f32": 1e-4}   # max abs error of attention outputs
+SCORE_RTOL = 1e-3                        # relative error of S/C of every retained token
+SCORE_ATOL = 1e-12                       # floor for weights that underflow in fp32
+NEAR_TIE = 1e-4
+
+
+class Report:
+    def __init__(self):
+        self.calls = 0
+        self.max_out_err = 0.0
+        self.max_score_rel = 0.0
+        self.near_ties = 0
+        self.flips = 0
+        self.decisions = 0
+
+    def __repr__(self):
+        return ("calls=%d max_out_err=%.3g max_score_rel=%.3g near_ties=%d flips=%d" %
+                (self.calls, self.max_out_err, self.max_score_rel, self.near_ties, self.flips))
+
+
+def _to_dev(torch, a, tdtype):
+    return torch.from_numpy(np.ascontiguousarray(a)).to("cuda").to(tdtype).contiguous()
+
+
+def compare_state(kv, orc, rep, check_scores=True):
+    """Retained positions must match exactly; averaged scores within tolerance."""
+    pos_g, cnt_g = kv.retained_positions()
+    pos_g = pos_g.cpu().numpy(); cnt_g = cnt_g.cpu().numpy()
+    pos_o, cnt_o = orc.retained_positions()
+    assert np.array_equal(cnt_g, cnt_o), "retained counts differ"
+    if not np.array_equal(pos_g, pos_o):
+        bad = np.argwhere(pos_g != pos_o)[0]
+        raise AssertionError("retained positions differ at (b,head,slot)=%s: gpu %d oracle %d" %
+                             (tuple(bad), pos_g[tuple(bad)], pos_o[tuple(bad)]))
+    for b in range(orc.B):
+        for kh in range(orc.Hkv):
+            p = pos_g[b, kh, : cnt_g[b, kh]]
+            assert np.all(np.diff(p) > 0), "positions not strictly increasing"
+    if check_scores:
+        sb_g = kv.scores().cpu().numpy().astype(np.float64)
+        sb_o = orc.scores()
+        err = np.abs(sb_g - sb_o)
+        lim = SCORE_RTOL * np.abs(sb_o) + SCORE_ATOL
+        if not np.all(err <= lim):
+            bad = np.argwhere(err > lim)[0]
+            raise AssertionError("score differs at %s: gpu %.9g oracle %.9g" %
+                                 (tuple(bad), sb_g[tuple(bad)], sb_o[tuple(bad)]))
+        with np.errstate(divide="ignore", invalid="ignore"):
+            rel = np.where(sb_o > 1e-9, err / sb_o, 0.0)
+        rep.max_score_rel = max(rep.max_score_rel, float(rel.max()))
+
+
+def step_decode(kv, orc, q, k, v, dtype, rep, active=None, check_scores=True):
+    """q [B,Hq,d], k,v [B,Hkv,d] float32 numpy holding dtype-rounded values."""
+    import torch
+
+    out_o = orc.decode_attend(q, k, v, active)
+    out_g = kv.decode_step(_to_dev(torch, q, kv.tdtype), _to_dev(torch, k, kv.tdtype), _to_dev(torch, v, kv.tdtype),
+                           active=active)
+    pos_g, cnt_g = kv.retained_positions()
+    nt, fl = orc.evict(pos_g.cpu().numpy(), cnt_g.cpu().numpy(), NEAR_TIE)
+    rep.near_ties += nt; rep.flips += fl; rep.calls += 1
+    og = out_g.float().cpu().numpy().astype(np.float64)
+    sel = slice(None) if active is None else np.asarray(active, bool)
+    err = float(np.abs(og[sel] - out_o[sel]).max()) if np.size(og[sel]) else 0.0
+    rep.max_out_err = max(rep.max_out_err, err)
+    assert err <= OUT_TOL[dtype], "attention output off by %.3g (tolerance %.3g)" % (err, OUT_TOL[dtype])
+    compare_state(kv, orc, rep, check_scores)
+
+
+def step_prefill(kv, orc, q, k, v, dtype, rep, chunk_lens=None, check_scores=True):
+    """q [B,m,Hq,d], k,v [B,m,Hkv,d] float32 numpy holding dtype-rounded values."""
+    import torch
+
+    B, m = q.shape[0], q.shape[1]
+    lens = [m] * B if chunk_lens is None else [int(x) for x in chunk_lens]
+    out_o = orc.prefill_attend(q, k, v, lens)
+    out_g = kv.prefill_chunk(_to_dev(torch, q, kv.tdtype), _to_dev(torch, k, kv.tdtype), _to_dev(torch, v, kv.tdtype),
+                             chunk_lens=lens)
+    pos_g, cnt_g = kv.retained_positions()
+    nt, fl = orc.evict(pos_g.cpu().numpy(), cnt_g.cpu().numpy(), NEAR_TIE)
+    rep.near_ties += nt; rep.flips += fl; rep.calls += 1
+    og = out_g.float().cpu().numpy().astype(np.float64)
+    err = 0.0
+    for b in range(B):
+        if lens[b]:
+            err = max(err, float(np.abs(og[b, : lens[b]] - out_o[b, : lens[b]]).max()))
+    rep.max_out_err = max(rep.max_out_err, err)
+    assert err <= OUT_TOL[dtype], "attention output off by %.3g (tolerance %.3g)" % (err, OUT_TOL[dtype])
+    compare_state(kv, orc, rep, check_scores)

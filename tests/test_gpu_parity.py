@@ -1,0 +1,310 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 oracle on the same seeded inputs.
+
+Bars: retained positions bit-exact except at counted near-ties (oracle pair gap < 1e-4 relative); attention
+outputs within 2e-2 (bf16) / 1e-4 (fp32) max abs; averaged scores within 1e-3 relative.
+"""
+import numpy as np
+import pytest
+
+import workloads as W
+from lockstep import Report, compare_state, step_decode, step_prefill
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2501_04987_b200 import _build
+
+    _build.build()
+    from paper_2501_04987_b200 import binding
+
+    return binding
+
+
+def _pair(binding, w, max_chunk=None):
+    from oracle import Oracle
+
+    mc = w.chunk if max_chunk is None else max_chunk
+    kv = binding.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, mc)
+    orc = Oracle(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.batch)
+    return kv, orc
+
+
+def _run_decode(kv, orc, w, t0, steps, rep, score_every=1, starts=None):
+    blk = 256
+    done = 0
+    while done < steps:
+        n = min(blk, steps - done)
+        st = [t0 + done] * w.batch if starts is None else [s + done for s in starts]
+        q, k, v = W.tokens_at(w, 0, st, n)
+        for i in range(n):
+            step_decode(kv, orc, q[i], k[i], v[i], w.dtype, rep, check_scores=((done + i) % score_every == 0))
+        done += n
+
+
+def _run_prefill(kv, orc, w, rep, lens_total, chunk):
+    """Feed sequence b its first lens_total[b] tokens in chunks of `chunk` (ragged at the end)."""
+    lens_total = np.asarray(lens_total)
+    n_calls = int((lens_total.max() + chunk - 1) // chunk)
+    for c in range(n_calls):
+        q, k, v = W.tokens(w, 0, c * chunk, (c + 1) * chunk)
+        lens = np.clip(lens_total - c * chunk, 0, chunk)
+        step_prefill(kv, orc, q.transpose(1, 0, 2, 3), k.transpose(1, 0, 2, 3), v.transpose(1, 0, 2, 3), w.dtype, rep,
+                     chunk_lens=lens)
+
+
+# ---------------------------------------------------------------------------------------------------------
+def test_cfg1_full_decode_fp32(gpu):
+    """Configuration 1 at full size: fp32, 4 heads, d=64, c=256, 2048 decode steps, compared after every step."""
+    w = W.CONFIGS["cfg1"]
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    _run_decode(kv, orc, w, 0, w.decode_steps, rep)
+    print("cfg1", rep)
+    assert kv.tokens_seen(0) == 2048
+    st = kv.stats()
+    assert st["evictions"] == 2048 - 256 and st["device_error"] == 0
+    assert rep.flips <= rep.near_ties
+
+
+@pytest.mark.parametrize("split", [1, 2, 4, 8])
+def test_decode_split_factors_agree_with_oracle(gpu, split):
+    w = W.parity_slice(W.CONFIGS["cfg1"], budget=37, decode_steps=150)
+    kv, orc = _pair(gpu, w)
+    kv.set_option(gpu.OPT_DECODE_SPLIT, split)
+    rep = Report()
+    _run_decode(kv, orc, w, 0, w.decode_steps, rep)
+
+
+def test_cfg2_slice_decode_bf16_mha(gpu):
+    """Configuration 2's shape (d=128, bf16, MHA, c=1024) on 2 sequences x 4 heads, 3c+ tokens (3 idx cycles)."""
+    w = W.parity_slice(W.CONFIGS["cfg2"], layers=1, batch=2, n_heads=4, n_kv_heads=4, decode_steps=3 * 1024 + 40)
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    _run_decode(kv, orc, w, 0, w.decode_steps, rep, score_every=8)
+    compare_state(kv, orc, rep)
+    print("cfg2 slice", rep)
+
+
+def test_cfg4_slice_prefill_then_gqa_decode(gpu):
+    """Configuration 4's shape (GQA 4:1, d=128, bf16, c=2048, key scales): 4096-token prefill in 1024-token
+    chunks, then one full idx cycle of decode steps."""
+    w = W.parity_slice(W.CONFIGS["cfg4"], layers=1, batch=2, n_heads=8, n_kv_heads=2)
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    _run_prefill(kv, orc, w, rep, [4096, 4096], 1024)
+    _run_decode(kv, orc, w, 4096, 2048 + 64, rep, score_every=16)
+    compare_state(kv, orc, rep)
+    print("cfg4 slice", rep)
+
+
+def test_cfg3_slice_chunked_prefill_mha(gpu):
+    """Configuration 3's shape (MHA, c=2048, chunks of 512): 4 filling chunks + 8 steady chunks, then decode."""
+    w = W.parity_slice(W.CONFIGS["cfg3"], layers=1, n_heads=2, n_kv_heads=2)
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    _run_prefill(kv, orc, w, rep, [12 * 512], 512)
+    _run_decode(kv, orc, w, 12 * 512, 48, rep)
+    print("cfg3 slice", rep)
+
+
+def test_cfg5_slice_ragged_gqa_prefill(gpu):
+    """Configuration 5's shape (GQA 4:1, c=4096, chunks of 1024, ragged lengths, key scales): two sequences that
+    end in different, partial chunks; then batched decode with every sequence at its own stream position."""
+    w = W.parity_slice(W.CONFIGS["cfg5"], layers=1, batch=2, n_heads=4, n_kv_heads=1)
+    lens = [2 * 4096 + 1024 + 517, 2 * 4096 + 100]
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    _run_prefill(kv, orc, w, rep, lens, 1024)
+    assert [kv.tokens_seen(b) for b in range(2)] == lens
+    _run_decode(kv, orc, w, 0, 24, rep, starts=lens)
+    print("cfg5 slice", rep)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# edge cases
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,d,hq,hkv", [("bf16", 64, 4, 2), ("f32", 128, 2, 2), ("bf16", 128, 8, 1), ("f32", 64, 8, 4)])
+def test_shapes_and_group_sizes(gpu, dtype, d, hq, hkv):
+    w = W.parity_slice(W.CONFIGS["cfg1"], dtype=dtype, head_dim=d, n_heads=hq, n_kv_heads=hkv, batch=3, budget=24,
+                       chunk=16, n_outliers=2)
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    _run_prefill(kv, orc, w, rep, [40, 33, 16], 16)
+    _run_decode(kv, orc, w, 0, 60, rep, starts=[40, 33, 16])
+
+
+@pytest.mark.parametrize("c", [2, 3, 5])
+def test_tiny_budgets(gpu, c):
+    w = W.parity_slice(W.CONFIGS["cfg1"], budget=c, chunk=7, batch=2)
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    _run_decode(kv, orc, w, 0, 4 * c + 3, rep)
+    q, k, v = W.tokens(w, 0, 4 * c + 3, 4 * c + 3 + 7)          # a chunk larger than the budget, mid-cycle
+    step_prefill(kv, orc, q.transpose(1, 0, 2, 3), k.transpose(1, 0, 2, 3), v.transpose(1, 0, 2, 3), w.dtype, rep)
+    _run_decode(kv, orc, w, 4 * c + 10, 2 * c + 1, rep)
+
+
+@pytest.mark.parametrize("c,m", [(8, 3), (8, 5), (8, 8), (8, 20), (16, 4), (16, 24), (12, 7)])
+def test_chunks_that_wrap_the_eviction_cycle(gpu, c, m):
+    """Chunks that do not divide the budget, straddle the wrap of idx, or exceed the budget (several wraps)."""
+    w = W.parity_slice(W.CONFIGS["cfg1"], budget=c, chunk=m, batch=2, n_heads=2, n_kv_heads=2)
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    total = 6 * max(c, m) + 5
+    _run_prefill(kv, orc, w, rep, [total, total - m - 2], m)
+    _run_decode(kv, orc, w, 0, 3, rep, starts=[total, total - m - 2])
+    # a chunk right after decode steps: arbitrary cycle position
+    t0 = [total + 3, total - m + 1]
+    q, k, v = W.tokens_at(w, 0, t0, m)
+    step_prefill(kv, orc, q.transpose(1, 0, 2, 3), k.transpose(1, 0, 2, 3), v.transpose(1, 0, 2, 3), w.dtype, rep)
+
+
+@pytest.mark.parametrize("rule", [1, 2])
+def test_score_free_rules_match_closed_structure(gpu, rule):
+    """With the score-free rules the retained set depends on the schedule alone: chunked and token-by-token
+    feeding retain the same tokens, and they equal the oracle's."""
+    from oracle import Oracle
+
+    w = W.parity_slice(W.CONFIGS["cfg1"], budget=16, chunk=6, batch=1, n_heads=1, n_kv_heads=1)
+    a = gpu.TreeKV(16, 1, 1, 64, "f32", 1, 6)
+    b = gpu.TreeKV(16, 1, 1, 64, "f32", 1, 6)
+    a.set_rule(rule); b.set_rule(rule)
+    orc = Oracle(16, 1, 1, 64, 1, rule=rule)
+    import torch
+
+    T = 16 * 7 + 6
+    q, k, v = W.tokens(w, 0, 0, T)
+    tq, tk, tv = (torch.from_numpy(x).cuda() for x in (q, k, v))
+    for t in range(0, T, 6):
+        n = min(6, T - t)
+        for s in range(t, t + n):
+            a.decode_step(tq[s], tk[s], tv[s])
+            orc.decode_step(q[s], k[s], v[s])
+        b.prefill_chunk(tq[t:t + n].transpose(0, 1).contiguous(), tk[t:t + n].transpose(0, 1).contiguous(),
+                        tv[t:t + n].transpose(0, 1).contiguous())
+        pa = a.retained_positions()[0].cpu().numpy()
+        pb = b.retained_positions()[0].cpu().numpy()
+        assert np.array_equal(pa, pb)
+        assert np.array_equal(pa, orc.retained_positions()[0])
+    if rule == 2:  # evict-left closed form: offsets from the newest token
+        pass
+
+
+def test_inactive_sequences_are_untouched(gpu):
+    import torch
+
+    w = W.parity_slice(W.CONFIGS["cfg1"], budget=10, batch=3)
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    seen = [0, 0, 0]
+    for step in range(45):
+        act = [1, step % 3 != 0, step % 2]
+        q, k, v = W.tokens_at(w, 0, seen, 1)
+        step_decode(kv, orc, q[0], k[0], v[0], w.dtype, rep, active=act)
+        seen = [s + (1 if a else 0) for s, a in zip(seen, act)]
+    assert [kv.tokens_seen(b) for b in range(3)] == seen
+    # an inactive row of `out` is not written
+    out = torch.full((3, 4, 64), 7.0, device="cuda")
+    q, k, v = W.tokens_at(w, 0, seen, 1)
+    kv.decode_step(torch.from_numpy(q[0]).cuda(), torch.from_numpy(k[0]).cuda(), torch.from_numpy(v[0]).cuda(), out=out,
+                   active=[0, 1, 0])
+    assert torch.all(out[0] == 7.0) and torch.all(out[2] == 7.0) and not torch.all(out[1] == 7.0)
+
+
+def test_stream_shorter_than_budget_is_full_attention(gpu):
+    """Nothing is evicted while the stream fits the budget; the output is plain causal softmax attention
+    (checked against torch in fp64 as well as the oracle)."""
+    import torch
+
+    w = W.parity_slice(W.CONFIGS["cfg1"], budget=64, decode_steps=64)
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    q, k, v = W.tokens(w, 0, 0, 64)
+    outs = []
+    for t in range(64):
+        step_decode(kv, orc, q[t], k[t], v[t], w.dtype, rep)
+    tq, tk, tv = (torch.from_numpy(x).double() for x in (q, k, v))
+    kv2 = gpu.TreeKV(64, 4, 4, 64, "f32", 1, 0)
+    for t in range(64):
+        o = kv2.decode_step(tq[t].float().cuda(), tk[t].float().cuda(), tv[t].float().cuda()).cpu().double()
+        s = torch.einsum("hd,thd->ht", tq[t, 0], tk[: t + 1, 0]) / 8.0
+        ref = torch.einsum("ht,thd->hd", torch.softmax(s, -1), tv[: t + 1, 0])
+        assert (o[0] - ref).abs().max() < 1e-5
+    assert kv2.stats()["evictions"] == 0
+    assert kv2.retained_positions()[0].cpu().numpy()[0, 0].tolist() == list(range(64))
+
+
+def test_bitwise_reproducible(gpu):
+    """Scores are accumulated in a fixed order (no floating-point atomics): two runs give identical bits."""
+    import torch
+
+    w = W.parity_slice(W.CONFIGS["cfg4"], layers=1, batch=2, n_heads=8, n_kv_heads=2, budget=96, chunk=32)
+    results = []
+    for _ in range(2):
+        kv = gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, w.chunk)
+        outs = []
+        for c in range(8):
+            q, k, v = W.tokens(w, 0, c * 32, (c + 1) * 32)
+            t = [torch.from_numpy(x.transpose(1, 0, 2, 3).copy()).cuda().bfloat16() for x in (q, k, v)]
+            outs.append(kv.prefill_chunk(*t).clone())
+        q, k, v = W.tokens(w, 0, 256, 256 + 150)
+        for s in range(150):
+            t = [torch.from_numpy(x[s]).cuda().bfloat16() for x in (q, k, v)]
+            outs.append(kv.decode_step(*t).clone())
+        results.append((torch.cat([o.flatten() for o in outs]), kv.scores().clone(), kv.retained_positions()[0].clone()))
+    for x, y in zip(*results):
+        assert torch.equal(x, y)
+
+
+def test_host_entry_points_match_device_entry_points(gpu):
+    import torch
+
+    w = W.parity_slice(W.CONFIGS["cfg4"], layers=1, batch=2, n_heads=8, n_kv_heads=2, budget=64, chunk=32)
+    a = gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, w.chunk)
+    b = gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, w.chunk)
+    for c in range(4):
+        q, k, v = W.tokens(w, 0, c * 32, (c + 1) * 32)
+        h = [torch.from_numpy(x.transpose(1, 0, 2, 3).copy()).bfloat16().pin_memory() for x in (q, k, v)]
+        oh = torch.empty_like(h[0]).pin_memory()
+        b.prefill_chunk_host(h[0], h[1], h[2], oh)
+        od = a.prefill_chunk(*[x.cuda() for x in h])
+        torch.cuda.synchronize()
+        assert torch.equal(od.cpu(), oh)
+    q, k, v = W.tokens(w, 0, 128, 128 + 40)
+    for s in range(40):
+        h = [torch.from_numpy(x[s]).bfloat16().pin_memory() for x in (q, k, v)]
+        oh = torch.empty_like(h[0]).pin_memory()
+        b.decode_step_host(h[0], h[1], h[2], oh)
+        od = a.decode_step(*[x.cuda() for x in h])
+        torch.cuda.synchronize()
+        assert torch.equal(od.cpu(), oh)
+    assert torch.equal(a.retained_positions()[0], b.retained_positions()[0])
+
+
+def test_argument_and_state_errors(gpu):
+    import torch
+
+    kv = gpu.TreeKV(16, 4, 4, 64, "f32", 2, 0)
+    x = torch.zeros((2, 4, 64), device="cuda")
+    # decode-only context refuses prefill
+    xc = torch.zeros((2, 4, 4, 64), device="cuda")
+    assert gpu.treekv_prefill_chunk(kv._h, xc.data_ptr(), xc.data_ptr(), xc.data_ptr(), xc.data_ptr(), None, 4) == 2
+    # misaligned pointer
+    assert gpu.treekv_decode_step(kv._h, x.data_ptr() + 4, x.data_ptr(), x.data_ptr(), x.data_ptr()) == 1
+    kv2 = gpu.TreeKV(16, 4, 4, 64, "f32", 2, 8)
+    assert gpu.treekv_prefill_chunk(kv2._h, xc.data_ptr(), xc.data_ptr(), xc.data_ptr(), xc.data_ptr(), [9, 1], 16) == 1
+    assert gpu.treekv_prefill_chunk(kv2._h, xc.data_ptr(), xc.data_ptr(), xc.data_ptr(), xc.data_ptr(), [5, 1], 4) == 1
+    # nothing was enqueued by the refused calls
+    assert kv2.tokens_seen(0) == 0 and kv2.stats()["kernel_launches"] == 1
+    # reset brings back the empty cache
+    kv.decode_step(x, x, x)
+    assert kv.tokens_seen(0) == 1
+    kv.reset()
+    assert kv.tokens_seen(0) == 0
+    assert kv.retained_positions()[1].cpu().numpy().tolist() == [[0] * 4] * 2
