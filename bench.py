@@ -1,0 +1,405 @@
+"""Benchmark of the TreeKV hot path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--workload cfg2] [--impl reference]
+
+Headline (value): decode steps/s on the Llama-2-7B-shaped configuration (32 layers, batch 8, 32 heads, d=128,
+bf16, budget 1024) with every cache full, one step = all 32 layers in order, inputs resident in HBM.
+`e2e`: the same step through the *_host entry points: host->device copies of q,k,v and the device->host copy
+of the output are inside the timed region, every step.
+`prefill`: chunked-prefill tokens/s on the Llama-2-7B-shaped prefill configuration (chunks of 512 to budget
+2048), steady state, with its own roofline entry.
+`roofline`: algorithmic bytes of one decode launch / its average duration, against the measured copy bandwidth.
+`cpu_baseline`: the fp64 oracle timed on this host's cores on a bounded sample of the same workload.
+
+With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no exchange step);
+value is the sum over ranks, timed as the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                    "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+        except Exception:
+            pass
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------------
+# algorithmic bytes / flops (what the method must move or compute)
+# ------------------------------------------------------------------------------------------------------
+def decode_bytes_per_unit(c, d, e, g):
+    """K,V stream + S read/write + appended row + one survivor row read/write + q in, out."""
+    return 2 * (c + 1) * d * e + 8 * (c + 1) + 2 * d * e + 4 * d * e + 2 * g * d * e
+
+
+def prefill_flops_per_head_chunk(m, L, d):
+    """QK^T for the statistics, QK^T again for the probabilities, PV; causal half of the diagonal block not counted."""
+    return 3 * 2 * d * (m * L + m * (m + 1) // 2)
+
+
+# ------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, smmax, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); smmax.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smmax), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def physical_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        ids = [x for x in vis.split(",") if x != ""]
+        if local_rank < len(ids) and ids[local_rank].isdigit():
+            return int(ids[local_rank])
+    return local_rank
+
+
+# ------------------------------------------------------------------------------------------------------
+# oracle timing (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------------
+def time_oracle_decode(w, seqs, steps):
+    """Oracle decode steps/s for the whole configuration, from a sample of `seqs` sequences of one layer with
+    full caches.  Returns (steps_per_s_full_config, cores, description)."""
+    from oracle import Oracle
+
+    ws = W.parity_slice(w, layers=1, batch=seqs)
+    orc = Oracle(ws.budget, ws.n_heads, ws.n_kv_heads, ws.head_dim, ws.batch)
+    # fill the caches with one causal chunk pass per 256 tokens (not timed)
+    t = 0
+    while t < ws.budget:
+        n = min(256, ws.budget - t)
+        q, k, v = W.tokens(ws, 0, t, t + n)
+        orc.prefill_chunk(q.transpose(1, 0, 2, 3), k.transpose(1, 0, 2, 3), v.transpose(1, 0, 2, 3))
+        t += n
+    q, k, v = W.tokens(ws, 0, t, t + steps)
+    q, k, v = (np.ascontiguousarray(x, dtype=np.float64) for x in (q, k, v))
+    t0 = time.perf_counter()
+    for s in range(steps):
+        orc.decode_step(q[s], k[s], v[s])
+    dt = time.perf_counter() - t0
+    layer_seq_steps_per_s = steps * seqs / dt
+    full = layer_seq_steps_per_s / (w.layers * w.batch)
+    cores = len(os.sched_getaffinity(0))
+    desc = ("oracle decode on %d of %d sequences of 1 of %d layers, caches full, %d steps in %.1f s; scaled by "
+            "(layers*batch)/(sample sequences) = %g" % (seqs, w.batch, w.layers, steps, dt, w.layers * w.batch / seqs))
+    return full, cores, desc
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import build_oracle
+
+    build_oracle()
+    seqs = min(2, w.batch)
+    steps = max(1, args.steps)
+    for _ in range(1):
+        pass
+    # warm-up steps are part of the cache fill; each "step" of this arm is one oracle decode step of the sample
+    val, cores, desc = time_oracle_decode(w, seqs, min(steps, 400))
+    line = {
+        "metric": "treekv_decode_steps_per_s", "value": val, "unit": "steps/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1000.0 / val, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+        "config": {"workload": w.name, "layers": w.layers, "batch": w.batch, "n_heads": w.n_heads,
+                   "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "budget": w.budget},
+        "cpu_baseline": {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=512)
+    ap.add_argument("--warmup", type=int, default=16)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg4"])
+    ap.add_argument("--prefill-workload", default="cfg3", choices=["cfg3", "cfg5"])
+    ap.add_argument("--prefill-chunks", type=int, default=4, help="timed steady-state chunks (0 = skip the prefill leg)")
+    ap.add_argument("--e2e-steps", type=int, default=64)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling small cases)")
+    args = ap.parse_args()
+
+    w = W.CONFIGS[args.workload]
+    if args.layers:
+        w = W.parity_slice(w, layers=args.layers)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2501_04987_b200 import _build
+
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2501_04987_b200 import binding
+
+    peaks = measured_peaks()
+    e = 2 if w.dtype == "bf16" else 4
+    tdtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    g = w.group
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ------------------------------------------------------------------ decode leg
+    wr = W.parity_slice(w, seed=w.seed + 1000 * rank)
+    ctxs = [binding.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, 0) for _ in range(w.layers)]
+    ring = 4
+    ins = []
+    for layer in range(w.layers):
+        # every cache will be full and mid-cycle when timing starts; the ring holds positions near there
+        q, k, v = W.tokens(wr, layer, w.budget + 37, w.budget + 37 + ring)
+        ins.append(tuple(torch.from_numpy(x).to(dev).to(tdtype).contiguous() for x in (q, k, v)))
+    outs = [torch.empty((w.batch, w.n_heads, w.head_dim), dtype=tdtype, device=dev) for _ in range(w.layers)]
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def decode_steps(n, start):
+        for s in range(start, start + n):
+            r = s % ring
+            for layer in range(w.layers):
+                q, k, v = ins[layer]
+                st = binding.lib.treekv_decode_step(ctxs[layer]._h, q[r].data_ptr(), k[r].data_ptr(), v[r].data_ptr(),
+                                                    outs[layer].data_ptr(), None, stream)
+                if st != 0:
+                    raise RuntimeError("treekv_decode_step: " + binding.status_string(st))
+
+    fill = w.budget + 37
+    decode_steps(fill, 0)                      # fill every cache (untimed)
+    decode_steps(max(3, args.warmup), fill)    # warm-up
+    launches0 = sum(c.stats()["kernel_launches"] for c in ctxs)
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    barrier()
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    decode_steps(args.steps, fill + args.warmup)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    launches = sum(c.stats()["kernel_launches"] for c in ctxs) - launches0
+    ms_per_step = ms_total / args.steps
+    steps_per_s = world * 1000.0 / ms_per_step
+
+    units = w.batch * w.n_kv_heads
+    bytes_per_launch = units * decode_bytes_per_unit(w.budget, w.head_dim, e, g)
+    launch_ms = ms_total / (args.steps * w.layers)
+    achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "kernel": "decode_kernel", "bytes_per_launch": bytes_per_launch, "launch_us": launch_ms * 1e3,
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # ------------------------------------------------------------------ e2e leg: host buffers through the C ABI
+    nb_q = w.batch * w.n_heads * w.head_dim * e
+    nb_k = w.batch * w.n_kv_heads * w.head_dim * e
+    h_in = [tuple(x.cpu().pin_memory() for x in ins[layer]) for layer in range(w.layers)]
+    h_out = [torch.empty((w.batch, w.n_heads, w.head_dim), dtype=tdtype).pin_memory() for _ in range(w.layers)]
+
+    def e2e_steps(n):
+        for s in range(n):
+            r = s % ring
+            for layer in range(w.layers):
+                q, k, v = h_in[layer]
+                st = binding.lib.treekv_decode_step_host(ctxs[layer]._h, q[r].data_ptr(), k[r].data_ptr(),
+                                                         v[r].data_ptr(), h_out[layer].data_ptr(), None, stream)
+                if st != 0:
+                    raise RuntimeError("treekv_decode_step_host: " + binding.status_string(st))
+
+    e2e_n = max(1, min(args.e2e_steps, args.steps))
+    e2e_steps(3)
+    barrier()
+    ev0.record()
+    e2e_steps(e2e_n)
+    ev1.record()
+    barrier()
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_n
+    e2e = {"value": world * 1000.0 / e2e_ms, "unit": "steps/s", "h2d_bytes_per_step": w.layers * (nb_q + 2 * nb_k),
+           "d2h_bytes_per_step": w.layers * nb_q, "steps": e2e_n, "ms_per_step": e2e_ms}
+    del ctxs, ins, outs
+    torch.cuda.empty_cache()
+
+    # ------------------------------------------------------------------ prefill leg
+    prefill = None
+    if args.prefill_chunks > 0:
+        pw = W.CONFIGS[args.prefill_workload]
+        if args.layers:
+            pw = W.parity_slice(pw, layers=args.layers)
+        prefill = run_prefill_leg(torch, binding, pw, args.prefill_chunks, dev, world, rank, barrier, max_over_ranks, peaks)
+
+    # ------------------------------------------------------------------ oracle on the host cores
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        val, cores, desc = time_oracle_decode(w, min(2, w.batch), 300)
+        cpu_baseline = {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        line = {
+            "metric": "treekv_decode_steps_per_s", "value": steps_per_s, "unit": "steps/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": w.name, "layers": w.layers, "batch_per_gpu": w.batch, "n_heads": w.n_heads,
+                       "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "budget": w.budget,
+                       "parallelism": "replicas x%d" % world,
+                       "l2": "no flush: one step streams %.2f GB of K/V (%.0f MB per layer) through a 126 MB L2"
+                             % (w.layers * bytes_per_launch / 1e9, bytes_per_launch / 1e6)},
+            "tokens_per_s": steps_per_s * w.batch,
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
+            "cpu_baseline": cpu_baseline, "prefill": prefill,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_prefill_leg(torch, binding, pw, n_chunks, dev, world, rank, barrier, max_over_ranks, peaks):
+    tdtype = torch.bfloat16 if pw.dtype == "bf16" else torch.float32
+    m, c = pw.chunk, pw.budget
+    ctxs = [binding.TreeKV(c, pw.n_heads, pw.n_kv_heads, pw.head_dim, pw.dtype, pw.batch, m) for _ in range(pw.layers)]
+    wr = W.parity_slice(pw, seed=pw.seed + 1000 * rank)
+    ring = 2
+    ins = []
+    for layer in range(pw.layers):
+        chunks = []
+        for r in range(ring):
+            q, k, v = W.tokens(wr, layer, c + r * m, c + (r + 1) * m)
+            chunks.append(tuple(torch.from_numpy(np.ascontiguousarray(x.transpose(1, 0, 2, 3))).to(dev).to(tdtype)
+                                for x in (q, k, v)))
+        ins.append(chunks)
+    out = torch.empty((pw.batch, m, pw.n_heads, pw.head_dim), dtype=tdtype, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def run(n, start):
+        for s in range(start, start + n):
+            for layer in range(pw.layers):
+                q, k, v = ins[layer][s % ring]
+                st = binding.lib.treekv_prefill_chunk(ctxs[layer]._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                                      out.data_ptr(), None, m, stream)
+                if st != 0:
+                    raise RuntimeError("treekv_prefill_chunk: " + binding.status_string(st))
+
+    fill_chunks = c // m
+    run(fill_chunks + 3, 0)  # fill the caches, then three steady chunks as warm-up
+    launches0 = sum(x.stats()["kernel_launches"] for x in ctxs)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    run(n_chunks, fill_chunks + 3)
+    ev1.record()
+    barrier()
+    ms = max_over_ranks(ev0.elapsed_time(ev1))
+    launches = sum(x.stats()["kernel_launches"] for x in ctxs) - launches0
+    tok_s = world * n_chunks * m * pw.batch / (ms * 1e-3)
+    flops_chunk = pw.layers * pw.batch * pw.n_heads * prefill_flops_per_head_chunk(m, c, pw.head_dim)
+    achieved = flops_chunk * n_chunks / (ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    return {"metric": "treekv_prefill_tokens_per_s", "value": tok_s, "unit": "tokens/s", "chunks": n_chunks,
+            "ms_per_chunk_all_layers": ms / n_chunks, "gpu_launches": int(launches),
+            "config": {"workload": pw.name, "layers": pw.layers, "batch_per_gpu": pw.batch, "n_heads": pw.n_heads,
+                       "n_kv_heads": pw.n_kv_heads, "head_dim": pw.head_dim, "budget": c, "chunk": m},
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                         "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " (sustained)",
+                         "flops_per_chunk_all_layers": flops_chunk}}
+
+
+if __name__ == "__main__":
+    main()
