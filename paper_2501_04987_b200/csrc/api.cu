@@ -5,27 +5,9 @@
 #include <string.h>
 
 #include "common.cuh"
+#include "ctx.cuh"
 
 using namespace treekv;
-
-struct treekv_ctx {
-    CacheView cv;
-    PrefillScratch ps;
-    treekv_dtype dt;
-    int max_chunk;
-    int G;
-    size_t elem;
-    // staging for the *_host entry points
-    void *st_q, *st_k, *st_v, *st_out;
-    // options
-    int opt_decode_split;
-    int opt_prefill_path;
-    // host-side record
-    int64_t n_seen[kMaxBatch];
-    uint64_t evictions;
-    uint64_t launches;
-    int last_cuda_error;
-};
 
 namespace {
 

@@ -1,0 +1,23 @@
+// Host-side context of one TreeKV layer (private to the library's .cu files).
+#pragma once
+
+#include "common.cuh"
+
+struct treekv_ctx {
+    treekv::CacheView cv;
+    treekv::PrefillScratch ps;
+    treekv_dtype dt;
+    int max_chunk;
+    int G;
+    size_t elem;
+    // staging for the *_host entry points
+    void *st_q, *st_k, *st_v, *st_out;
+    // options
+    int opt_decode_split;
+    int opt_prefill_path;
+    // host-side record
+    int64_t n_seen[treekv::kMaxBatch];
+    uint64_t evictions;
+    uint64_t launches;
+    int last_cuda_error;
+};
