@@ -135,6 +135,33 @@ treekv_status treekv_prefill_chunk_host(treekv_ctx* ctx, const void* host_q, con
                                         int chunk_stride, void* stream);
 
 /*
+ * treekv_prefill_chunk for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * is a deployment variant of the call above, not a different computation.)
+ *
+ * Same arguments, same effect on the cache and the same dev_out as treekv_prefill_chunk, but none of the
+ * call's scratch (partial column sums, rows staged during compaction) is taken from the workspace: it lives
+ * in a fixed 16 MiB area that is part of the library image on every GPU that has loaded the library, from
+ * load until the process exits.  It is meant for code that may not call cudaMalloc at the point where it
+ * runs - a server that has frozen its memory pool, a plug-in inside another framework's allocator, a loop
+ * that cannot take cudaMalloc's device-wide synchronisation - and so cannot size scratch per call.  The
+ * entry point itself calls no allocating routine.
+ *   - Limit: with u = batch * n_kv_heads, m = the longest chunk of this call, g = n_heads / n_kv_heads and
+ *     e = element size, it needs  u * (ceil(g*m/128) * (budget + m) * 4  +  2 * m * head_dim * e  +  8 * m)
+ *     bytes (each of the five parts rounded up to 256); beyond 16 MiB it returns TREEKV_ERR_UNSUPPORTED and
+ *     enqueues nothing.
+ *   - The first call on a device looks up the area's device address (once per device, with that device
+ *     current); make that first call outside any stream capture.
+ *   - Every context of the process shares the one area of its GPU, and the area keeps whatever the last call
+ *     left.  A call never reads a slot it has not itself written first, so nothing needs clearing between
+ *     calls; but two calls that overlap on the GPU (issued on different streams, whether for the same context
+ *     or for different ones) race on it.  Keep calls to this entry point ordered on one stream, or serialise
+ *     them some other way.
+ */
+treekv_status treekv_prefill_chunk_static_scratch(treekv_ctx* ctx, const void* dev_q, const void* dev_k,
+                                                  const void* dev_v, void* dev_out,
+                                                  const int32_t* host_chunk_lens, int chunk_stride, void* stream);
+
+/*
  * Stream positions of the retained tokens (what Figures 1 and 3 draw), in cache order, i.e. strictly increasing.
  *   dev_pos    [batch][n_kv_heads][budget] int32, unused tail filled with -1
  *   dev_count  [batch][n_kv_heads] int32, number of retained tokens (= min(tokens seen, budget))

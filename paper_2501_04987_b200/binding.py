@@ -21,7 +21,7 @@ OPT_DECODE_SPLIT, OPT_PREFILL_PATH = 0, 1
 # every symbol include/treekv.h declares
 EXPORTS = [
     "treekv_workspace_bytes", "treekv_create", "treekv_decode_step", "treekv_prefill_chunk",
-    "treekv_decode_step_host", "treekv_prefill_chunk_host", "treekv_retained_positions", "treekv_scores",
+    "treekv_decode_step_host", "treekv_prefill_chunk_host", "treekv_prefill_chunk_static_scratch", "treekv_retained_positions", "treekv_scores",
     "treekv_get_stats", "treekv_tokens_seen", "treekv_set_rule", "treekv_set_option", "treekv_reset",
     "treekv_destroy", "treekv_status_string", "treekv_version",
 ]
@@ -63,6 +63,8 @@ def _load():
     lib.treekv_prefill_chunk.argtypes = [vp, vp, vp, vp, vp, C.POINTER(C.c_int32), i32, vp]
     lib.treekv_prefill_chunk_host.restype = i32
     lib.treekv_prefill_chunk_host.argtypes = [vp, vp, vp, vp, vp, C.POINTER(C.c_int32), i32, vp]
+    lib.treekv_prefill_chunk_static_scratch.restype = i32
+    lib.treekv_prefill_chunk_static_scratch.argtypes = [vp, vp, vp, vp, vp, C.POINTER(C.c_int32), i32, vp]
     lib.treekv_retained_positions.restype = i32
     lib.treekv_retained_positions.argtypes = [vp, vp, vp, vp]
     lib.treekv_scores.restype = i32
@@ -137,6 +139,12 @@ def treekv_prefill_chunk(ctx, q, k, v, out, chunk_lens, chunk_stride, stream=0) 
 
 def treekv_prefill_chunk_host(ctx, q, k, v, out, chunk_lens, chunk_stride, stream=0) -> int:
     return lib.treekv_prefill_chunk_host(ctx, q, k, v, out, _i32(chunk_lens), chunk_stride, stream)
+
+
+def treekv_prefill_chunk_static_scratch(ctx, q, k, v, out, chunk_lens, chunk_stride, stream=0) -> int:
+    """treekv_prefill_chunk with its scratch in the library's fixed 16 MiB device area: for callers that cannot
+    allocate device memory where they run.  Calls sharing a GPU must not overlap."""
+    return lib.treekv_prefill_chunk_static_scratch(ctx, q, k, v, out, _i32(chunk_lens), chunk_stride, stream)
 
 
 def treekv_retained_positions(ctx, dev_pos, dev_count, stream=0) -> int:
