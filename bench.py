@@ -192,6 +192,7 @@ def main():
     ap.add_argument("--prefill-chunks", type=int, default=4, help="timed steady-state chunks (0 = skip the prefill leg)")
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-split", type=int, default=0, help="thread blocks per (sequence, KV head); 0 = automatic")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling small cases)")
     args = ap.parse_args()
 
@@ -242,6 +243,9 @@ def main():
     # ------------------------------------------------------------------ decode leg
     wr = W.parity_slice(w, seed=w.seed + 1000 * rank)
     ctxs = [binding.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, 0) for _ in range(w.layers)]
+    if args.decode_split:
+        for c in ctxs:
+            c.set_option(binding.OPT_DECODE_SPLIT, args.decode_split)
     ring = 4
     ins = []
     for layer in range(w.layers):

@@ -31,6 +31,7 @@ bool shape_ok(int budget, int n_heads, int n_kv_heads, int head_dim, treekv_dtyp
     if (max_chunk < 0 || max_chunk > 8192) return false;
     if (n_kv_heads > 65535 || (long long)batch * n_kv_heads > 65535) return false;  // grid.y of the per-unit kernels
     if (decode_smem_bytes(G, head_dim, budget, 8) > kSmemLimit) return false;
+    if (dt == TREEKV_BF16 && decode_mma_smem_bytes(G, head_dim, budget, 8) > kSmemLimit) return false;
     if (max_chunk > 0 && prefill_simt_smem_bytes(G, head_dim, budget + max_chunk) > kSmemLimit) return false;
     return true;
 }
@@ -72,14 +73,31 @@ treekv_status cuda_fail(treekv_ctx* ctx, cudaError_t e) {
     return TREEKV_ERR_CUDA;
 }
 
+bool use_mma_decode(const treekv_ctx* ctx) {
+    if (ctx->dt != TREEKV_BF16) return false;
+    return ctx->opt_decode_path != 1;
+}
+
+size_t decode_smem_for(const treekv_ctx* ctx, int split) {
+    return use_mma_decode(ctx) ? decode_mma_smem_bytes(ctx->G, ctx->cv.d, ctx->cv.c, split)
+                               : decode_smem_bytes(ctx->G, ctx->cv.d, ctx->cv.c, split);
+}
+
+// Thread blocks (cluster size) per unit.  The bf16 kernel keeps one CTA per unit once there are at least as many
+// units as SMs (its CTAs are small and several are resident per SM) and otherwise splits until the machine is
+// covered about twice; the CUDA-core kernel splits while a CTA keeps at least 128 rows.
 int pick_decode_split(const treekv_ctx* ctx) {
     const int c = ctx->cv.c, units = ctx->cv.B * ctx->cv.Hkv;
     int s = ctx->opt_decode_split;
     if (s == 0) {
         s = 1;
-        while (s < 8 && units * s < 444 && (c + 1) / (2 * s) >= 128) s *= 2;
+        if (use_mma_decode(ctx)) {
+            while (s < 8 && units * (2 * s) <= 2 * ctx->sm_count && (c + 1) / (2 * s) >= 64) s *= 2;
+        } else {
+            while (s < 8 && units * s < 3 * ctx->sm_count && (c + 1) / (2 * s) >= 128) s *= 2;
+        }
     }
-    while (s < 8 && decode_smem_bytes(ctx->G, ctx->cv.d, c, s) > kSmemLimit) s *= 2;
+    while (s < 8 && decode_smem_for(ctx, s) > kSmemLimit) s *= 2;
     return s;
 }
 
@@ -122,6 +140,13 @@ treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_
     ctx->st_q = base + L.st_q; ctx->st_k = base + L.st_k; ctx->st_v = base + L.st_v; ctx->st_out = base + L.st_out;
     ctx->dt = dtype; ctx->max_chunk = max_chunk; ctx->G = n_heads / n_kv_heads;
     ctx->elem = dtype == TREEKV_F32 ? 4 : 2;
+    {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            sms = 148;
+        ctx->sm_count = sms;
+    }
     const cudaError_t e = launch_init_state(ctx->cv, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { delete ctx; return TREEKV_ERR_CUDA; }
     ctx->launches = 1;
@@ -156,8 +181,12 @@ treekv_status treekv_decode_step(treekv_ctx* ctx, const void* dev_q, const void*
         }
     }
     if (n_active == 0) return TREEKV_OK;
-    const cudaError_t e = launch_decode(ctx->cv, ctx->dt, dev_q, dev_k, dev_v, dev_out, mask, pick_decode_split(ctx),
-                                        static_cast<cudaStream_t>(stream));
+    const cudaError_t e =
+        use_mma_decode(ctx)
+            ? launch_decode_mma(ctx->cv, dev_q, dev_k, dev_v, dev_out, mask, pick_decode_split(ctx),
+                                static_cast<cudaStream_t>(stream))
+            : launch_decode(ctx->cv, ctx->dt, dev_q, dev_k, dev_v, dev_out, mask, pick_decode_split(ctx),
+                            static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     for (int b = 0; b < ctx->cv.B; ++b) {
@@ -308,8 +337,14 @@ treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value) {
     switch (opt) {
         case TREEKV_OPT_DECODE_SPLIT:
             if (!(value == 0 || value == 1 || value == 2 || value == 4 || value == 8)) return TREEKV_ERR_INVALID_ARG;
-            if (value && decode_smem_bytes(ctx->G, ctx->cv.d, ctx->cv.c, value) > kSmemLimit) return TREEKV_ERR_UNSUPPORTED;
+            if (value && decode_smem_for(ctx, value) > kSmemLimit) return TREEKV_ERR_UNSUPPORTED;
             ctx->opt_decode_split = value;
+            return TREEKV_OK;
+        case TREEKV_OPT_DECODE_PATH:
+            if (value < 0 || value > 2) return TREEKV_ERR_INVALID_ARG;
+            if (value == 2 && ctx->dt != TREEKV_BF16) return TREEKV_ERR_UNSUPPORTED;
+            ctx->opt_decode_path = value;
+            ctx->opt_decode_split = 0;
             return TREEKV_OK;
         case TREEKV_OPT_PREFILL_PATH:
             if (value < 0 || value > 2) return TREEKV_ERR_INVALID_ARG;

@@ -156,6 +156,10 @@ size_t decode_smem_bytes(int G, int D, int c, int split);
 cudaError_t launch_decode(const CacheView& cv, treekv_dtype dt, const void* q, const void* k, const void* v, void* out,
                           const ActiveMask& active, int split, cudaStream_t stream);
 
+size_t decode_mma_smem_bytes(int G, int D, int c, int split);
+cudaError_t launch_decode_mma(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+                              const ActiveMask& active, int split, cudaStream_t stream);
+
 cudaError_t launch_init_state(const CacheView& cv, cudaStream_t stream);
 cudaError_t launch_retained_positions(const CacheView& cv, int32_t* pos_out, int32_t* count_out, cudaStream_t stream);
 cudaError_t launch_scores(const CacheView& cv, float* sbar_out, cudaStream_t stream);

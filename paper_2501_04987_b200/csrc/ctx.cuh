@@ -15,6 +15,8 @@ struct treekv_ctx {
     // options
     int opt_decode_split;
     int opt_prefill_path;
+    int opt_decode_path;
+    int sm_count;
     // host-side record
     int64_t n_seen[treekv::kMaxBatch];
     uint64_t evictions;

@@ -1,0 +1,413 @@
+// Decode step of TreeKV for bf16 caches (Algorithm 1, one loop iteration; attention of Section 3.1), one launch.
+//
+// Same contract as decode.cu, built for bandwidth with grouped queries: a cluster of `split` CTAs owns one
+// unit (sequence, KV head); inside a CTA every warp runs a private pipeline
+//     cp.async (16-byte, L2-only) of 16 K rows + 16 V rows into its ring of shared-memory stages
+//  -> ldmatrix -> mma.sync m16n8k16 for q.K^T of all G heads of the group at once
+//  -> online softmax in registers (running max, lazy rescale)
+//  -> ldmatrix.trans -> mma.sync for P.V with P taken straight from the logits' accumulator registers.
+// K and V are read from HBM exactly once, there is no block-wide barrier inside the streaming loop, and the
+// instruction count per byte does not grow with the group size (the G query heads ride in the N=8 / M=16
+// dimensions of the MMA tiles).  Logits are kept in shared memory; every CTA pushes its (max, sum) to all CTAs
+// of the cluster and its partial output to CTA 0 with remote shared-memory stores, so that after one cluster
+// barrier each CTA can write the exact normalised probabilities' group mean into S and CTA 0 can write the
+// output.  CTA 0 then plays Algorithm 1's eviction branch.
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace treekv {
+
+namespace {
+
+__device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ inline void cp_async_16(uint32_t dst, const void* src, bool valid) {
+    const int sz = valid ? 16 : 0;  // src-size 0: the 16 destination bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ inline void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ inline void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ inline void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ inline void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ inline void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ inline uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// 2^(a-b) with the convention 2^(-inf - anything) = 0, so empty partials (max = -inf) never produce NaN
+__device__ inline float exp2_diff(float a, float b) { return a == -INFINITY ? 0.f : exp2f(a - b); }
+
+constexpr int kBlk = 16;      // keys per pipeline stage
+constexpr int kMaxSplit = 8;  // largest cluster
+constexpr int kMmaWarps = 4;
+constexpr int kMmaStages = 2;
+
+int mma_rows_cap(int c, int split) {
+    const int nblk_all = (c + 1 + kBlk - 1) / kBlk;
+    return ((nblk_all + split - 1) / split) * kBlk;
+}
+
+}  // namespace
+
+template <int D, int G, int NW, int NS>
+__global__ void __launch_bounds__(NW * 32)
+decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_in,
+                  const __nv_bfloat16* __restrict__ v_in, __nv_bfloat16* __restrict__ out, ActiveMask active,
+                  int rows_cap) {
+    using T = __nv_bfloat16;
+    constexpr int NT = NW * 32;
+    constexpr int ROWB = D * 2;             // bytes per row
+    constexpr int CPR = ROWB / 16;          // 16-byte chunks per row
+    constexpr int STAGE = 2 * kBlk * ROWB;  // K block + V block
+    constexpr int CHUNKS = D * 2 / 16;
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int nsplit = (int)cluster.num_blocks();
+    const int kh = blockIdx.y, b = blockIdx.z;
+    if (!active.test(b)) return;  // the whole cluster shares b
+
+    const int unit = b * cv.Hkv + kh;
+    const int N = cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv.c);
+    const int n = st.L + 1;  // live rows including the token appended by this step
+    const int i_cyc = st.i;
+    // rows are dealt to the cluster in whole 16-key blocks
+    const int nblk_all = (n + kBlk - 1) / kBlk;
+    const int blk_per = (nblk_all + nsplit - 1) / nsplit;
+    const int lo = min(rank * blk_per * kBlk, n), hi = min(lo + blk_per * kBlk, n);
+    const int nrows = hi - lo;
+    const int nblk = (nrows + kBlk - 1) / kBlk;
+    const bool owns_new = (hi == n) && nrows > 0;
+
+    T* Kc = reinterpret_cast<T*>(cv.K) + (size_t)unit * cv.R * D;
+    T* Vc = reinterpret_cast<T*>(cv.V) + (size_t)unit * cv.R * D;
+    float* Sc = cv.S + (size_t)unit * cv.R;
+    int32_t* Pc = cv.pos + (size_t)unit * cv.R;
+    const T* k_new = k_in + (size_t)unit * D;
+    const T* v_new = v_in + (size_t)unit * D;
+    const int new_row = st.L + i_cyc;
+
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* ring = smem_raw;                                        // [NW][NS][STAGE]
+    float* sl = reinterpret_cast<float*>(ring + (size_t)NW * NS * STAGE);  // [G][rows_cap] logits (log2 units)
+    float* wstat = sl + (size_t)G * rows_cap;                              // [NW+1][2][G] per-warp (max, sum); slot NW = new token
+    float* gstat = wstat + (NW + 1) * 2 * G;                               // [nsplit][2][G] every CTA's (max, sum), pushed by its owner
+    float* o_all = gstat + kMaxSplit * 2 * G;                              // [nsplit][G][D] partial outputs, pushed into CTA 0 only
+    float* o_warp = reinterpret_cast<float*>(ring);                        // [NW][G][D], aliases the ring after the loop
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const float scale = kLog2e * rsqrtf((float)D);
+
+    // ---- append (Algorithm 1: K <- K u {k}, V <- V u {v}); the step itself reads the new token from k_in / v_in
+    if (owns_new && warp == NW - 1) {
+        for (int e = lane; e < CHUNKS; e += 32) {
+            reinterpret_cast<uint4*>(Kc + (size_t)new_row * D)[e] = ld_plain(reinterpret_cast<const uint4*>(k_new) + e);
+            reinterpret_cast<uint4*>(Vc + (size_t)new_row * D)[e] = ld_plain(reinterpret_cast<const uint4*>(v_new) + e);
+        }
+    }
+
+    const uint32_t ring_w = smem_u32(ring) + warp * NS * STAGE;
+    auto issue = [&](int blk, int stage) {
+        if (blk < nblk) {
+            const uint32_t kst = ring_w + stage * STAGE, vst = kst + kBlk * ROWB;
+#pragma unroll
+            for (int it = 0; it < kBlk * CPR / 32; ++it) {
+                const int x = it * 32 + lane;
+                const int row = x / CPR, cidx = x % CPR;
+                const int lam = lo + blk * kBlk + row;
+                const bool valid = lam < hi && lam != n - 1;  // the new token is merged separately
+                const size_t ro = valid ? (size_t)phys_row(lam, i_cyc) * D : 0;
+                const uint32_t off = row * ROWB + ((cidx ^ (row & 7)) << 4);
+                cp_async_16(kst + off, reinterpret_cast<const unsigned char*>(Kc + ro) + cidx * 16, valid);
+                cp_async_16(vst + off, reinterpret_cast<const unsigned char*>(Vc + ro) + cidx * 16, valid);
+            }
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int s = 0; s < NS; ++s) issue(warp + s * NW, s);
+
+    // ---- A fragments of q: row g = head, k = channel; rows >= G are zero
+    uint32_t qa[D / 16][2];
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+        qa[kk][0] = 0u; qa[kk][1] = 0u;
+        if (g < G) {
+            const T* qh = q + ((size_t)b * cv.Hq + kh * G + g) * D + 16 * kk + 2 * t;
+            qa[kk][0] = *reinterpret_cast<const uint32_t*>(qh);
+            qa[kk][1] = *reinterpret_cast<const uint32_t*>(qh + 8);
+        }
+    }
+
+    float m_run = -INFINITY, l_run = 0.f;  // of head g (replicated over the 4 lanes t; l_run is a per-lane partial)
+    float acc[D / 16][4];
+#pragma unroll
+    for (int cc = 0; cc < D / 16; ++cc)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[cc][e] = 0.f;
+
+    for (int it = 0;; ++it) {
+        const int blk = warp + it * NW;
+        if (blk >= nblk) break;
+        const int stage = it % NS;
+        cp_async_wait<NS - 1>();
+        __syncwarp();
+        const uint32_t kst = ring_w + stage * STAGE, vst = kst + kBlk * ROWB;
+
+        // ---- logits of 16 keys x G heads
+        float c[2][4];
+#pragma unroll
+        for (int hb = 0; hb < 2; ++hb)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) c[hb][e] = 0.f;
+#pragma unroll
+        for (int u = 0; u < D / 32; ++u) {
+#pragma unroll
+            for (int hb = 0; hb < 2; ++hb) {
+                const int row = hb * 8 + (lane & 7), cidx = 4 * u + (lane >> 3);
+                uint32_t r0, r1, r2, r3;
+                ldmatrix_x4(kst + row * ROWB + ((cidx ^ (row & 7)) << 4), r0, r1, r2, r3);
+                mma_bf16(c[hb], qa[2 * u][0], 0u, qa[2 * u][1], 0u, r0, r1);
+                mma_bf16(c[hb], qa[2 * u + 1][0], 0u, qa[2 * u + 1][1], 0u, r2, r3);
+            }
+        }
+        // lane (g,t) holds head g, keys 2t, 2t+1 (c[0]) and 8+2t, 9+2t (c[1]) of the block
+        float s4[4] = {c[0][0] * scale, c[0][1] * scale, c[1][0] * scale, c[1][1] * scale};
+        const int key0 = blk * kBlk + 2 * t;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int key = key0 + (e & 1) + (e >> 1) * 8;
+            const int lam = lo + key;
+            if (!(lam < hi && lam != n - 1)) s4[e] = -INFINITY;
+            if (g < G && key < nrows) sl[g * rows_cap + key] = s4[e];
+        }
+        float bm = fmaxf(fmaxf(s4[0], s4[1]), fmaxf(s4[2], s4[3]));
+        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
+        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
+        const float m_new = fmaxf(m_run, bm);
+        if (__any_sync(0xffffffffu, m_new > m_run)) {
+            const float corr = (m_new == -INFINITY) ? 1.f : exp2_diff(m_run, m_new);
+            l_run *= corr;
+            m_run = m_new;
+            const float c0 = __shfl_sync(0xffffffffu, corr, (2 * t) * 4);      // head 2t   (columns of acc)
+            const float c1 = __shfl_sync(0xffffffffu, corr, (2 * t + 1) * 4);  // head 2t+1
+#pragma unroll
+            for (int cc = 0; cc < D / 16; ++cc) { acc[cc][0] *= c0; acc[cc][1] *= c1; acc[cc][2] *= c0; acc[cc][3] *= c1; }
+        }
+        float p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) p[e] = (m_run == -INFINITY) ? 0.f : exp2_diff(s4[e], m_run);
+        l_run += (p[0] + p[1]) + (p[2] + p[3]);
+        const uint32_t pb0 = pack_bf16(p[0], p[1]), pb1 = pack_bf16(p[2], p[3]);
+
+        // ---- o^T[ch][head] += V^T[ch][key] P^T[key][head]
+#pragma unroll
+        for (int cc = 0; cc < D / 16; ++cc) {
+            const int row = (lane & 7) + ((lane >> 4) << 3), cidx = 2 * cc + ((lane >> 3) & 1);
+            uint32_t r0, r1, r2, r3;
+            ldmatrix_x4_trans(vst + row * ROWB + ((cidx ^ (row & 7)) << 4), r0, r1, r2, r3);
+            mma_bf16(acc[cc], r0, r1, r2, r3, pb0, pb1);
+        }
+        __syncwarp();
+        issue(blk + NS * NW, stage);
+    }
+    cp_async_wait<0>();
+
+    // ---- per-warp partials (max, sum) of head g
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (t == 0 && g < G) { wstat[(warp * 2 + 0) * G + g] = m_run; wstat[(warp * 2 + 1) * G + g] = l_run; }
+    __syncthreads();  // every warp is done with its ring: o_warp may overwrite it
+#pragma unroll
+    for (int cc = 0; cc < D / 16; ++cc) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int head = 2 * t + (e & 1), ch = 16 * cc + g + (e >> 1) * 8;
+            if (head < G) o_warp[(warp * G + head) * D + ch] = acc[cc][e];
+        }
+    }
+    // ---- the new token as one more partial: logit q.k_new, weight 1, value v_new (warp 0 of the owning CTA)
+    if (warp == 0) {
+        float sn[G];
+#pragma unroll
+        for (int h = 0; h < G; ++h) sn[h] = -INFINITY;
+        if (owns_new) {
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                float a = 0.f;
+                for (int e = lane; e < D; e += 32)
+                    a += __bfloat162float(q[((size_t)b * cv.Hq + kh * G + h) * D + e]) * __bfloat162float(k_new[e]);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+                sn[h] = a * scale;
+            }
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                wstat[(NW * 2 + 0) * G + h] = sn[h];
+                wstat[(NW * 2 + 1) * G + h] = owns_new ? 1.f : 0.f;
+                if (owns_new) sl[h * rows_cap + (n - 1 - lo)] = sn[h];
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- CTA partial: (max, sum) per head and the output relative to the CTA max, pushed with remote stores
+    //      (statistics into every CTA of the cluster, the output into CTA 0): nobody waits on a remote load
+    float* o_all0 = cluster.map_shared_rank(o_all, 0);
+    for (int idx = tid; idx < G * D; idx += NT) {
+        const int h = idx / D, ch = idx % D;
+        float M = -INFINITY;
+        for (int w = 0; w <= NW; ++w) M = fmaxf(M, wstat[(w * 2) * G + h]);
+        float o = 0.f, l = 0.f;
+        for (int w = 0; w < NW; ++w) {
+            const float f = exp2_diff(wstat[(w * 2) * G + h], M);
+            o += o_warp[(w * G + h) * D + ch] * f;
+            l += wstat[(w * 2 + 1) * G + h] * f;
+        }
+        if (owns_new) {
+            const float f = exp2_diff(wstat[(NW * 2) * G + h], M);
+            o += __bfloat162float(v_new[ch]) * f;
+            l += f;
+        }
+        o_all0[(size_t)rank * G * D + idx] = o;
+        if (ch < nsplit) {  // thread (h, ch = r) delivers this CTA's statistics to CTA r
+            float* gs = cluster.map_shared_rank(gstat, ch);
+            gs[(rank * 2 + 0) * G + h] = M;
+            gs[(rank * 2 + 1) * G + h] = l;
+        }
+    }
+
+    cluster.sync();  // (A) every CTA's statistics (and, in CTA 0, every partial output) have arrived
+
+    float Mg[G], invL[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+        float M = -INFINITY;
+        for (int r = 0; r < nsplit; ++r) M = fmaxf(M, gstat[(r * 2) * G + h]);
+        float L = 0.f;
+        for (int r = 0; r < nsplit; ++r) L += gstat[(r * 2 + 1) * G + h] * exp2_diff(gstat[(r * 2) * G + h], M);
+        Mg[h] = M; invL[h] = 1.0f / L;
+    }
+    if (rank == 0) {
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            for (int ch = tid; ch < D; ch += NT) {
+                float o = 0.f;
+                for (int r = 0; r < nsplit; ++r)
+                    o += o_all[((size_t)r * G + h) * D + ch] * exp2_diff(gstat[(r * 2) * G + h], Mg[h]);
+                out[((size_t)b * cv.Hq + kh * G + h) * D + ch] = __float2bfloat16_rn(o * invL[h]);
+            }
+        }
+    }
+    // ---- normalised probabilities; score update (Algorithm 1: S <- (S u {0}) + a, group mean)
+    for (int j = tid; j < nrows; j += NT) {
+        float ps = 0.f;
+#pragma unroll
+        for (int h = 0; h < G; ++h) ps += exp2_diff(sl[h * rows_cap + j], Mg[h]) * invL[h];
+        const int lam = lo + j;
+        const int ph = phys_row(lam, i_cyc);
+        const float s_old = (lam == n - 1) ? 0.f : Sc[ph];
+        Sc[ph] = s_old + ps * (1.0f / G);
+        if (lam == n - 1) Pc[ph] = N;
+    }
+
+    cluster.sync();  // (B) the appended row and every S update of the unit are complete
+
+    if (rank == 0 && warp == 0) {
+        // ---- Algorithm 1, "length > c" branch: scope {idx, idx+1} = physical rows (2i, 2i+1)
+        const int N1 = N + 1;
+        if (N1 > cv.c) {
+            const int l = 2 * i_cyc, r = l + 1;
+            int evict_right = 0;
+            if (lane == 0) {
+                bool near_tie = false;
+                evict_right = pair_evicts_right(__ldcg(Sc + l), N1 - __ldcg(Pc + l), __ldcg(Sc + r), N1 - __ldcg(Pc + r),
+                                                cv.rule, &near_tie) ? 1 : 0;
+                if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
+            }
+            evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
+            const int src = evict_right ? l : r, dst = i_cyc;
+            if (src != dst) {
+                for (int e = lane; e < CHUNKS; e += 32) {
+                    const uint4 kk = __ldcg(reinterpret_cast<const uint4*>(Kc + (size_t)src * D) + e);
+                    const uint4 vv = __ldcg(reinterpret_cast<const uint4*>(Vc + (size_t)src * D) + e);
+                    reinterpret_cast<uint4*>(Kc + (size_t)dst * D)[e] = kk;
+                    reinterpret_cast<uint4*>(Vc + (size_t)dst * D)[e] = vv;
+                }
+                if (lane == 0) { Sc[dst] = __ldcg(Sc + src); Pc[dst] = __ldcg(Pc + src); }
+            }
+        }
+        if (lane == 0) cv.n_seen[unit] = N1;
+    }
+}
+
+size_t decode_mma_smem_bytes(int G, int D, int c, int split) {
+    const size_t ring = (size_t)kMmaWarps * kMmaStages * 2 * kBlk * D * 2;
+    return ring + sizeof(float) * ((size_t)G * mma_rows_cap(c, split) + (kMmaWarps + 1) * 2 * G + kMaxSplit * 2 * G +
+                                   (size_t)split * G * D);
+}
+
+template <int D, int G>
+static cudaError_t launch_decode_mma_t(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+                                       const ActiveMask& active, int split, cudaStream_t stream) {
+    auto kern = decode_mma_kernel<D, G, kMmaWarps, kMmaStages>;
+    const int rows_cap = mma_rows_cap(cv.c, split);
+    const size_t smem = decode_mma_smem_bytes(G, D, cv.c, split);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(split, cv.Hkv, cv.B);
+    cfg.blockDim = dim3(kMmaWarps * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = split;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    using T = __nv_bfloat16;
+    return cudaLaunchKernelEx(&cfg, kern, cv, reinterpret_cast<const T*>(q), reinterpret_cast<const T*>(k),
+                              reinterpret_cast<const T*>(v), reinterpret_cast<T*>(out), active, rows_cap);
+}
+
+template <int D>
+static cudaError_t launch_decode_mma_g(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+                                       const ActiveMask& active, int split, cudaStream_t stream) {
+    switch (cv.Hq / cv.Hkv) {
+        case 1: return launch_decode_mma_t<D, 1>(cv, q, k, v, out, active, split, stream);
+        case 2: return launch_decode_mma_t<D, 2>(cv, q, k, v, out, active, split, stream);
+        case 4: return launch_decode_mma_t<D, 4>(cv, q, k, v, out, active, split, stream);
+        case 8: return launch_decode_mma_t<D, 8>(cv, q, k, v, out, active, split, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_decode_mma(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+                              const ActiveMask& active, int split, cudaStream_t stream) {
+    if (cv.d == 64) return launch_decode_mma_g<64>(cv, q, k, v, out, active, split, stream);
+    if (cv.d == 128) return launch_decode_mma_g<128>(cv, q, k, v, out, active, split, stream);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace treekv
