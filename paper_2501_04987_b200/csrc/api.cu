@@ -6,6 +6,7 @@
 
 #include "common.cuh"
 #include "ctx.cuh"
+#include "tma.cuh"
 
 using namespace treekv;
 
@@ -71,6 +72,10 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 treekv_status cuda_fail(treekv_ctx* ctx, cudaError_t e) {
     if (ctx) ctx->last_cuda_error = (int)e;
     return TREEKV_ERR_CUDA;
+}
+
+bool use_tc_prefill(const treekv_ctx* ctx) {
+    return ctx->has_tma && ctx->opt_prefill_path != 1;
 }
 
 bool use_mma_decode(const treekv_ctx* ctx) {
@@ -147,7 +152,19 @@ treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_
             sms = 148;
         ctx->sm_count = sms;
     }
-    const cudaError_t e = launch_init_state(ctx->cv, static_cast<cudaStream_t>(stream));
+    ctx->has_tma = false;
+    if (dtype == TREEKV_BF16 && head_dim == 128 && max_chunk > 0) {
+        const uint64_t rows = (uint64_t)batch * n_kv_heads * L.R;
+        const uint64_t dims[2] = {(uint64_t)head_dim, rows};
+        const uint64_t strides[1] = {(uint64_t)head_dim * 2};
+        const uint32_t box[2] = {64u, 128u};
+        ctx->has_tma = make_tensor_map_bf16(&ctx->tmK, ctx->cv.K, 2, dims, strides, box) &&
+                       make_tensor_map_bf16(&ctx->tmV, ctx->cv.V, 2, dims, strides, box);
+    }
+    // The workspace starts as zeros: the tensor-core prefill reads whole 128-row tiles, and rows that hold no token
+    // yet must be finite (they are multiplied by a probability of exactly zero).
+    cudaError_t e = cudaMemsetAsync(dev_workspace, 0, L.total, static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = launch_init_state(ctx->cv, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { delete ctx; return TREEKV_ERR_CUDA; }
     ctx->launches = 1;
     *out = ctx;
@@ -222,7 +239,17 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, chunk_stride, max_m, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = launch_prefill_simt(ctx->cv, ctx->dt, ctx->ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
+    if (use_tc_prefill(ctx)) {
+        // q is [batch*chunk_stride tokens][n_heads][128]; a tile is 64 channels x G heads x 128/G tokens
+        CUtensorMap tmQ;
+        const uint64_t dims[3] = {128ull, (uint64_t)ctx->cv.Hq, (uint64_t)ctx->cv.B * (uint64_t)chunk_stride};
+        const uint64_t strides[2] = {256ull, (uint64_t)ctx->cv.Hq * 256ull};
+        const uint32_t box[3] = {64u, (uint32_t)ctx->G, (uint32_t)(128 / ctx->G)};
+        if (!make_tensor_map_bf16(&tmQ, dev_q, 3, dims, strides, box)) return TREEKV_ERR_CUDA;
+        e = launch_prefill_tc(ctx->cv, ctx->ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s);
+    } else {
+        e = launch_prefill_simt(ctx->cv, ctx->dt, ctx->ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     e = launch_chunk_scores(ctx->cv, ctx->ps, lens, max_m, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
@@ -348,7 +375,7 @@ treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value) {
             return TREEKV_OK;
         case TREEKV_OPT_PREFILL_PATH:
             if (value < 0 || value > 2) return TREEKV_ERR_INVALID_ARG;
-            if (value == 2) return TREEKV_ERR_UNSUPPORTED;
+            if (value == 2 && !ctx->has_tma) return TREEKV_ERR_UNSUPPORTED;
             ctx->opt_prefill_path = value;
             return TREEKV_OK;
     }

@@ -11,6 +11,7 @@
 // are [0, L).  "Live index" lambda in [0, L) maps to the physical row  lambda < i ? lambda : lambda + i.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -174,5 +175,10 @@ cudaError_t launch_chunk_finalize(const CacheView& cv, const ChunkLens& lens, cu
 size_t prefill_simt_smem_bytes(int G, int D, int n_max);
 cudaError_t launch_prefill_simt(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const void* q, void* out,
                                 const ChunkLens& lens, int chunk_stride, int max_m, cudaStream_t stream);
+
+size_t prefill_tc_smem_bytes();
+cudaError_t launch_prefill_tc(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                              const CUtensorMap& tmV, void* out, const ChunkLens& lens, int chunk_stride, int max_m,
+                              cudaStream_t stream);
 
 }  // namespace treekv

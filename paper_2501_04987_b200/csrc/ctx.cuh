@@ -6,6 +6,8 @@
 struct treekv_ctx {
     treekv::CacheView cv;
     treekv::PrefillScratch ps;
+    CUtensorMap tmK, tmV;  // 2-D maps over the K and V slabs (rows x head_dim), box 128 rows x 64 channels (bf16, d=128)
+    bool has_tma;
     treekv_dtype dt;
     int max_chunk;
     int G;

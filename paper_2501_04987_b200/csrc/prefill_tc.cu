@@ -1,0 +1,347 @@
+// Chunked-prefill attention of TreeKV on the 5th-generation tensor cores (bf16, head_dim 128).
+//
+// What it computes (Section 3.1 of the paper applied to a chunk): for a tile of 128 query rows (row = token * G
+// + head-in-group) of one unit (sequence, KV head), out = softmax(q K^T / sqrt(d)) V over every cached row and
+// the chunk rows up to the query's own, and the tile's column sums of that probability matrix, which the score
+// update adds to S (Algorithm 1: S <- S + a, for all steps of the chunk at once).
+//
+// How: two passes over the key tiles, both on tcgen05.mma with TMA-fed, 128-byte-swizzled shared-memory tiles
+// and accumulators in tensor memory.
+//   pass A  S = Q K^T (tensor-memory lane = query): running row max and sum -> log-sum-exp per query.
+//   pass B  S^T = K Q^T (lane = key): P^T = exp2(S^T * scale - lse[query]) is already normalised, so its row
+//           sums over the queries ARE the column sums (one register add per element, no cross-lane reduction),
+//           and O^T += V^T P^T accumulates the output with no rescaling.  P^T goes to shared memory as the
+//           MN-major B operand; V is consumed as the MN-major A operand straight from its row-major tile.
+// Same three contractions and two exponentials per element as "attention, then recompute against the final
+// log-sum-exp", with the probabilities used for the output and for the scores being the same numbers.
+//
+// Warp roles: warp 0 issues TMA, warp 1 issues MMA and owns the tensor-memory allocation, warps 2-5 are the
+// softmax warps (one tensor-memory lane quarter each).  All waits are bounded mbarrier waits; a wait that gives
+// up sets an error word and the CTA drains to its exit, where tensor memory is released.
+#include "common.cuh"
+#include "tma.cuh"
+
+namespace treekv {
+
+namespace {
+
+constexpr int kSlot = 32768;   // one tile: [2 halves of 64 channels or 64 queries][128 rows][128 bytes]
+constexpr int kHalf = 16384;
+constexpr int kRing = 4;       // K / V tiles in flight
+constexpr int kTcThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr int kD = 128;
+
+enum Bar { Q_FULL = 0, RING_FULL = 1, RING_EMPTY = 5, S_FULL = 9, S_FREE = 11, P_FULL = 13, P_FREE = 15, O_FULL = 17, N_BARS = 18 };
+
+struct KeyTiles {
+    int i;     // cycle position: live rows [0,i) and [2i, ...)
+    int L;     // cached rows before the chunk
+    int nvis;  // live indices [0, nvis) are visible to at least one query of this tile
+    int nA;    // tiles over the old segment [0, i)
+    int NT;    // all tiles
+};
+// key tile j: first live index, first physical row, rows that exist
+__device__ inline void tile_of(const KeyTiles& kt, int j, int& lam0, int& row0, int& valid) {
+    if (j < kt.nA) { lam0 = j * 128; row0 = lam0; valid = min(128, kt.i - lam0); }
+    else { lam0 = kt.i + (j - kt.nA) * 128; row0 = lam0 + kt.i; valid = min(128, kt.nvis - lam0); }
+}
+
+}  // namespace
+
+template <int G>
+__global__ void __launch_bounds__(kTcThreads, 1)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                  const __grid_constant__ CUtensorMap tmV, CacheView cv, PrefillScratch ps,
+                  __nv_bfloat16* __restrict__ out, ChunkLens lens, int chunk_stride) {
+    constexpr int TOK = 128 / G;
+    const int unit = blockIdx.y, qt = blockIdx.x;
+    const int b = unit / cv.Hkv, kh = unit % cv.Hkv;
+    const int m = lens.m[b];
+    const int t0 = qt * TOK;
+    if (t0 >= m) return;
+    const int t1 = min(t0 + TOK, m);
+    const int N = cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv.c);
+    KeyTiles kt;
+    kt.i = st.i; kt.L = st.L; kt.nvis = st.L + t1;
+    kt.nA = (st.i + 127) / 128;
+    kt.NT = kt.nA + (kt.nvis - st.i + 127) / 128;
+    const int NT = kt.NT;
+    const int n = st.L + m;
+
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t bars[N_BARS];
+    __shared__ uint32_t tmem_slot;
+    const uint32_t base = (smem_addr_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_addr_u32(smem_raw));
+    const uint32_t sQ = base, sRing = base + kSlot, sP = base + (1 + kRing) * kSlot;
+    float* lse = reinterpret_cast<float*>(base_ptr + (3 + kRing) * kSlot);  // [128] log2-domain log-sum-exp per query row
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t bar0 = smem_addr_u32(&bars[0]);
+    auto bar = [&](int idx) { return bar0 + 8u * (uint32_t)idx; };
+
+    if (tid == 0) {
+        mbar_init(bar(Q_FULL), 1);
+        for (int s = 0; s < kRing; ++s) { mbar_init(bar(RING_FULL + s), 1); mbar_init(bar(RING_EMPTY + s), 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_FREE + s), 4);
+            mbar_init(bar(P_FULL + s), 4); mbar_init(bar(P_FREE + s), 1);
+        }
+        mbar_init(bar(O_FULL), 1);
+        mbar_fence_init();
+    }
+    if (warp == 1) { tmem_alloc(smem_addr_u32(&tmem_slot), kTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+    const uint32_t tmS = tmem, tmO = tmem + 256;  // S / S^T double buffer at columns 0 and 128; O^T at 256
+
+    bool ok = true;
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            mbar_arrive_expect_tx(bar(Q_FULL), kSlot);
+            tma_load_3d(sQ, &tmQ, 0, kh * G, b * chunk_stride + t0, bar(Q_FULL));
+            tma_load_3d(sQ + kHalf, &tmQ, 64, kh * G, b * chunk_stride + t0, bar(Q_FULL));
+            int ld = 0;
+            for (int pass = 0; pass < 2 && ok; ++pass) {
+                for (int j = 0; j < NT && ok; ++j) {
+                    int lam0, row0, valid;
+                    tile_of(kt, j, lam0, row0, valid);
+                    const int grow = unit * cv.R + row0;
+                    for (int which = 0; which <= pass; ++which) {  // pass A: K only; pass B: K then V
+                        const int slot = ld % kRing;
+                        if (!mbar_wait(bar(RING_EMPTY + slot), ((ld / kRing) & 1) ^ 1)) { ok = false; break; }
+                        const uint32_t dst = sRing + slot * kSlot;
+                        mbar_arrive_expect_tx(bar(RING_FULL + slot), kSlot);
+                        const CUtensorMap* mp = which == 0 ? &tmK : &tmV;
+                        tma_load_2d(dst, mp, 0, grow, bar(RING_FULL + slot));
+                        tma_load_2d(dst + kHalf, mp, 64, grow, bar(RING_FULL + slot));
+                        ++ld;
+                    }
+                }
+            }
+            if (!ok) atomicOr(&cv.stats->error, 4u);
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            constexpr uint32_t idesc_kk = umma_idesc_bf16(128, 128, 0, 0);  // both operands K-major (rows x channels)
+            constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, 1, 1);  // V^T and P^T: MN-major
+            ok = mbar_wait(bar(Q_FULL), 0);
+            tc_fence_after();
+            int sc = 0;  // S tiles issued (both passes): buffer sc & 1
+            // ---- pass A: S = Q K^T
+            for (int j = 0; j < NT && ok; ++j) {
+                const int ld = j, slot = ld % kRing, buf = sc & 1;
+                ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), ((sc >> 1) & 1) ^ 1);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t sK = sRing + slot * kSlot;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * kHalf + (kk & 3) * 32;
+                    umma_bf16(tmS + buf * 128, umma_desc_sw128(sQ + off, 16, 1024), umma_desc_sw128(sK + off, 16, 1024),
+                              idesc_kk, kk > 0);
+                }
+                umma_commit(bar(RING_EMPTY + slot));
+                umma_commit(bar(S_FULL + buf));
+                ++sc;
+            }
+            // ---- pass B: S^T_j = K_j Q^T issued one tile ahead of O^T_{j-1} += V_{j-1}^T P_{j-1}^T
+            for (int j = 0; j <= NT && ok; ++j) {
+                if (j < NT) {
+                    const int ld = NT + 2 * j, slot = ld % kRing, buf = sc & 1;
+                    ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), ((sc >> 1) & 1) ^ 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sK = sRing + slot * kSlot;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t off = (kk >> 2) * kHalf + (kk & 3) * 32;
+                        umma_bf16(tmS + buf * 128, umma_desc_sw128(sK + off, 16, 1024), umma_desc_sw128(sQ + off, 16, 1024),
+                                  idesc_kk, kk > 0);
+                    }
+                    umma_commit(bar(RING_EMPTY + slot));
+                    umma_commit(bar(S_FULL + buf));
+                    ++sc;
+                }
+                if (j >= 1) {
+                    const int pj = j - 1, pbuf = pj & 1;
+                    const int ld = NT + 2 * pj + 1, slot = ld % kRing;
+                    ok = mbar_wait(bar(P_FULL + pbuf), (pj >> 1) & 1) && mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sV = sRing + slot * kSlot, sPT = sP + pbuf * kSlot;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step: 16 rows of 128 bytes
+                        umma_bf16(tmO, umma_desc_sw128(sV + kk * 2048, kHalf, 1024), umma_desc_sw128(sPT + kk * 2048, kHalf, 1024),
+                                  idesc_pv, (pj > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    umma_commit(bar(RING_EMPTY + slot));
+                    umma_commit(bar(P_FREE + pbuf));
+                }
+            }
+            if (ok) umma_commit(bar(O_FULL));
+            else atomicOr(&cv.stats->error, 8u);
+        }
+    } else {
+        // ================= softmax warps =================
+        const int quarter = warp & 3;          // tensor-memory lanes [32*quarter, +32) belong to this warp
+        const int row = quarter * 32 + lane;   // pass A: query row; pass B: key of the tile; epilogue: channel
+        const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+        const float sc2 = kLog2e * rsqrtf((float)kD);
+        uint32_t v[32];
+        int sc = 0;
+        // ---- pass A: row statistics
+        {
+            const int tq = min(t0 + row / G, t1 - 1);  // rows past the chunk repeat the last real row: finite, unused
+            float mrun = -INFINITY, lrun = 0.f;
+            for (int j = 0; j < NT && ok; ++j) {
+                const int buf = sc & 1;
+                if (!mbar_wait(bar(S_FULL + buf), (sc >> 1) & 1)) { ok = false; break; }
+                tc_fence_after();
+                int lam0, row0, valid;
+                tile_of(kt, j, lam0, row0, valid);
+                const int limit = max(0, min(valid, kt.L + tq - lam0 + 1));  // columns [0, limit) are visible to this row
+#pragma unroll 1
+                for (int cg = 0; cg < 4; ++cg) {
+                    tmem_ld32(tmS + lane_off + buf * 128 + cg * 32, v);
+                    tmem_ld_wait();
+                    float x[32];
+                    float cmax = -INFINITY;
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        x[e] = (cg * 32 + e < limit) ? __uint_as_float(v[e]) * sc2 : -INFINITY;
+                        cmax = fmaxf(cmax, x[e]);
+                    }
+                    if (cmax > -INFINITY) {
+                        const float mnew = fmaxf(mrun, cmax);
+                        float s = 0.f;
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) s += exp2f(x[e] - mnew);
+                        lrun = lrun * exp2f(mrun - mnew) + s;
+                        mrun = mnew;
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(S_FREE + buf));
+                ++sc;
+            }
+            lse[row] = mrun + log2f(lrun);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");  // the four softmax warps: lse[] is complete
+        // ---- pass B: probabilities, column sums, P^T for the tensor cores
+        const int rmax = G * (t1 - t0);  // query columns [rmax, 128) are padding
+        float* part = ps.colsum + ((size_t)unit * ps.QT + qt) * ps.n_max;
+        for (int j = 0; j < NT && ok; ++j) {
+            const int buf = sc & 1, pbuf = j & 1;
+            if (!mbar_wait(bar(S_FULL + buf), (sc >> 1) & 1) || !mbar_wait(bar(P_FREE + pbuf), ((j >> 1) & 1) ^ 1)) { ok = false; break; }
+            tc_fence_after();
+            int lam0, row0, valid;
+            tile_of(kt, j, lam0, row0, valid);
+            const bool kvalid = row < valid;
+            const int lam = lam0 + row;
+            const int rmin = kvalid ? max(0, G * (lam - kt.L - t0)) : 128;  // first query column that sees this key
+            float colsum = 0.f;
+            unsigned char* prow = base_ptr + (1 + kRing) * kSlot + pbuf * kSlot + row * 128;
+#pragma unroll 1
+            for (int cg = 0; cg < 4; ++cg) {
+                tmem_ld32(tmS + lane_off + buf * 128 + cg * 32, v);
+                tmem_ld_wait();
+                if (cg == 3) {  // last read of this S^T buffer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(S_FREE + buf));
+                }
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {  // 8 query columns -> one 16-byte chunk of the P^T row
+                    float p[8];
+#pragma unroll
+                    for (int h4 = 0; h4 < 2; ++h4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(lse + cg * 32 + q4 * 8 + h4 * 4);
+                        const float ls[4] = {l4.x, l4.y, l4.z, l4.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int r = cg * 32 + q4 * 8 + h4 * 4 + e;
+                            const float x = __uint_as_float(v[q4 * 8 + h4 * 4 + e]) * sc2 - ls[e];
+                            const float pe = (r >= rmin && r < rmax) ? exp2f(x) : 0.f;
+                            p[h4 * 4 + e] = pe;
+                            colsum += pe;
+                        }
+                    }
+                    uint4 pk;
+                    __nv_bfloat162 t2;
+                    t2 = __floats2bfloat162_rn(p[0], p[1]); pk.x = *reinterpret_cast<uint32_t*>(&t2);
+                    t2 = __floats2bfloat162_rn(p[2], p[3]); pk.y = *reinterpret_cast<uint32_t*>(&t2);
+                    t2 = __floats2bfloat162_rn(p[4], p[5]); pk.z = *reinterpret_cast<uint32_t*>(&t2);
+                    t2 = __floats2bfloat162_rn(p[6], p[7]); pk.w = *reinterpret_cast<uint32_t*>(&t2);
+                    const int cidx = cg * 4 + q4;  // 16-byte chunk of the 128-query row: half = cidx / 8
+                    *reinterpret_cast<uint4*>(prow + (cidx >> 3) * kHalf + (((cidx & 7) ^ (row & 7)) << 4)) = pk;
+                }
+            }
+            if (kvalid) part[lam] = colsum;
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(P_FULL + pbuf));
+            ++sc;
+        }
+        // keys this tile's queries cannot see contribute nothing
+        for (int lam = kt.nvis + (tid - 64); lam < n; lam += 128) part[lam] = 0.f;
+        // ---- epilogue: O^T (lane = channel, column = query row) -> out[token][head][channel]
+        if (ok && mbar_wait(bar(O_FULL), 0)) {
+            tc_fence_after();
+#pragma unroll 1
+            for (int cg = 0; cg < 4; ++cg) {
+                tmem_ld32(tmO + lane_off + cg * 32, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const int r = cg * 32 + e;
+                    if (r < rmax)
+                        out[(((size_t)b * chunk_stride + t0 + r / G) * cv.Hq + kh * G + (r % G)) * kD + row] =
+                            __float2bfloat16_rn(__uint_as_float(v[e]));
+                }
+            }
+            tc_fence_before();
+        } else {
+            atomicOr(&cv.stats->error, 16u);
+        }
+    }
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+}
+
+size_t prefill_tc_smem_bytes() { return 1024 + (size_t)(3 + kRing) * kSlot + 512 + 64; }
+
+template <int G>
+static cudaError_t launch_prefill_tc_t(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ,
+                                       const CUtensorMap& tmK, const CUtensorMap& tmV, void* out, const ChunkLens& lens,
+                                       int chunk_stride, int max_m, cudaStream_t stream) {
+    auto kern = prefill_tc_kernel<G>;
+    const size_t smem = prefill_tc_smem_bytes();
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid((max_m * G + kQTileRows - 1) / kQTileRows, cv.B * cv.Hkv);
+    kern<<<grid, kTcThreads, smem, stream>>>(tmQ, tmK, tmV, cv, ps, reinterpret_cast<__nv_bfloat16*>(out), lens, chunk_stride);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_tc(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                              const CUtensorMap& tmV, void* out, const ChunkLens& lens, int chunk_stride, int max_m,
+                              cudaStream_t stream) {
+    if (cv.d != kD) return cudaErrorInvalidValue;
+    switch (cv.Hq / cv.Hkv) {
+        case 1: return launch_prefill_tc_t<1>(cv, ps, tmQ, tmK, tmV, out, lens, chunk_stride, max_m, stream);
+        case 2: return launch_prefill_tc_t<2>(cv, ps, tmQ, tmK, tmV, out, lens, chunk_stride, max_m, stream);
+        case 4: return launch_prefill_tc_t<4>(cv, ps, tmQ, tmK, tmV, out, lens, chunk_stride, max_m, stream);
+        case 8: return launch_prefill_tc_t<8>(cv, ps, tmQ, tmK, tmV, out, lens, chunk_stride, max_m, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace treekv
