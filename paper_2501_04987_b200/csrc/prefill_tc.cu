@@ -15,8 +15,9 @@
 // Same three contractions and two exponentials per element as "attention, then recompute against the final
 // log-sum-exp", with the probabilities used for the output and for the scores being the same numbers.
 //
-// Warp roles: warp 0 issues TMA, warp 1 issues MMA and owns the tensor-memory allocation, warps 2-5 are the
-// softmax warps (one tensor-memory lane quarter each).  All waits are bounded mbarrier waits; a wait that gives
+// Warp roles: warp 0 issues TMA, warp 1 issues MMA and owns the tensor-memory allocation, warps 2-9 are two
+// groups of four softmax warps (one tensor-memory lane quarter per warp); group g owns the S buffer, the P^T
+// buffer and the key tiles of parity g, so the two groups alternate tiles and overlap each other's latency.  All waits are bounded mbarrier waits; a wait that gives
 // up sets an error word and the CTA drains to its exit, where tensor memory is released.
 #include "common.cuh"
 #include "tma.cuh"
@@ -28,7 +29,7 @@ namespace {
 constexpr int kSlot = 32768;   // one tile: [2 halves of 64 channels or 64 queries][128 rows][128 bytes]
 constexpr int kHalf = 16384;
 constexpr int kRing = 4;       // K / V tiles in flight
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 320;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kD = 128;
 
@@ -76,7 +77,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t base = (smem_addr_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_addr_u32(smem_raw));
     const uint32_t sQ = base, sRing = base + kSlot, sP = base + (1 + kRing) * kSlot;
-    float* lse = reinterpret_cast<float*>(base_ptr + (3 + kRing) * kSlot);  // [128] log2-domain log-sum-exp per query row
+    float* lse = reinterpret_cast<float*>(base_ptr + (3 + kRing) * kSlot);  // [640] statistics of the query rows
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t bar0 = smem_addr_u32(&bars[0]);
@@ -133,11 +134,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, 1, 1);  // V^T and P^T: MN-major
             ok = mbar_wait(bar(Q_FULL), 0);
             tc_fence_after();
-            int sc = 0;  // S tiles issued (both passes): buffer sc & 1
+            int use[2] = {0, 0};  // times each S buffer has been handed to the softmax warps (both passes)
             // ---- pass A: S = Q K^T
             for (int j = 0; j < NT && ok; ++j) {
-                const int ld = j, slot = ld % kRing, buf = sc & 1;
-                ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), ((sc >> 1) & 1) ^ 1);
+                const int ld = j, slot = ld % kRing, buf = j & 1;
+                ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), (use[buf] & 1) ^ 1);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t sK = sRing + slot * kSlot;
@@ -149,13 +150,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 }
                 umma_commit(bar(RING_EMPTY + slot));
                 umma_commit(bar(S_FULL + buf));
-                ++sc;
+                ++use[buf];
             }
             // ---- pass B: S^T_j = K_j Q^T issued one tile ahead of O^T_{j-1} += V_{j-1}^T P_{j-1}^T
             for (int j = 0; j <= NT && ok; ++j) {
                 if (j < NT) {
-                    const int ld = NT + 2 * j, slot = ld % kRing, buf = sc & 1;
-                    ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), ((sc >> 1) & 1) ^ 1);
+                    const int ld = NT + 2 * j, slot = ld % kRing, buf = j & 1;
+                    ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), (use[buf] & 1) ^ 1);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sK = sRing + slot * kSlot;
@@ -167,7 +168,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     }
                     umma_commit(bar(RING_EMPTY + slot));
                     umma_commit(bar(S_FULL + buf));
-                    ++sc;
+                    ++use[buf];
                 }
                 if (j >= 1) {
                     const int pj = j - 1, pbuf = pj & 1;
@@ -190,90 +191,123 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
     } else {
         // ================= softmax warps =================
+        const int grp = (warp - 2) >> 2;       // group 0: warps 2-5, group 1: warps 6-9; group g owns tiles j = g (mod 2)
         const int quarter = warp & 3;          // tensor-memory lanes [32*quarter, +32) belong to this warp
         const int row = quarter * 32 + lane;   // pass A: query row; pass B: key of the tile; epilogue: channel
         const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
         const float sc2 = kLog2e * rsqrtf((float)kD);
+        const uint32_t tmSg = tmS + grp * 128 + lane_off;
+        float* nlse = lse;                     // [128] minus the log2-domain log-sum-exp of every query row
+        float* part_m = lse + 128;             // [2][128] per-group running max
+        float* part_l = lse + 384;             // [2][128] per-group running sum
         uint32_t v[32];
-        int sc = 0;
-        // ---- pass A: row statistics
+        int use = 0;  // times this group's S buffer has been filled (both passes)
+        // ---- pass A: row statistics over this group's tiles
         {
             const int tq = min(t0 + row / G, t1 - 1);  // rows past the chunk repeat the last real row: finite, unused
             float mrun = -INFINITY, lrun = 0.f;
-            for (int j = 0; j < NT && ok; ++j) {
-                const int buf = sc & 1;
-                if (!mbar_wait(bar(S_FULL + buf), (sc >> 1) & 1)) { ok = false; break; }
+            for (int j = grp; j < NT && ok; j += 2) {
+                if (!mbar_wait(bar(S_FULL + grp), use & 1)) { ok = false; break; }
                 tc_fence_after();
                 int lam0, row0, valid;
                 tile_of(kt, j, lam0, row0, valid);
                 const int limit = max(0, min(valid, kt.L + tq - lam0 + 1));  // columns [0, limit) are visible to this row
+                const bool full = __all_sync(0xffffffffu, limit >= 128);
 #pragma unroll 1
                 for (int cg = 0; cg < 4; ++cg) {
-                    tmem_ld32(tmS + lane_off + buf * 128 + cg * 32, v);
+                    tmem_ld32(tmSg + cg * 32, v);
                     tmem_ld_wait();
-                    float x[32];
-                    float cmax = -INFINITY;
+                    if (full) {
+                        float cmax = __uint_as_float(v[0]);
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        x[e] = (cg * 32 + e < limit) ? __uint_as_float(v[e]) * sc2 : -INFINITY;
-                        cmax = fmaxf(cmax, x[e]);
-                    }
-                    if (cmax > -INFINITY) {
-                        const float mnew = fmaxf(mrun, cmax);
-                        float s = 0.f;
+                        for (int e = 1; e < 32; ++e) cmax = fmaxf(cmax, __uint_as_float(v[e]));
+                        const float mnew = fmaxf(mrun, cmax * sc2);
+                        float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) s += exp2f(x[e] - mnew);
-                        lrun = lrun * exp2f(mrun - mnew) + s;
+                        for (int e = 0; e < 32; e += 2) {
+                            s0 += exp2f(fmaf(__uint_as_float(v[e]), sc2, -mnew));
+                            s1 += exp2f(fmaf(__uint_as_float(v[e + 1]), sc2, -mnew));
+                        }
+                        lrun = lrun * exp2f(mrun - mnew) + (s0 + s1);
                         mrun = mnew;
+                    } else {
+                        float x[32];
+                        float cmax = -INFINITY;
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) {
+                            x[e] = (cg * 32 + e < limit) ? __uint_as_float(v[e]) * sc2 : -INFINITY;
+                            cmax = fmaxf(cmax, x[e]);
+                        }
+                        if (cmax > -INFINITY) {
+                            const float mnew = fmaxf(mrun, cmax);
+                            float sacc = 0.f;
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) sacc += exp2f(x[e] - mnew);
+                            lrun = lrun * exp2f(mrun - mnew) + sacc;
+                            mrun = mnew;
+                        }
                     }
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(S_FREE + buf));
-                ++sc;
+                if (lane == 0) mbar_arrive(bar(S_FREE + grp));
+                ++use;
             }
-            lse[row] = mrun + log2f(lrun);
+            part_m[grp * 128 + row] = mrun;
+            part_l[grp * 128 + row] = lrun;
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");  // the four softmax warps: lse[] is complete
+        asm volatile("bar.sync 1, 256;" ::: "memory");  // both groups: the partial statistics are complete
+        if (grp == 0) {
+            const float m0 = part_m[row], m1 = part_m[128 + row];
+            const float M = fmaxf(m0, m1);
+            const float l = (m0 == -INFINITY ? 0.f : part_l[row] * exp2f(m0 - M)) +
+                            (m1 == -INFINITY ? 0.f : part_l[128 + row] * exp2f(m1 - M));
+            nlse[row] = -(M + log2f(l));
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");  // nlse[] is complete
         // ---- pass B: probabilities, column sums, P^T for the tensor cores
         const int rmax = G * (t1 - t0);  // query columns [rmax, 128) are padding
         float* part = ps.colsum + ((size_t)unit * ps.QT + qt) * ps.n_max;
-        for (int j = 0; j < NT && ok; ++j) {
-            const int buf = sc & 1, pbuf = j & 1;
-            if (!mbar_wait(bar(S_FULL + buf), (sc >> 1) & 1) || !mbar_wait(bar(P_FREE + pbuf), ((j >> 1) & 1) ^ 1)) { ok = false; break; }
+        int puse = 0;  // times this group's P^T buffer has been filled
+        for (int j = grp; j < NT && ok; j += 2) {
+            if (!mbar_wait(bar(S_FULL + grp), use & 1) || !mbar_wait(bar(P_FREE + grp), (puse & 1) ^ 1)) { ok = false; break; }
             tc_fence_after();
             int lam0, row0, valid;
             tile_of(kt, j, lam0, row0, valid);
             const bool kvalid = row < valid;
             const int lam = lam0 + row;
             const int rmin = kvalid ? max(0, G * (lam - kt.L - t0)) : 128;  // first query column that sees this key
+            const bool full = __all_sync(0xffffffffu, rmin == 0) && rmax == 128;
             float colsum = 0.f;
-            unsigned char* prow = base_ptr + (1 + kRing) * kSlot + pbuf * kSlot + row * 128;
+            unsigned char* prow = base_ptr + (1 + kRing) * kSlot + grp * kSlot + row * 128;
 #pragma unroll 1
             for (int cg = 0; cg < 4; ++cg) {
-                tmem_ld32(tmS + lane_off + buf * 128 + cg * 32, v);
+                tmem_ld32(tmSg + cg * 32, v);
                 tmem_ld_wait();
                 if (cg == 3) {  // last read of this S^T buffer
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(S_FREE + buf));
+                    if (lane == 0) mbar_arrive(bar(S_FREE + grp));
                 }
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {  // 8 query columns -> one 16-byte chunk of the P^T row
                     float p[8];
 #pragma unroll
                     for (int h4 = 0; h4 < 2; ++h4) {
-                        const float4 l4 = *reinterpret_cast<const float4*>(lse + cg * 32 + q4 * 8 + h4 * 4);
+                        const float4 l4 = *reinterpret_cast<const float4*>(nlse + cg * 32 + q4 * 8 + h4 * 4);
                         const float ls[4] = {l4.x, l4.y, l4.z, l4.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const int r = cg * 32 + q4 * 8 + h4 * 4 + e;
-                            const float x = __uint_as_float(v[q4 * 8 + h4 * 4 + e]) * sc2 - ls[e];
-                            const float pe = (r >= rmin && r < rmax) ? exp2f(x) : 0.f;
-                            p[h4 * 4 + e] = pe;
-                            colsum += pe;
+                            const float pe = exp2f(fmaf(__uint_as_float(v[q4 * 8 + h4 * 4 + e]), sc2, ls[e]));
+                            if (full) {
+                                p[h4 * 4 + e] = pe;
+                            } else {
+                                const int r = cg * 32 + q4 * 8 + h4 * 4 + e;
+                                p[h4 * 4 + e] = (r >= rmin && r < rmax) ? pe : 0.f;
+                            }
                         }
                     }
+                    colsum += ((p[0] + p[1]) + (p[2] + p[3])) + ((p[4] + p[5]) + (p[6] + p[7]));
                     uint4 pk;
                     __nv_bfloat162 t2;
                     t2 = __floats2bfloat162_rn(p[0], p[1]); pk.x = *reinterpret_cast<uint32_t*>(&t2);
@@ -287,16 +321,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (kvalid) part[lam] = colsum;
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(P_FULL + pbuf));
-            ++sc;
+            if (lane == 0) mbar_arrive(bar(P_FULL + grp));
+            ++use;
+            ++puse;
         }
         // keys this tile's queries cannot see contribute nothing
-        for (int lam = kt.nvis + (tid - 64); lam < n; lam += 128) part[lam] = 0.f;
-        // ---- epilogue: O^T (lane = channel, column = query row) -> out[token][head][channel]
+        for (int lam = kt.nvis + (tid - 64); lam < n; lam += 256) part[lam] = 0.f;
+        // ---- epilogue: O^T (lane = channel, column = query row) -> out[token][head][channel]; each group half the columns
         if (ok && mbar_wait(bar(O_FULL), 0)) {
             tc_fence_after();
 #pragma unroll 1
-            for (int cg = 0; cg < 4; ++cg) {
+            for (int cg = 2 * grp; cg < 2 * grp + 2; ++cg) {
                 tmem_ld32(tmO + lane_off + cg * 32, v);
                 tmem_ld_wait();
 #pragma unroll
@@ -316,7 +351,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
-size_t prefill_tc_smem_bytes() { return 1024 + (size_t)(3 + kRing) * kSlot + 512 + 64; }
+size_t prefill_tc_smem_bytes() { return 1024 + (size_t)(3 + kRing) * kSlot + 640 * sizeof(float); }
 
 template <int G>
 static cudaError_t launch_prefill_tc_t(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ,
