@@ -77,7 +77,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t base = (smem_addr_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_addr_u32(smem_raw));
     const uint32_t sQ = base, sRing = base + kSlot, sP = base + (1 + kRing) * kSlot;
-    float* lse = reinterpret_cast<float*>(base_ptr + (3 + kRing) * kSlot);  // [640] statistics of the query rows
+    float* lse = reinterpret_cast<float*>(base_ptr + (3 + kRing) * kSlot);  // [128] minus log-sum-exp of the query rows
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t bar0 = smem_addr_u32(&bars[0]);
@@ -198,8 +198,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const float sc2 = kLog2e * rsqrtf((float)kD);
         const uint32_t tmSg = tmS + grp * 128 + lane_off;
         float* nlse = lse;                     // [128] minus the log2-domain log-sum-exp of every query row
-        float* part_m = lse + 128;             // [2][128] per-group running max
-        float* part_l = lse + 384;             // [2][128] per-group running sum
+        // per-group running (max, sum) of pass A, [2][128] each; they borrow the P^T area, which pass A does not use
+        float* part_m = reinterpret_cast<float*>(base_ptr + (1 + kRing) * kSlot);
+        float* part_l = part_m + 256;
         uint32_t v[32];
         int use = 0;  // times this group's S buffer has been filled (both passes)
         // ---- pass A: row statistics over this group's tiles
@@ -351,7 +352,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
-size_t prefill_tc_smem_bytes() { return 1024 + (size_t)(3 + kRing) * kSlot + 640 * sizeof(float); }
+size_t prefill_tc_smem_bytes() { return 1024 + (size_t)(3 + kRing) * kSlot + 128 * sizeof(float); }
 
 template <int G>
 static cudaError_t launch_prefill_tc_t(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ,
