@@ -48,6 +48,13 @@ __device__ inline void tile_of(const KeyTiles& kt, int j, int& lam0, int& row0, 
     else { lam0 = kt.i + (j - kt.nA) * 128; row0 = lam0 + kt.i; valid = min(128, kt.nvis - lam0); }
 }
 
+// 2^x on the special-function unit, one instruction (inputs here are <= ~0; results below 2^-126 flush to zero)
+__device__ inline float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 }  // namespace
 
 template <int G>
@@ -201,7 +208,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // per-group running (max, sum) of pass A, [2][128] each; they borrow the P^T area, which pass A does not use
         float* part_m = reinterpret_cast<float*>(base_ptr + (1 + kRing) * kSlot);
         float* part_l = part_m + 256;
-        uint32_t v[32];
+        uint32_t va[32], vb[32];  // two chunks of 32 columns: the next one is in flight while this one is used
         int use = 0;  // times this group's S buffer has been filled (both passes)
         // ---- pass A: row statistics over this group's tiles
         {
@@ -214,10 +221,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 tile_of(kt, j, lam0, row0, valid);
                 const int limit = max(0, min(valid, kt.L + tq - lam0 + 1));  // columns [0, limit) are visible to this row
                 const bool full = __all_sync(0xffffffffu, limit >= 128);
-#pragma unroll 1
-                for (int cg = 0; cg < 4; ++cg) {
-                    tmem_ld32(tmSg + cg * 32, v);
-                    tmem_ld_wait();
+                auto stats32 = [&](const uint32_t (&v)[32], int cg) {
                     if (full) {
                         float cmax = __uint_as_float(v[0]);
 #pragma unroll
@@ -226,10 +230,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         float s0 = 0.f, s1 = 0.f;
 #pragma unroll
                         for (int e = 0; e < 32; e += 2) {
-                            s0 += exp2f(fmaf(__uint_as_float(v[e]), sc2, -mnew));
-                            s1 += exp2f(fmaf(__uint_as_float(v[e + 1]), sc2, -mnew));
+                            s0 += ex2(fmaf(__uint_as_float(v[e]), sc2, -mnew));
+                            s1 += ex2(fmaf(__uint_as_float(v[e + 1]), sc2, -mnew));
                         }
-                        lrun = lrun * exp2f(mrun - mnew) + (s0 + s1);
+                        lrun = lrun * ex2(mrun - mnew) + (s0 + s1);
                         mrun = mnew;
                     } else {
                         float x[32];
@@ -243,12 +247,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                             const float mnew = fmaxf(mrun, cmax);
                             float sacc = 0.f;
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) sacc += exp2f(x[e] - mnew);
-                            lrun = lrun * exp2f(mrun - mnew) + sacc;
+                            for (int e = 0; e < 32; ++e) sacc += ex2(x[e] - mnew);
+                            lrun = lrun * ex2(mrun - mnew) + sacc;
                             mrun = mnew;
                         }
                     }
-                }
+                };
+                tmem_ld32(tmSg, va);
+                tmem_ld_wait_for(va);
+                tmem_ld32(tmSg + 32, vb);
+                stats32(va, 0);
+                tmem_ld_wait_for(vb);
+                tmem_ld32(tmSg + 64, va);
+                stats32(vb, 1);
+                tmem_ld_wait_for(va);
+                tmem_ld32(tmSg + 96, vb);
+                stats32(va, 2);
+                tmem_ld_wait_for(vb);
+                stats32(vb, 3);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(S_FREE + grp));
@@ -261,8 +277,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (grp == 0) {
             const float m0 = part_m[row], m1 = part_m[128 + row];
             const float M = fmaxf(m0, m1);
-            const float l = (m0 == -INFINITY ? 0.f : part_l[row] * exp2f(m0 - M)) +
-                            (m1 == -INFINITY ? 0.f : part_l[128 + row] * exp2f(m1 - M));
+            const float l = (m0 == -INFINITY ? 0.f : part_l[row] * ex2(m0 - M)) +
+                            (m1 == -INFINITY ? 0.f : part_l[128 + row] * ex2(m1 - M));
             nlse[row] = -(M + log2f(l));
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");  // nlse[] is complete
@@ -281,15 +297,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const bool full = __all_sync(0xffffffffu, rmin == 0) && rmax == 128;
             float colsum = 0.f;
             unsigned char* prow = base_ptr + (1 + kRing) * kSlot + grp * kSlot + row * 128;
-#pragma unroll 1
-            for (int cg = 0; cg < 4; ++cg) {
-                tmem_ld32(tmSg + cg * 32, v);
-                tmem_ld_wait();
-                if (cg == 3) {  // last read of this S^T buffer
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(S_FREE + grp));
-                }
+            auto probs32 = [&](const uint32_t (&v)[32], int cg) {
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {  // 8 query columns -> one 16-byte chunk of the P^T row
                     float p[8];
@@ -299,7 +307,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         const float ls[4] = {l4.x, l4.y, l4.z, l4.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float pe = exp2f(fmaf(__uint_as_float(v[q4 * 8 + h4 * 4 + e]), sc2, ls[e]));
+                            const float pe = ex2(fmaf(__uint_as_float(v[q4 * 8 + h4 * 4 + e]), sc2, ls[e]));
                             if (full) {
                                 p[h4 * 4 + e] = pe;
                             } else {
@@ -318,7 +326,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     const int cidx = cg * 4 + q4;  // 16-byte chunk of the 128-query row: half = cidx / 8
                     *reinterpret_cast<uint4*>(prow + (cidx >> 3) * kHalf + (((cidx & 7) ^ (row & 7)) << 4)) = pk;
                 }
-            }
+            };
+            tmem_ld32(tmSg, va);
+            tmem_ld_wait_for(va);
+            tmem_ld32(tmSg + 32, vb);
+            probs32(va, 0);
+            tmem_ld_wait_for(vb);
+            tmem_ld32(tmSg + 64, va);
+            probs32(vb, 1);
+            tmem_ld_wait_for(va);
+            tmem_ld32(tmSg + 96, vb);
+            probs32(va, 2);
+            tmem_ld_wait_for(vb);
+            tc_fence_before();  // last read of this S^T buffer
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(S_FREE + grp));
+            probs32(vb, 3);
             if (kvalid) part[lam] = colsum;
             fence_proxy_async_smem();
             __syncwarp();
@@ -333,14 +356,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tc_fence_after();
 #pragma unroll 1
             for (int cg = 2 * grp; cg < 2 * grp + 2; ++cg) {
-                tmem_ld32(tmO + lane_off + cg * 32, v);
-                tmem_ld_wait();
+                tmem_ld32(tmO + lane_off + cg * 32, va);
+                tmem_ld_wait_for(va);
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     const int r = cg * 32 + e;
                     if (r < rmax)
                         out[(((size_t)b * chunk_stride + t0 + r / G) * cv.Hq + kh * G + (r % G)) * kD + row] =
-                            __float2bfloat16_rn(__uint_as_float(v[e]));
+                            __float2bfloat16_rn(__uint_as_float(va[e]));
                 }
             }
             tc_fence_before();
