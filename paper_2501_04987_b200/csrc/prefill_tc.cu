@@ -159,39 +159,41 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 umma_commit(bar(S_FULL + buf));
                 ++use[buf];
             }
-            // ---- pass B: S^T_j = K_j Q^T issued one tile ahead of O^T_{j-1} += V_{j-1}^T P_{j-1}^T
-            for (int j = 0; j <= NT && ok; ++j) {
-                if (j < NT) {
-                    const int ld = NT + 2 * j, slot = ld % kRing, buf = j & 1;
-                    ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), (use[buf] & 1) ^ 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t sK = sRing + slot * kSlot;
+            // ---- pass B: S^T_j = K_j Q^T runs two tiles ahead of O^T_j += V_j^T P_j^T, so that the group that
+            //      owns buffer j & 1 finds S^T_{j+2} ready when it finishes tile j (its buffer is free as soon as
+            //      it has read tile j into registers, long before P_j^T is complete)
+            auto issue_st = [&](int j) {
+                const int ld = NT + 2 * j, slot = ld % kRing, buf = j & 1;
+                ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), (use[buf] & 1) ^ 1);
+                if (!ok) return;
+                tc_fence_after();
+                const uint32_t sK = sRing + slot * kSlot;
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t off = (kk >> 2) * kHalf + (kk & 3) * 32;
-                        umma_bf16(tmS + buf * 128, umma_desc_sw128(sK + off, 16, 1024), umma_desc_sw128(sQ + off, 16, 1024),
-                                  idesc_kk, kk > 0);
-                    }
-                    umma_commit(bar(RING_EMPTY + slot));
-                    umma_commit(bar(S_FULL + buf));
-                    ++use[buf];
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * kHalf + (kk & 3) * 32;
+                    umma_bf16(tmS + buf * 128, umma_desc_sw128(sK + off, 16, 1024), umma_desc_sw128(sQ + off, 16, 1024),
+                              idesc_kk, kk > 0);
                 }
-                if (j >= 1) {
-                    const int pj = j - 1, pbuf = pj & 1;
-                    const int ld = NT + 2 * pj + 1, slot = ld % kRing;
-                    ok = mbar_wait(bar(P_FULL + pbuf), (pj >> 1) & 1) && mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t sV = sRing + slot * kSlot, sPT = sP + pbuf * kSlot;
+                umma_commit(bar(RING_EMPTY + slot));
+                umma_commit(bar(S_FULL + buf));
+                ++use[buf];
+            };
+            for (int j = 0; j < 2 && j < NT && ok; ++j) issue_st(j);
+            for (int pj = 0; pj < NT && ok; ++pj) {
+                if (pj + 2 < NT) { issue_st(pj + 2); if (!ok) break; }
+                const int pbuf = pj & 1;
+                const int ld = NT + 2 * pj + 1, slot = ld % kRing;
+                ok = mbar_wait(bar(P_FULL + pbuf), (pj >> 1) & 1) && mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t sV = sRing + slot * kSlot, sPT = sP + pbuf * kSlot;
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step: 16 rows of 128 bytes
-                        umma_bf16(tmO, umma_desc_sw128(sV + kk * 2048, kHalf, 1024), umma_desc_sw128(sPT + kk * 2048, kHalf, 1024),
-                                  idesc_pv, (pj > 0 || kk > 0) ? 1u : 0u);
-                    }
-                    umma_commit(bar(RING_EMPTY + slot));
-                    umma_commit(bar(P_FREE + pbuf));
+                for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step: 16 rows of 128 bytes
+                    umma_bf16(tmO, umma_desc_sw128(sV + kk * 2048, kHalf, 1024), umma_desc_sw128(sPT + kk * 2048, kHalf, 1024),
+                              idesc_pv, (pj > 0 || kk > 0) ? 1u : 0u);
                 }
+                umma_commit(bar(RING_EMPTY + slot));
+                umma_commit(bar(P_FREE + pbuf));
             }
             if (ok) umma_commit(bar(O_FULL));
             else atomicOr(&cv.stats->error, 8u);
@@ -264,10 +266,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 tmem_ld32(tmSg + 96, vb);
                 stats32(va, 2);
                 tmem_ld_wait_for(vb);
-                stats32(vb, 3);
-                tc_fence_before();
+                tc_fence_before();  // last read of this S buffer: hand it back before the arithmetic on it
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(S_FREE + grp));
+                stats32(vb, 3);
                 ++use;
             }
             part_m[grp * 128 + row] = mrun;
