@@ -19,6 +19,8 @@
 // groups of four softmax warps (one tensor-memory lane quarter per warp); group g owns the S buffer, the P^T
 // buffer and the key tiles of parity g, so the two groups alternate tiles and overlap each other's latency.  All waits are bounded mbarrier waits; a wait that gives
 // up sets an error word and the CTA drains to its exit, where tensor memory is released.
+#include <type_traits>
+
 #include "common.cuh"
 #include "tma.cuh"
 
@@ -299,7 +301,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const bool full = __all_sync(0xffffffffu, rmin == 0) && rmax == 128;
             float colsum = 0.f;
             unsigned char* prow = base_ptr + (1 + kRing) * kSlot + grp * kSlot + row * 128;
-            auto probs32 = [&](const uint32_t (&v)[32], int cg) {
+            auto probs32 = [&](auto full_tag, const uint32_t (&v)[32], int cg) {
+                constexpr bool kFull = decltype(full_tag)::value;  // every (key, query) pair of the warp's rows is visible
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {  // 8 query columns -> one 16-byte chunk of the P^T row
                     float p[8];
@@ -310,7 +313,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float pe = ex2(fmaf(__uint_as_float(v[q4 * 8 + h4 * 4 + e]), sc2, ls[e]));
-                            if (full) {
+                            if constexpr (kFull) {
                                 p[h4 * 4 + e] = pe;
                             } else {
                                 const int r = cg * 32 + q4 * 8 + h4 * 4 + e;
@@ -332,18 +335,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tmem_ld32(tmSg, va);
             tmem_ld_wait_for(va);
             tmem_ld32(tmSg + 32, vb);
-            probs32(va, 0);
+            if (full) probs32(std::true_type{}, va, 0); else probs32(std::false_type{}, va, 0);
             tmem_ld_wait_for(vb);
             tmem_ld32(tmSg + 64, va);
-            probs32(vb, 1);
+            if (full) probs32(std::true_type{}, vb, 1); else probs32(std::false_type{}, vb, 1);
             tmem_ld_wait_for(va);
             tmem_ld32(tmSg + 96, vb);
-            probs32(va, 2);
+            if (full) probs32(std::true_type{}, va, 2); else probs32(std::false_type{}, va, 2);
             tmem_ld_wait_for(vb);
             tc_fence_before();  // last read of this S^T buffer
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(S_FREE + grp));
-            probs32(vb, 3);
+            if (full) probs32(std::true_type{}, vb, 3); else probs32(std::false_type{}, vb, 3);
             if (kvalid) part[lam] = colsum;
             fence_proxy_async_smem();
             __syncwarp();
