@@ -291,7 +291,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         float* part = ps.colsum + ((size_t)unit * ps.QT + qt) * ps.n_max;
         int puse = 0;  // times this group's P^T buffer has been filled
         for (int j = grp; j < NT && ok; j += 2) {
-            if (!mbar_wait(bar(S_FULL + grp), use & 1) || !mbar_wait(bar(P_FREE + grp), (puse & 1) ^ 1)) { ok = false; break; }
+            if (!mbar_wait(bar(S_FULL + grp), use & 1)) { ok = false; break; }
             tc_fence_after();
             int lam0, row0, valid;
             tile_of(kt, j, lam0, row0, valid);
@@ -335,6 +335,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tmem_ld32(tmSg, va);
             tmem_ld_wait_for(va);
             tmem_ld32(tmSg + 32, vb);
+            // the P^T buffer is only needed now: the O^T MMA of two tiles ago has had the time of the loads to finish
+            if (!mbar_wait(bar(P_FREE + grp), (puse & 1) ^ 1)) { ok = false; }
             if (full) probs32(std::true_type{}, va, 0); else probs32(std::false_type{}, va, 0);
             tmem_ld_wait_for(vb);
             tmem_ld32(tmSg + 64, va);
