@@ -117,22 +117,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tma_load_3d(sQ, &tmQ, 0, kh * G, b * chunk_stride + t0, bar(Q_FULL));
             tma_load_3d(sQ + kHalf, &tmQ, 64, kh * G, b * chunk_stride + t0, bar(Q_FULL));
             int ld = 0;
-            for (int pass = 0; pass < 2 && ok; ++pass) {
-                for (int j = 0; j < NT && ok; ++j) {
-                    int lam0, row0, valid;
-                    tile_of(kt, j, lam0, row0, valid);
-                    const int grow = unit * cv.R + row0;
-                    for (int which = 0; which <= pass; ++which) {  // pass A: K only; pass B: K then V
-                        const int slot = ld % kRing;
-                        if (!mbar_wait(bar(RING_EMPTY + slot), ((ld / kRing) & 1) ^ 1)) { ok = false; break; }
-                        const uint32_t dst = sRing + slot * kSlot;
-                        mbar_arrive_expect_tx(bar(RING_FULL + slot), kSlot);
-                        const CUtensorMap* mp = which == 0 ? &tmK : &tmV;
-                        tma_load_2d(dst, mp, 0, grow, bar(RING_FULL + slot));
-                        tma_load_2d(dst + kHalf, mp, 64, grow, bar(RING_FULL + slot));
-                        ++ld;
-                    }
-                }
+            auto load_tile = [&](const CUtensorMap* mp, int j) {
+                int lam0, row0, valid;
+                tile_of(kt, j, lam0, row0, valid);
+                const int grow = unit * cv.R + row0;
+                const int slot = ld % kRing;
+                if (!mbar_wait(bar(RING_EMPTY + slot), ((ld / kRing) & 1) ^ 1)) { ok = false; return; }
+                const uint32_t dst = sRing + slot * kSlot;
+                mbar_arrive_expect_tx(bar(RING_FULL + slot), kSlot);
+                tma_load_2d(dst, mp, 0, grow, bar(RING_FULL + slot));
+                tma_load_2d(dst + kHalf, mp, 64, grow, bar(RING_FULL + slot));
+                ++ld;
+            };
+            // pass A: K tiles in order.  Pass B: the same order in which the MMA warp consumes them - K runs three
+            // tiles ahead of V (K_0 K_1 K_2 | V_0 K_3 | V_1 K_4 | ...), so a K tile is requested as soon as the S^T
+            // two tiles back has executed and its load latency hides behind two tiles of work.
+            for (int j = 0; j < NT && ok; ++j) load_tile(&tmK, j);
+            for (int j = 0; j < 3 && j < NT && ok; ++j) load_tile(&tmK, j);
+            for (int j = 0; j < NT && ok; ++j) {
+                load_tile(&tmV, j);
+                if (ok && j + 3 < NT) load_tile(&tmK, j + 3);
             }
             if (!ok) atomicOr(&cv.stats->error, 4u);
         }
@@ -165,7 +169,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             //      owns buffer j & 1 finds S^T_{j+2} ready when it finishes tile j (its buffer is free as soon as
             //      it has read tile j into registers, long before P_j^T is complete)
             auto issue_st = [&](int j) {
-                const int ld = NT + 2 * j, slot = ld % kRing, buf = j & 1;
+                const int ld = NT + (j < 3 ? j : 2 * j - 2), slot = ld % kRing, buf = j & 1;  // see the producer's load order
                 ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), (use[buf] & 1) ^ 1);
                 if (!ok) return;
                 tc_fence_after();
@@ -184,7 +188,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int pj = 0; pj < NT && ok; ++pj) {
                 if (pj + 2 < NT) { issue_st(pj + 2); if (!ok) break; }
                 const int pbuf = pj & 1;
-                const int ld = NT + 2 * pj + 1, slot = ld % kRing;
+                const int ld = NT + min(3, NT) + pj + min(pj, max(0, NT - 3)), slot = ld % kRing;
                 ok = mbar_wait(bar(P_FULL + pbuf), (pj >> 1) & 1) && mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1);
                 if (!ok) break;
                 tc_fence_after();
