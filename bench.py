@@ -6,8 +6,10 @@ Headline (value): decode steps/s on the Llama-2-7B-shaped configuration (32 laye
 bf16, budget 1024) with every cache full, one step = all 32 layers in order, inputs resident in HBM.
 `e2e`: the same step through the *_host entry points: host->device copies of q,k,v and the device->host copy
 of the output are inside the timed region, every step.
-`prefill`: chunked-prefill tokens/s on the Llama-2-7B-shaped prefill configuration (chunks of 512 to budget
-2048), steady state, with its own roofline entry.
+`prefill`: chunked-prefill tokens/s (through all layers) on the Llama-3-8B-shaped prefill configuration (batch 4,
+chunks of 1024 to budget 4096), steady state with full chunks, with its own tensor roofline entry.
+`decode_alt` / `prefill_alt`: the same two measurements on the other decode (Llama-3-8B GQA, batch 32, budget 2048)
+and prefill (Llama-2-7B, chunks of 512 to budget 2048) configurations.
 `roofline`: algorithmic bytes of one decode launch / its average duration, against the measured copy bandwidth.
 `cpu_baseline`: the fp64 oracle timed on this host's cores on a bounded sample of the same workload.
 
@@ -188,7 +190,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg4"])
-    ap.add_argument("--prefill-workload", default="cfg3", choices=["cfg3", "cfg5"])
+    ap.add_argument("--prefill-workload", default="cfg5", choices=["cfg3", "cfg5"])
+    ap.add_argument("--no-alt", action="store_true", help="skip the second decode and prefill configurations")
     ap.add_argument("--prefill-chunks", type=int, default=4, help="timed steady-state chunks (0 = skip the prefill leg)")
     ap.add_argument("--e2e-steps", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -224,9 +227,6 @@ def main():
     from paper_2501_04987_b200 import binding
 
     peaks = measured_peaks()
-    e = 2 if w.dtype == "bf16" else 4
-    tdtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
-    g = w.group
 
     def barrier():
         if world > 1:
@@ -240,12 +240,69 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    # ------------------------------------------------------------------ decode leg
+    # ------------------------------------------------------------------ decode leg (headline) + e2e
+    dec = run_decode_leg(torch, binding, w, args.steps, max(3, args.warmup), args.e2e_steps, args.decode_split, dev, world,
+                         rank, local_rank, barrier, max_over_ranks, peaks, sample_clocks=True)
+    steps_per_s, ms_per_step, launches = dec["value"], dec["ms_per_step"], dec["gpu_launches"]
+    roofline, e2e, clocks, bytes_per_launch = dec["roofline"], dec["e2e"], dec["clocks"], dec["roofline"]["bytes_per_launch"]
+    decode_alt = None
+    if not args.no_alt:
+        wa = W.CONFIGS["cfg4" if w.name == "cfg2" else "cfg2"]
+        if args.layers:
+            wa = W.parity_slice(wa, layers=args.layers)
+        decode_alt = run_decode_leg(torch, binding, wa, max(16, args.steps // 4), 3, 0, args.decode_split, dev, world, rank,
+                                    local_rank, barrier, max_over_ranks, peaks, sample_clocks=False)
+
+    # ------------------------------------------------------------------ prefill leg
+    prefill = None
+    if args.prefill_chunks > 0:
+        pw = W.CONFIGS[args.prefill_workload]
+        if args.layers:
+            pw = W.parity_slice(pw, layers=args.layers)
+        prefill = run_prefill_leg(torch, binding, pw, args.prefill_chunks, dev, world, rank, barrier, max_over_ranks, peaks)
+    prefill_alt = None
+    if args.prefill_chunks > 0 and not args.no_alt:
+        pa = W.CONFIGS["cfg3" if args.prefill_workload == "cfg5" else "cfg5"]
+        if args.layers:
+            pa = W.parity_slice(pa, layers=args.layers)
+        prefill_alt = run_prefill_leg(torch, binding, pa, args.prefill_chunks, dev, world, rank, barrier, max_over_ranks, peaks)
+
+    # ------------------------------------------------------------------ oracle on the host cores
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        val, cores, desc = time_oracle_decode(w, min(2, w.batch), 300)
+        cpu_baseline = {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        line = {
+            "metric": "treekv_decode_steps_per_s", "value": steps_per_s, "unit": "steps/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": w.name, "layers": w.layers, "batch_per_gpu": w.batch, "n_heads": w.n_heads,
+                       "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "budget": w.budget,
+                       "parallelism": "replicas x%d" % world,
+                       "l2": "no flush: one step streams %.2f GB of K/V (%.0f MB per layer) through a 126 MB L2"
+                             % (w.layers * bytes_per_launch / 1e9, bytes_per_launch / 1e6)},
+            "tokens_per_s": steps_per_s * w.batch,
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
+            "cpu_baseline": cpu_baseline, "prefill": prefill, "decode_alt": decode_alt, "prefill_alt": prefill_alt,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_decode_leg(torch, binding, w, steps, warmup, e2e_steps, decode_split, dev, world, rank, local_rank, barrier,
+                   max_over_ranks, peaks, sample_clocks):
+    """Decode steps/s of one configuration with every cache full; optionally the same through the host entry points."""
+    e = 2 if w.dtype == "bf16" else 4
+    tdtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    g = w.group
     wr = W.parity_slice(w, seed=w.seed + 1000 * rank)
     ctxs = [binding.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, 0) for _ in range(w.layers)]
-    if args.decode_split:
+    if decode_split:
         for c in ctxs:
-            c.set_option(binding.OPT_DECODE_SPLIT, args.decode_split)
+            c.set_option(binding.OPT_DECODE_SPLIT, decode_split)
     ring = 4
     ins = []
     for layer in range(w.layers):
@@ -266,93 +323,68 @@ def main():
                     raise RuntimeError("treekv_decode_step: " + binding.status_string(st))
 
     fill = w.budget + 37
-    decode_steps(fill, 0)                      # fill every cache (untimed)
-    decode_steps(max(3, args.warmup), fill)    # warm-up
+    decode_steps(fill, 0)          # fill every cache (untimed)
+    decode_steps(warmup, fill)     # warm-up
     launches0 = sum(c.stats()["kernel_launches"] for c in ctxs)
     sampler = ClockSampler(physical_gpu_index(local_rank))
     barrier()
-    if rank == 0:
+    if rank == 0 and sample_clocks:
         sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
-    decode_steps(args.steps, fill + args.warmup)
+    decode_steps(steps, fill + warmup)
     ev1.record()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop() if (rank == 0 and sample_clocks) else None
     ms_total = max_over_ranks(ev0.elapsed_time(ev1))
     launches = sum(c.stats()["kernel_launches"] for c in ctxs) - launches0
-    ms_per_step = ms_total / args.steps
+    ms_per_step = ms_total / steps
     steps_per_s = world * 1000.0 / ms_per_step
 
     units = w.batch * w.n_kv_heads
     bytes_per_launch = units * decode_bytes_per_unit(w.budget, w.head_dim, e, g)
-    launch_ms = ms_total / (args.steps * w.layers)
+    launch_ms = ms_total / (steps * w.layers)
     achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
-                "kernel": "decode_kernel", "bytes_per_launch": bytes_per_launch, "launch_us": launch_ms * 1e3,
-                "frac_of_nominal_8TBs": achieved / 8000.0}
+                "kernel": "decode_mma_kernel" if w.dtype == "bf16" else "decode_kernel",
+                "bytes_per_launch": bytes_per_launch, "launch_us": launch_ms * 1e3, "frac_of_nominal_8TBs": achieved / 8000.0}
 
-    # ------------------------------------------------------------------ e2e leg: host buffers through the C ABI
-    nb_q = w.batch * w.n_heads * w.head_dim * e
-    nb_k = w.batch * w.n_kv_heads * w.head_dim * e
-    h_in = [tuple(x.cpu().pin_memory() for x in ins[layer]) for layer in range(w.layers)]
-    h_out = [torch.empty((w.batch, w.n_heads, w.head_dim), dtype=tdtype).pin_memory() for _ in range(w.layers)]
+    e2e = None
+    if e2e_steps > 0:
+        # host buffers through the C ABI: pinned q,k,v copied in and the output copied back, every layer, every step
+        nb_q = w.batch * w.n_heads * w.head_dim * e
+        nb_k = w.batch * w.n_kv_heads * w.head_dim * e
+        h_in = [tuple(x.cpu().pin_memory() for x in ins[layer]) for layer in range(w.layers)]
+        h_out = [torch.empty((w.batch, w.n_heads, w.head_dim), dtype=tdtype).pin_memory() for _ in range(w.layers)]
 
-    def e2e_steps(n):
-        for s in range(n):
-            r = s % ring
-            for layer in range(w.layers):
-                q, k, v = h_in[layer]
-                st = binding.lib.treekv_decode_step_host(ctxs[layer]._h, q[r].data_ptr(), k[r].data_ptr(),
-                                                         v[r].data_ptr(), h_out[layer].data_ptr(), None, stream)
-                if st != 0:
-                    raise RuntimeError("treekv_decode_step_host: " + binding.status_string(st))
+        def e2e_run(n):
+            for s in range(n):
+                r = s % ring
+                for layer in range(w.layers):
+                    q, k, v = h_in[layer]
+                    st = binding.lib.treekv_decode_step_host(ctxs[layer]._h, q[r].data_ptr(), k[r].data_ptr(),
+                                                             v[r].data_ptr(), h_out[layer].data_ptr(), None, stream)
+                    if st != 0:
+                        raise RuntimeError("treekv_decode_step_host: " + binding.status_string(st))
 
-    e2e_n = max(1, min(args.e2e_steps, args.steps))
-    e2e_steps(3)
-    barrier()
-    ev0.record()
-    e2e_steps(e2e_n)
-    ev1.record()
-    barrier()
-    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_n
-    e2e = {"value": world * 1000.0 / e2e_ms, "unit": "steps/s", "h2d_bytes_per_step": w.layers * (nb_q + 2 * nb_k),
-           "d2h_bytes_per_step": w.layers * nb_q, "steps": e2e_n, "ms_per_step": e2e_ms}
+        e2e_n = max(1, min(e2e_steps, steps))
+        e2e_run(3)
+        barrier()
+        ev0.record()
+        e2e_run(e2e_n)
+        ev1.record()
+        barrier()
+        e2e_ms = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_n
+        e2e = {"value": world * 1000.0 / e2e_ms, "unit": "steps/s", "h2d_bytes_per_step": w.layers * (nb_q + 2 * nb_k),
+               "d2h_bytes_per_step": w.layers * nb_q, "steps": e2e_n, "ms_per_step": e2e_ms}
     del ctxs, ins, outs
     torch.cuda.empty_cache()
-
-    # ------------------------------------------------------------------ prefill leg
-    prefill = None
-    if args.prefill_chunks > 0:
-        pw = W.CONFIGS[args.prefill_workload]
-        if args.layers:
-            pw = W.parity_slice(pw, layers=args.layers)
-        prefill = run_prefill_leg(torch, binding, pw, args.prefill_chunks, dev, world, rank, barrier, max_over_ranks, peaks)
-
-    # ------------------------------------------------------------------ oracle on the host cores
-    cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        val, cores, desc = time_oracle_decode(w, min(2, w.batch), 300)
-        cpu_baseline = {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc}
-
-    if rank == 0:
-        line = {
-            "metric": "treekv_decode_steps_per_s", "value": steps_per_s, "unit": "steps/s", "n_gpus": world,
-            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
-            "config": {"workload": w.name, "layers": w.layers, "batch_per_gpu": w.batch, "n_heads": w.n_heads,
-                       "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "budget": w.budget,
-                       "parallelism": "replicas x%d" % world,
-                       "l2": "no flush: one step streams %.2f GB of K/V (%.0f MB per layer) through a 126 MB L2"
-                             % (w.layers * bytes_per_launch / 1e9, bytes_per_launch / 1e6)},
+    return {"metric": "treekv_decode_steps_per_s", "value": steps_per_s, "unit": "steps/s", "steps": steps,
+            "ms_per_step": ms_per_step, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "e2e": e2e,
             "tokens_per_s": steps_per_s * w.batch,
-            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
-            "cpu_baseline": cpu_baseline, "prefill": prefill,
-        }
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+            "config": {"workload": w.name, "layers": w.layers, "batch_per_gpu": w.batch, "n_heads": w.n_heads,
+                       "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "budget": w.budget}}
 
 
 def run_prefill_leg(torch, binding, pw, n_chunks, dev, world, rank, barrier, max_over_ranks, peaks):
@@ -360,7 +392,7 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, world, rank, barrier, max
     m, c = pw.chunk, pw.budget
     ctxs = [binding.TreeKV(c, pw.n_heads, pw.n_kv_heads, pw.head_dim, pw.dtype, pw.batch, m) for _ in range(pw.layers)]
     wr = W.parity_slice(pw, seed=pw.seed + 1000 * rank)
-    ring = 2
+    ring = 1  # the same chunk values every call: timing does not depend on them
     ins = []
     for layer in range(pw.layers):
         chunks = []
@@ -396,6 +428,8 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, world, rank, barrier, max
     flops_chunk = pw.layers * pw.batch * pw.n_heads * prefill_flops_per_head_chunk(m, c, pw.head_dim)
     achieved = flops_chunk * n_chunks / (ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
+    del ctxs, ins
+    torch.cuda.empty_cache()
     return {"metric": "treekv_prefill_tokens_per_s", "value": tok_s, "unit": "tokens/s", "chunks": n_chunks,
             "ms_per_chunk_all_layers": ms / n_chunks, "gpu_launches": int(launches),
             "config": {"workload": pw.name, "layers": pw.layers, "batch_per_gpu": pw.batch, "n_heads": pw.n_heads,

@@ -83,9 +83,11 @@ _TOKEN_BLOCK = 256
 _TENSOR_ID = {"q": 0, "k": 1, "v": 2}
 
 
-def _normal_block(seed: int, tensor: str, layer: int, seq: int, blk: int, n_heads: int, d: int) -> np.ndarray:
+def _normal_block(seed: int, tensor: str, layer: int, seq: int, blk: int, n_heads: int, d: int, rows: int = _TOKEN_BLOCK) -> np.ndarray:
+    """First `rows` tokens of a 256-token block (the generator fills the block token by token, so a prefix of the
+    block is the same whether or not the rest is drawn)."""
     bitgen = np.random.Philox(key=seed, counter=[blk, seq, layer, _TENSOR_ID[tensor]])
-    return np.random.Generator(bitgen).standard_normal((_TOKEN_BLOCK, n_heads, d), dtype=np.float32)
+    return np.random.Generator(bitgen).standard_normal((rows, n_heads, d), dtype=np.float32)
 
 
 def _normal_tokens(seed, tensor, layer, seq, t0, t1, n_heads, d):
@@ -95,7 +97,7 @@ def _normal_tokens(seed, tensor, layer, seq, t0, t1, n_heads, d):
         blk = t // _TOKEN_BLOCK
         lo = t - blk * _TOKEN_BLOCK
         hi = min(_TOKEN_BLOCK, t1 - blk * _TOKEN_BLOCK)
-        out[t - t0 : t - t0 + hi - lo] = _normal_block(seed, tensor, layer, seq, blk, n_heads, d)[lo:hi]
+        out[t - t0 : t - t0 + hi - lo] = _normal_block(seed, tensor, layer, seq, blk, n_heads, d, hi)[lo:hi]
         t += hi - lo
     return out
 
