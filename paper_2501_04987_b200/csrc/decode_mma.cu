@@ -124,19 +124,40 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     }
 
     const uint32_t ring_w = smem_u32(ring) + warp * NS * STAGE;
+    // Copy of one 16-row block: lane (half = lane / CPR... ) moves 16-byte chunk `cidx` of rows rsub*(16/RPI) + it.
+    // Shared-memory layout of a tile: row r at r * ROWB, its 16-byte chunk c at position c ^ (r & 7).
+    constexpr int RPI = 32 / CPR;          // rows copied per warp-wide cp.async (2 for d=128, 4 for d=64)
+    constexpr int ITERS = kBlk / RPI;      // iterations per tile (8 or 4)
+    const int c_rsub = lane / CPR, c_cidx = lane % CPR;
+    const uint32_t c_lane_off = c_rsub * ITERS * ROWB;  // lane's first row = rsub * ITERS
+    const int c_row7 = (c_rsub * ITERS) & 7;            // (row & 7) of iteration `it` is c_row7 + it (no carry)
     auto issue = [&](int blk, int stage) {
         if (blk < nblk) {
             const uint32_t kst = ring_w + stage * STAGE, vst = kst + kBlk * ROWB;
+            const int lam0 = lo + blk * kBlk;
+            // fast path: all 16 rows exist, none is the new token, and they are consecutive physical rows
+            const bool whole = (lam0 + kBlk <= hi) && (lam0 + kBlk <= n - 1) && (lam0 >= i_cyc || lam0 + kBlk <= i_cyc);
+            if (whole) {
+                const size_t r0 = (size_t)phys_row(lam0, i_cyc) + c_rsub * ITERS;
+                const unsigned char* ks = reinterpret_cast<const unsigned char*>(Kc) + r0 * ROWB + c_cidx * 16;
+                const unsigned char* vs = reinterpret_cast<const unsigned char*>(Vc) + r0 * ROWB + c_cidx * 16;
 #pragma unroll
-            for (int it = 0; it < kBlk * CPR / 32; ++it) {
-                const int x = it * 32 + lane;
-                const int row = x / CPR, cidx = x % CPR;
-                const int lam = lo + blk * kBlk + row;
-                const bool valid = lam < hi && lam != n - 1;  // the new token is merged separately
-                const size_t ro = valid ? (size_t)phys_row(lam, i_cyc) * D : 0;
-                const uint32_t off = row * ROWB + ((cidx ^ (row & 7)) << 4);
-                cp_async_16(kst + off, reinterpret_cast<const unsigned char*>(Kc + ro) + cidx * 16, valid);
-                cp_async_16(vst + off, reinterpret_cast<const unsigned char*>(Vc + ro) + cidx * 16, valid);
+                for (int it = 0; it < ITERS; ++it) {
+                    const uint32_t off = c_lane_off + it * ROWB + ((c_cidx ^ (c_row7 + it)) << 4);
+                    cp_async_16(kst + off, ks + it * ROWB, true);
+                    cp_async_16(vst + off, vs + it * ROWB, true);
+                }
+            } else {
+#pragma unroll
+                for (int it = 0; it < ITERS; ++it) {
+                    const int row = c_rsub * ITERS + it;
+                    const int lam = lam0 + row;
+                    const bool valid = lam < hi && lam != n - 1;  // the new token is merged separately
+                    const size_t ro = valid ? (size_t)phys_row(lam, i_cyc) * ROWB : 0;
+                    const uint32_t off = c_lane_off + it * ROWB + ((c_cidx ^ (c_row7 + it)) << 4);
+                    cp_async_16(kst + off, reinterpret_cast<const unsigned char*>(Kc) + ro + c_cidx * 16, valid);
+                    cp_async_16(vst + off, reinterpret_cast<const unsigned char*>(Vc) + ro + c_cidx * 16, valid);
+                }
             }
         }
         cp_async_commit();
@@ -154,6 +175,20 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
             qa[kk][0] = *reinterpret_cast<const uint32_t*>(qh);
             qa[kk][1] = *reinterpret_cast<const uint32_t*>(qh + 8);
         }
+    }
+
+    // per-lane ldmatrix offsets inside a K tile (4 matrices = 8 keys x 32 channels) and a V tile (4 matrices = 16 keys
+    // x 16 channels), swizzle included; the row half hb adds 8 rows
+    uint32_t koff[D / 32], voff[D / 16];
+#pragma unroll
+    for (int u = 0; u < D / 32; ++u) {
+        const int row = lane & 7, cidx = 4 * u + (lane >> 3);
+        koff[u] = row * ROWB + ((cidx ^ row) << 4);
+    }
+#pragma unroll
+    for (int cc = 0; cc < D / 16; ++cc) {
+        const int row = (lane & 7) + ((lane >> 4) << 3), cidx = 2 * cc + ((lane >> 3) & 1);
+        voff[cc] = row * ROWB + ((cidx ^ (row & 7)) << 4);
     }
 
     float m_run = -INFINITY, l_run = 0.f;  // of head g (replicated over the 4 lanes t; l_run is a per-lane partial)
@@ -181,9 +216,8 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         for (int u = 0; u < D / 32; ++u) {
 #pragma unroll
             for (int hb = 0; hb < 2; ++hb) {
-                const int row = hb * 8 + (lane & 7), cidx = 4 * u + (lane >> 3);
                 uint32_t r0, r1, r2, r3;
-                ldmatrix_x4(kst + row * ROWB + ((cidx ^ (row & 7)) << 4), r0, r1, r2, r3);
+                ldmatrix_x4(kst + hb * 8 * ROWB + koff[u], r0, r1, r2, r3);
                 mma_bf16(c[hb], qa[2 * u][0], 0u, qa[2 * u][1], 0u, r0, r1);
                 mma_bf16(c[hb], qa[2 * u + 1][0], 0u, qa[2 * u + 1][1], 0u, r2, r3);
             }
@@ -220,9 +254,8 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         // ---- o^T[ch][head] += V^T[ch][key] P^T[key][head]
 #pragma unroll
         for (int cc = 0; cc < D / 16; ++cc) {
-            const int row = (lane & 7) + ((lane >> 4) << 3), cidx = 2 * cc + ((lane >> 3) & 1);
             uint32_t r0, r1, r2, r3;
-            ldmatrix_x4_trans(vst + row * ROWB + ((cidx ^ (row & 7)) << 4), r0, r1, r2, r3);
+            ldmatrix_x4_trans(vst + voff[cc], r0, r1, r2, r3);
             mma_bf16(acc[cc], r0, r1, r2, r3, pb0, pb1);
         }
         __syncwarp();
