@@ -109,6 +109,10 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     float* wstat = sl + (size_t)G * rows_cap;                              // [NW+1][2][G] per-warp (max, sum); slot NW = new token
     float* gstat = wstat + (NW + 1) * 2 * G;                               // [nsplit][2][G] every CTA's (max, sum), pushed by its owner
     float* o_all = gstat + kMaxSplit * 2 * G;                              // [nsplit][G][D] partial outputs, pushed into CTA 0 only
+    float* s_old = o_all + (size_t)nsplit * G * D;                         // [rows_cap] S of this CTA's rows, prefetched
+    unsigned char* pair_kv = reinterpret_cast<unsigned char*>(                   // [4][ROWB] K,V of the scope's two rows
+        (reinterpret_cast<uintptr_t>(s_old + rows_cap) + 15) & ~uintptr_t(15));
+    float* pair_s = reinterpret_cast<float*>(pair_kv + 4 * ROWB);          // [2] updated S of rows 2i, 2i+1 (split == 1)
     float* o_warp = reinterpret_cast<float*>(ring);                        // [NW][G][D], aliases the ring after the loop
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -162,8 +166,56 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         }
         cp_async_commit();
     };
+    // ---- prefetch what the epilogue needs, so that after the streaming loop nothing waits on a global load:
+    //      S of this CTA's rows (4-byte cp.async; they join the first commit group), and in CTA 0 the K/V rows of
+    //      the eviction scope (rows 2i and 2i+1; the new token's row comes from k_in / v_in)
+    const bool will_evict = (N + 1 > cv.c);
+    int pos_l = 0, pos_r = 0;  // stream positions of the scope's two tokens (used by lane 0 of warp 0 in CTA 0)
+    if (rank == 0 && will_evict && tid == 0) {
+        pos_l = Pc[2 * i_cyc];
+        pos_r = (2 * i_cyc + 1 == new_row) ? N : Pc[2 * i_cyc + 1];
+    }
+    for (int j = tid; j < nrows; j += NT) {
+        const int lam = lo + j;
+        if (lam != n - 1)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(s_old + j)), "l"(Sc + phys_row(lam, i_cyc)) : "memory");
+    }
+    if (rank == 0 && will_evict && warp == NW - 1) {
+        for (int e = lane; e < 4 * CPR; e += 32) {
+            const int which = e / CPR, cidx = e % CPR;   // 0: K left, 1: K right, 2: V left, 3: V right
+            const int prow = 2 * i_cyc + (which & 1);
+            const T* srcrow = (prow == new_row) ? ((which < 2) ? k_new : v_new)
+                                                : ((which < 2) ? Kc : Vc) + (size_t)prow * D;
+            cp_async_16(smem_u32(pair_kv + which * ROWB + cidx * 16), reinterpret_cast<const unsigned char*>(srcrow) + cidx * 16, true);
+        }
+    }
 #pragma unroll
     for (int s = 0; s < NS; ++s) issue(warp + s * NW, s);
+
+    // ---- the new token's logit q.k_new (warp 0 of the owning CTA), computed while the first tiles are in flight
+    if (warp == 0) {
+        float sn[G];
+#pragma unroll
+        for (int h = 0; h < G; ++h) sn[h] = -INFINITY;
+        if (owns_new) {
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                float a = 0.f;
+                for (int e = lane; e < D; e += 32)
+                    a += __bfloat162float(q[((size_t)b * cv.Hq + kh * G + h) * D + e]) * __bfloat162float(k_new[e]);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+                sn[h] = a * scale;
+            }
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                wstat[(NW * 2 + 0) * G + h] = sn[h];
+                wstat[(NW * 2 + 1) * G + h] = owns_new ? 1.f : 0.f;
+            }
+        }
+    }
 
     // ---- A fragments of q: row g = head, k = channel; rows >= G are zero
     uint32_t qa[D / 16][2];
@@ -276,31 +328,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
             if (head < G) o_warp[(warp * G + head) * D + ch] = acc[cc][e];
         }
     }
-    // ---- the new token as one more partial: logit q.k_new, weight 1, value v_new (warp 0 of the owning CTA)
-    if (warp == 0) {
-        float sn[G];
-#pragma unroll
-        for (int h = 0; h < G; ++h) sn[h] = -INFINITY;
-        if (owns_new) {
-#pragma unroll
-            for (int h = 0; h < G; ++h) {
-                float a = 0.f;
-                for (int e = lane; e < D; e += 32)
-                    a += __bfloat162float(q[((size_t)b * cv.Hq + kh * G + h) * D + e]) * __bfloat162float(k_new[e]);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-                sn[h] = a * scale;
-            }
-        }
-        if (lane == 0) {
-#pragma unroll
-            for (int h = 0; h < G; ++h) {
-                wstat[(NW * 2 + 0) * G + h] = sn[h];
-                wstat[(NW * 2 + 1) * G + h] = owns_new ? 1.f : 0.f;
-                if (owns_new) sl[h * rows_cap + (n - 1 - lo)] = sn[h];
-            }
-        }
-    }
+    if (owns_new && tid < G) sl[tid * rows_cap + (n - 1 - lo)] = wstat[(NW * 2 + 0) * G + tid];  // the new token's logit
     __syncthreads();
 
     // ---- CTA partial: (max, sum) per head and the output relative to the CTA max, pushed with remote stores
@@ -358,45 +386,46 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         for (int h = 0; h < G; ++h) ps += exp2_diff(sl[h * rows_cap + j], Mg[h]) * invL[h];
         const int lam = lo + j;
         const int ph = phys_row(lam, i_cyc);
-        const float s_old = (lam == n - 1) ? 0.f : Sc[ph];
-        Sc[ph] = s_old + ps * (1.0f / G);
+        const float s_new = ((lam == n - 1) ? 0.f : s_old[j]) + ps * (1.0f / G);
+        Sc[ph] = s_new;
         if (lam == n - 1) Pc[ph] = N;
+        if (nsplit == 1 && (ph >> 1) == i_cyc) pair_s[ph & 1] = s_new;  // the scope's scores stay on chip
     }
 
     cluster.sync();  // (B) the appended row and every S update of the unit are complete
 
-    if (rank == 0 && warp == 0) {
+    if (rank == 0 && warp == 0 && will_evict) {
         // ---- Algorithm 1, "length > c" branch: scope {idx, idx+1} = physical rows (2i, 2i+1)
         const int N1 = N + 1;
-        if (N1 > cv.c) {
-            const int l = 2 * i_cyc, r = l + 1;
-            int evict_right = 0;
-            if (lane == 0) {
-                bool near_tie = false;
-                evict_right = pair_evicts_right(__ldcg(Sc + l), N1 - __ldcg(Pc + l), __ldcg(Sc + r), N1 - __ldcg(Pc + r),
-                                                cv.rule, &near_tie) ? 1 : 0;
-                if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
-            }
-            evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
-            const int src = evict_right ? l : r, dst = i_cyc;
-            if (src != dst) {
-                for (int e = lane; e < CHUNKS; e += 32) {
-                    const uint4 kk = __ldcg(reinterpret_cast<const uint4*>(Kc + (size_t)src * D) + e);
-                    const uint4 vv = __ldcg(reinterpret_cast<const uint4*>(Vc + (size_t)src * D) + e);
-                    reinterpret_cast<uint4*>(Kc + (size_t)dst * D)[e] = kk;
-                    reinterpret_cast<uint4*>(Vc + (size_t)dst * D)[e] = vv;
-                }
-                if (lane == 0) { Sc[dst] = __ldcg(Sc + src); Pc[dst] = __ldcg(Pc + src); }
+        const int l = 2 * i_cyc, r = l + 1;
+        int evict_right = 0;
+        if (lane == 0) {
+            bool near_tie = false;
+            const float S_l = nsplit == 1 ? pair_s[0] : __ldcg(Sc + l);
+            const float S_r = nsplit == 1 ? pair_s[1] : __ldcg(Sc + r);
+            evict_right = pair_evicts_right(S_l, N1 - pos_l, S_r, N1 - pos_r, cv.rule, &near_tie) ? 1 : 0;
+            if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
+            const int src = evict_right ? l : r;
+            if (src != i_cyc) { Sc[i_cyc] = evict_right ? S_l : S_r; Pc[i_cyc] = evict_right ? pos_l : pos_r; }
+        }
+        evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
+        const int src = evict_right ? l : r, dst = i_cyc;
+        if (src != dst) {  // survivor's K and V rows were staged in shared memory at kernel start
+            const unsigned char* ksrc = pair_kv + (evict_right ? 0 : 1) * ROWB;
+            const unsigned char* vsrc = pair_kv + (evict_right ? 2 : 3) * ROWB;
+            for (int e = lane; e < CHUNKS; e += 32) {
+                reinterpret_cast<uint4*>(Kc + (size_t)dst * D)[e] = reinterpret_cast<const uint4*>(ksrc)[e];
+                reinterpret_cast<uint4*>(Vc + (size_t)dst * D)[e] = reinterpret_cast<const uint4*>(vsrc)[e];
             }
         }
-        if (lane == 0) cv.n_seen[unit] = N1;
     }
+    if (rank == 0 && tid == 0) cv.n_seen[unit] = N + 1;
 }
 
 size_t decode_mma_smem_bytes(int G, int D, int c, int split) {
     const size_t ring = (size_t)kMmaWarps * kMmaStages * 2 * kBlk * D * 2;
     return ring + sizeof(float) * ((size_t)G * mma_rows_cap(c, split) + (kMmaWarps + 1) * 2 * G + kMaxSplit * 2 * G +
-                                   (size_t)split * G * D);
+                                   (size_t)split * G * D + (size_t)mma_rows_cap(c, split) + 2) + 4 * (size_t)D * 2 + 16;
 }
 
 template <int D, int G>
