@@ -170,6 +170,8 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     //      S of this CTA's rows (4-byte cp.async; they join the first commit group), and in CTA 0 the K/V rows of
     //      the eviction scope (rows 2i and 2i+1; the new token's row comes from k_in / v_in)
     const bool will_evict = (N + 1 > cv.c);
+    static_assert(NT % D == 0, "a thread always combines the same channel");
+    const float vnew_r = owns_new ? __bfloat162float(v_new[tid % D]) : 0.f;  // this thread's channel of the new value row
     int pos_l = 0, pos_r = 0;  // stream positions of the scope's two tokens (used by lane 0 of warp 0 in CTA 0)
     if (rank == 0 && will_evict && tid == 0) {
         pos_l = Pc[2 * i_cyc];
@@ -346,7 +348,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         }
         if (owns_new) {
             const float f = exp2_diff(wstat[(NW * 2) * G + h], M);
-            o += __bfloat162float(v_new[ch]) * f;
+            o += vnew_r * f;
             l += f;
         }
         o_all0[(size_t)rank * G * D + idx] = o;
@@ -434,8 +436,15 @@ static cudaError_t launch_decode_mma_t(const CacheView& cv, const void* q, const
     auto kern = decode_mma_kernel<D, G, kMmaWarps, kMmaStages>;
     const int rows_cap = mma_rows_cap(cv.c, split);
     const size_t smem = decode_mma_smem_bytes(G, D, cv.c, split);
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    static size_t smem_set[64] = {};  // per device: the opt-in limit only ever needs raising
+    int dev = 0;
+    cudaGetDevice(&dev);
+    dev &= 63;
+    if (smem > smem_set[dev]) {
+        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        smem_set[dev] = smem;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(split, cv.Hkv, cv.B);
     cfg.blockDim = dim3(kMmaWarps * 32);
