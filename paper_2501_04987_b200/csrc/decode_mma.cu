@@ -92,8 +92,8 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     const int blk_per = (nblk_all + nsplit - 1) / nsplit;
     const int lo = min(rank * blk_per * kBlk, n), hi = min(lo + blk_per * kBlk, n);
     const int nrows = hi - lo;
-    const int nblk = (nrows + kBlk - 1) / kBlk;
     const bool owns_new = (hi == n) && nrows > 0;
+    const int nblk = (nrows - (owns_new ? 1 : 0) + kBlk - 1) / kBlk;  // tiles of cached rows; the new token is merged separately
 
     T* Kc = reinterpret_cast<T*>(cv.K) + (size_t)unit * cv.R * D;
     T* Vc = reinterpret_cast<T*>(cv.V) + (size_t)unit * cv.R * D;

@@ -1,0 +1,196 @@
+"""Parity at the configurations' full per-layer sizes, in the launch configuration the benchmark times.
+
+One layer of each configuration is run at its full batch / head count / budget / chunk size.  The oracle cannot
+follow every unit at these sizes, so:
+  * decode (configuration 2's shape): single-head oracles follow sampled (sequence, head) units in lock-step;
+  * chunked prefill (configurations 4 and 5): sampled output rows are recomputed one by one in fp64 as plain
+    softmax attention over [tokens retained before the chunk | chunk tokens up to the row's own] from the raw
+    input stream, and the cache invariants that hold at any size are checked after every call (length = min(seen,
+    budget), strictly increasing positions, every averaged score in [0, 1]).
+Inputs are seeded Gaussians drawn with torch on the device (keys with the configuration's outlier channels or
+per-sequence scale; no rotary embedding here - the lock-step tests on slices use the full recipe).
+"""
+import math
+
+import numpy as np
+import pytest
+
+import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2501_04987_b200 import _build
+
+    _build.build()
+    from paper_2501_04987_b200 import binding
+
+    return binding
+
+
+def _draw(torch, gen, shape, scale_last=None, seq_scale=None):
+    x = torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32)
+    if scale_last is not None:
+        x[..., scale_last] *= 8.0
+    if seq_scale is not None:
+        x *= seq_scale.view(-1, *([1] * (x.dim() - 1)))
+    return x.to(torch.bfloat16)
+
+
+def _softmax_rows(q, K, V):
+    s = K @ q / math.sqrt(q.shape[0])
+    s -= s.max()
+    p = np.exp(s)
+    p /= p.sum()
+    return p @ V
+
+
+def _check_invariants(kv, seen):
+    pos, cnt = kv.retained_positions()
+    pos = pos.cpu().numpy(); cnt = cnt.cpu().numpy()
+    sb = kv.scores().cpu().numpy()
+    B = pos.shape[0]
+    for b in range(B):
+        want = min(seen[b], kv.budget)
+        assert np.all(cnt[b] == want)
+        if want > 1:
+            assert np.all(np.diff(pos[b, :, :want], axis=1) > 0)
+        if want:
+            assert np.all(sb[b, :, :want] >= 0) and np.all(sb[b, :, :want] <= 1.0 + 1e-5)
+            assert np.all(pos[b, :, :want] < seen[b]) and np.all(pos[b, :, 0] >= 0)
+    return pos, cnt
+
+
+def test_cfg2_full_layer_decode_sampled_units(gpu):
+    """Configuration 2, one full layer: 8 sequences x 32 heads, budget 1024, past one full idx cycle of decode."""
+    import torch
+    from oracle import Oracle
+
+    w = W.CONFIGS["cfg2"]
+    kv = gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, 0)
+    gen = torch.Generator(device="cuda"); gen.manual_seed(w.seed)
+    out_ch = W.outlier_channels(w.head_dim, w.n_outliers)
+    sampled = [(0, 0), (3, 17), (7, 31)]
+    orcs = [Oracle(w.budget, 1, 1, w.head_dim, 1) for _ in sampled]
+    steps = w.budget + 1024 + 60
+    flips = near = 0
+    max_err = 0.0
+    for t in range(steps):
+        q = _draw(torch, gen, (w.batch, w.n_heads, w.head_dim))
+        k = _draw(torch, gen, (w.batch, w.n_kv_heads, w.head_dim), scale_last=out_ch)
+        v = _draw(torch, gen, (w.batch, w.n_kv_heads, w.head_dim))
+        out = kv.decode_step(q, k, v)
+        pos, cnt = kv.retained_positions()
+        for (b, h), orc in zip(sampled, orcs):
+            qo = q[b, h].float().cpu().numpy()[None, None]
+            ko = k[b, h].float().cpu().numpy()[None, None]
+            vo = v[b, h].float().cpu().numpy()[None, None]
+            ref = orc.decode_attend(qo, ko, vo)
+            hp = pos[b, h].cpu().numpy()[None, None]; hc = cnt[b, h].cpu().numpy()[None, None]
+            nt, fl = orc.evict(hp, hc, 1e-4)
+            near += nt; flips += fl
+            err = float(np.abs(out[b, h].float().cpu().numpy() - ref[0, 0]).max())
+            max_err = max(max_err, err)
+            assert err <= 2e-2, (t, b, h, err)
+            assert np.array_equal(orc.retained_positions()[0][0, 0], hp[0, 0]), (t, b, h)
+        if t % 97 == 0 or t == steps - 1:
+            sb = kv.scores().cpu().numpy()
+            for (b, h), orc in zip(sampled, orcs):
+                so = orc.scores()[0, 0]
+                assert np.all(np.abs(sb[b, h] - so) <= 1e-3 * np.abs(so) + 1e-12), (t, b, h)
+    _check_invariants(kv, [steps] * w.batch)
+    st = kv.stats()
+    assert st["device_error"] == 0 and st["evictions"] == w.batch * (steps - w.budget)
+    print("cfg2 full layer: max out err %.3g, near-ties %d, flips %d" % (max_err, near, flips))
+
+
+def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6):
+    import torch
+
+    B, Hq, Hkv, d, m, c = w.batch, w.n_heads, w.n_kv_heads, w.head_dim, w.chunk, w.budget
+    g = Hq // Hkv
+    kv = gpu.TreeKV(c, Hq, Hkv, d, w.dtype, B, m)
+    gen = torch.Generator(device="cuda"); gen.manual_seed(w.seed)
+    rs = np.random.default_rng(w.seed)
+    seq_scale = torch.from_numpy(W.seq_key_scales(w)).cuda() if w.key_scale else None
+    sampled = [(0, 0), (B - 1, Hkv - 1), (B // 2, Hkv // 2)]
+    hist_k = {u: np.zeros((0, d)) for u in sampled}   # full key / value streams of the sampled units (fp64)
+    hist_v = {u: np.zeros((0, d)) for u in sampled}
+    seen = [0] * B
+    lens_total = list(lens_total)
+    n_calls = (max(lens_total) + m - 1) // m
+    max_err = 0.0
+    for call in range(n_calls):
+        lens = [max(0, min(m, L - call * m)) for L in lens_total]
+        q = _draw(torch, gen, (B, m, Hq, d))
+        k = _draw(torch, gen, (B, m, Hkv, d), seq_scale=seq_scale)
+        v = _draw(torch, gen, (B, m, Hkv, d))
+        pos_before, cnt_before = kv.retained_positions()
+        pos_before = pos_before.cpu().numpy(); cnt_before = cnt_before.cpu().numpy()
+        out = kv.prefill_chunk(q, k, v, chunk_lens=lens)
+        for (b, kh) in sampled:
+            mb = lens[b]
+            if mb == 0:
+                continue
+            kc = k[b, :mb, kh].float().cpu().numpy().astype(np.float64)
+            vc = v[b, :mb, kh].float().cpu().numpy().astype(np.float64)
+            Kall = np.concatenate([hist_k[(b, kh)], kc]); Vall = np.concatenate([hist_v[(b, kh)], vc])
+            hist_k[(b, kh)], hist_v[(b, kh)] = Kall, Vall
+            keep = pos_before[b, kh, : cnt_before[b, kh]]
+            rows = sorted(set([0, mb - 1] + [int(x) for x in rs.integers(0, mb, n_sample_rows)]))
+            for t in rows:
+                vis = np.concatenate([keep, np.arange(seen[b], seen[b] + t + 1)])
+                for hh in (0, g - 1):
+                    h = kh * g + hh
+                    ref = _softmax_rows(q[b, t, h].float().cpu().numpy().astype(np.float64), Kall[vis], Vall[vis])
+                    err = float(np.abs(out[b, t, h].float().cpu().numpy() - ref).max())
+                    max_err = max(max_err, err)
+                    assert err <= 2e-2, (call, b, t, h, err)
+        seen = [s + l for s, l in zip(seen, lens)]
+        _check_invariants(kv, seen)
+    assert [kv.tokens_seen(b) for b in range(B)] == seen
+    # batched decode steps at ragged stream positions: sampled rows against brute force over the retained set
+    for step in range(decode_steps):
+        q = _draw(torch, gen, (B, Hq, d))
+        k = _draw(torch, gen, (B, Hkv, d), seq_scale=seq_scale)
+        v = _draw(torch, gen, (B, Hkv, d))
+        pos_before, cnt_before = kv.retained_positions()
+        pos_before = pos_before.cpu().numpy(); cnt_before = cnt_before.cpu().numpy()
+        out = kv.decode_step(q, k, v)
+        for (b, kh) in sampled:
+            hist_k[(b, kh)] = np.concatenate([hist_k[(b, kh)], k[b, kh].float().cpu().numpy().astype(np.float64)[None]])
+            hist_v[(b, kh)] = np.concatenate([hist_v[(b, kh)], v[b, kh].float().cpu().numpy().astype(np.float64)[None]])
+            vis = np.concatenate([pos_before[b, kh, : cnt_before[b, kh]], [seen[b]]])
+            for hh in (0, g - 1):
+                h = kh * g + hh
+                ref = _softmax_rows(q[b, h].float().cpu().numpy().astype(np.float64), hist_k[(b, kh)][vis], hist_v[(b, kh)][vis])
+                err = float(np.abs(out[b, h].float().cpu().numpy() - ref).max())
+                max_err = max(max_err, err)
+                assert err <= 2e-2, (step, b, h, err)
+        seen = [s + 1 for s in seen]
+    _check_invariants(kv, seen)
+    assert kv.stats()["device_error"] == 0
+    return max_err
+
+
+def test_cfg4_full_layer_prefill_then_decode(gpu):
+    """Configuration 4, one full layer: 32 sequences, 32 query / 8 KV heads, budget 2048, 4096-token prefill in
+    chunks of 1024 (8192 CTAs of the tensor-core kernel per chunk), then decode steps."""
+    w = W.CONFIGS["cfg4"]
+    err = _prefill_fullsize(gpu, w, [4096] * w.batch, decode_steps=40)
+    print("cfg4 full layer: max sampled out err %.3g" % err)
+
+
+def test_cfg5_full_layer_ragged_prefill(gpu):
+    """Configuration 5's per-layer shape (4 sequences, GQA 4:1, budget 4096, chunks of 1024) with ragged lengths that
+    end in different, partial chunks; lengths are cut to about 2.5 budgets to keep the run short."""
+    w = W.CONFIGS["cfg5"]
+    lens = [2 * 4096 + 1024 + 517, 2 * 4096 + 100, 10 * 1024, 2 * 4096 + 1]
+    err = _prefill_fullsize(gpu, w, lens, decode_steps=24)
+    print("cfg5 full layer: max sampled out err %.3g" % err)
