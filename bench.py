@@ -125,6 +125,58 @@ def physical_gpu_index(local_rank):
     return local_rank
 
 
+def whole_job_rate(world, units_per_rank, ms):
+    """Units per second of all replicas together: every rank processed `units_per_rank` within `ms` (the max)."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
+class Replicas:
+    """The N > 1 plumbing: every rank runs an independent replica (the path has no exchange step), so the only
+    collectives are the barrier around a timed region and the max of the ranks' device times.  `backend` "nccl"
+    needs `device`; "gloo" runs the same logic on CPU ranks."""
+
+    def __init__(self, backend="nccl", device=None):
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.device = device
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+
+            if backend == "nccl":
+                dist.init_process_group("nccl", device_id=device)
+            else:
+                dist.init_process_group(backend)
+            self.dist = dist
+
+    def barrier(self):
+        """All ranks have reached this point and this rank's device is idle."""
+        if self.dist is not None:
+            self.dist.barrier()
+        if self.device is not None:
+            import torch
+
+            torch.cuda.synchronize(self.device)
+
+    def max_over_ranks(self, ms):
+        if self.dist is None:
+            return float(ms)
+        import torch
+
+        t = torch.tensor([ms], dtype=torch.float64, device=self.device if self.device is not None else "cpu")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def whole_job_rate(self, units_per_rank, ms):
+        return whole_job_rate(self.world, units_per_rank, ms)
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
+            self.dist = None
+
+
 # ------------------------------------------------------------------------------------------------------
 # oracle timing (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------------
@@ -165,8 +217,6 @@ def run_reference(args, w):
     build_oracle()
     seqs = min(2, w.batch)
     steps = max(1, args.steps)
-    for _ in range(1):
-        pass
     # warm-up steps are part of the cache fill; each "step" of this arm is one oracle decode step of the sample
     val, cores, desc = time_oracle_decode(w, seqs, min(steps, 400))
     line = {
@@ -207,38 +257,23 @@ def main():
         return
 
     import torch
-    import torch.distributed as dist
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    rep = Replicas("nccl", dev)
+    rank, world = rep.rank, rep.world
 
     from paper_2501_04987_b200 import _build
 
     if rank == 0:
         _build.build()
-    if world > 1:
-        dist.barrier()
+    rep.barrier()
     from paper_2501_04987_b200 import binding
 
     peaks = measured_peaks()
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    barrier, max_over_ranks = rep.barrier, rep.max_over_ranks
 
     # ------------------------------------------------------------------ decode leg (headline) + e2e
     dec = run_decode_leg(torch, binding, w, args.steps, max(3, args.warmup), args.e2e_steps, args.decode_split, dev, world,
@@ -288,8 +323,7 @@ def main():
             "cpu_baseline": cpu_baseline, "prefill": prefill, "decode_alt": decode_alt, "prefill_alt": prefill_alt,
         }
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    rep.close()
 
 
 def run_decode_leg(torch, binding, w, steps, warmup, e2e_steps, decode_split, dev, world, rank, local_rank, barrier,
@@ -339,7 +373,7 @@ def run_decode_leg(torch, binding, w, steps, warmup, e2e_steps, decode_split, de
     ms_total = max_over_ranks(ev0.elapsed_time(ev1))
     launches = sum(c.stats()["kernel_launches"] for c in ctxs) - launches0
     ms_per_step = ms_total / steps
-    steps_per_s = world * 1000.0 / ms_per_step
+    steps_per_s = whole_job_rate(world, steps, ms_total)
 
     units = w.batch * w.n_kv_heads
     bytes_per_launch = units * decode_bytes_per_unit(w.budget, w.head_dim, e, g)
@@ -376,7 +410,7 @@ def run_decode_leg(torch, binding, w, steps, warmup, e2e_steps, decode_split, de
         ev1.record()
         barrier()
         e2e_ms = max_over_ranks(ev0.elapsed_time(ev1)) / e2e_n
-        e2e = {"value": world * 1000.0 / e2e_ms, "unit": "steps/s", "h2d_bytes_per_step": w.layers * (nb_q + 2 * nb_k),
+        e2e = {"value": whole_job_rate(world, 1, e2e_ms), "unit": "steps/s", "h2d_bytes_per_step": w.layers * (nb_q + 2 * nb_k),
                "d2h_bytes_per_step": w.layers * nb_q, "steps": e2e_n, "ms_per_step": e2e_ms}
     del ctxs, ins, outs
     torch.cuda.empty_cache()
@@ -424,7 +458,7 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, world, rank, barrier, max
     barrier()
     ms = max_over_ranks(ev0.elapsed_time(ev1))
     launches = sum(x.stats()["kernel_launches"] for x in ctxs) - launches0
-    tok_s = world * n_chunks * m * pw.batch / (ms * 1e-3)
+    tok_s = whole_job_rate(world, n_chunks * m * pw.batch, ms)
     flops_chunk = pw.layers * pw.batch * pw.n_heads * prefill_flops_per_head_chunk(m, c, pw.head_dim)
     achieved = flops_chunk * n_chunks / (ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
