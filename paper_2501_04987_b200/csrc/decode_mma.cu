@@ -12,6 +12,8 @@
 // of the cluster and its partial output to CTA 0 with remote shared-memory stores, so that after one cluster
 // barrier each CTA can write the exact normalised probabilities' group mean into S and CTA 0 can write the
 // output.  CTA 0 then plays Algorithm 1's eviction branch.
+#include <algorithm>
+
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -80,7 +82,11 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     const int rank = (int)cluster.block_rank();
     const int nsplit = (int)cluster.num_blocks();
     const int kh = blockIdx.y, b = blockIdx.z;
+    // Programmatic dependent launch: the next kernel in the stream may be scheduled while this one runs (it does
+    // the same), and nothing below the wait is read before the previous kernel's writes are complete and visible.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (!active.test(b)) return;  // the whole cluster shares b
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int unit = b * cv.Hkv + kh;
     const int N = cv.n_seen[unit];
@@ -359,7 +365,9 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         }
     }
 
-    cluster.sync();  // (A) every CTA's statistics (and, in CTA 0, every partial output) have arrived
+    // a cluster of one needs no cluster-scope release of its global stores: a block barrier orders shared memory
+    auto unit_barrier = [&]() { if (nsplit == 1) __syncthreads(); else cluster.sync(); };
+    unit_barrier();  // (A) every CTA's statistics (and, in CTA 0, every partial output) have arrived
 
     float Mg[G], invL[G];
 #pragma unroll
@@ -382,19 +390,29 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         }
     }
     // ---- normalised probabilities; score update (Algorithm 1: S <- (S u {0}) + a, group mean)
-    for (int j = tid; j < nrows; j += NT) {
+    //      (a masked or padded logit is -inf and 2^-inf = 0, so exp2f needs no guard here: Mg is finite)
+    const int ncached = nrows - (owns_new ? 1 : 0);
+#pragma unroll 4
+    for (int j = tid; j < ncached; j += NT) {
         float ps = 0.f;
 #pragma unroll
-        for (int h = 0; h < G; ++h) ps += exp2_diff(sl[h * rows_cap + j], Mg[h]) * invL[h];
-        const int lam = lo + j;
-        const int ph = phys_row(lam, i_cyc);
-        const float s_new = ((lam == n - 1) ? 0.f : s_old[j]) + ps * (1.0f / G);
+        for (int h = 0; h < G; ++h) ps += exp2f(sl[h * rows_cap + j] - Mg[h]) * invL[h];
+        const int ph = phys_row(lo + j, i_cyc);
+        const float s_new = s_old[j] + ps * (1.0f / G);
         Sc[ph] = s_new;
-        if (lam == n - 1) Pc[ph] = N;
         if (nsplit == 1 && (ph >> 1) == i_cyc) pair_s[ph & 1] = s_new;  // the scope's scores stay on chip
     }
+    if (owns_new && tid == NT - 1) {  // the appended token starts from S = 0
+        float ps = 0.f;
+#pragma unroll
+        for (int h = 0; h < G; ++h) ps += exp2f(sl[h * rows_cap + ncached] - Mg[h]) * invL[h];
+        const float s_new = ps * (1.0f / G);
+        Sc[new_row] = s_new;
+        Pc[new_row] = N;
+        if (nsplit == 1 && (new_row >> 1) == i_cyc) pair_s[new_row & 1] = s_new;
+    }
 
-    cluster.sync();  // (B) the appended row and every S update of the unit are complete
+    unit_barrier();  // (B) the appended row and every S update of the unit are complete
 
     if (rank == 0 && warp == 0 && will_evict) {
         // ---- Algorithm 1, "length > c" branch: scope {idx, idx+1} = physical rows (2i, 2i+1)
@@ -435,11 +453,23 @@ static cudaError_t launch_decode_mma_t(const CacheView& cv, const void* q, const
                                        const ActiveMask& active, int split, cudaStream_t stream) {
     auto kern = decode_mma_kernel<D, G, kMmaWarps, kMmaStages>;
     const int rows_cap = mma_rows_cap(cv.c, split);
-    const size_t smem = decode_mma_smem_bytes(G, D, cv.c, split);
+    size_t smem = decode_mma_smem_bytes(G, D, cv.c, split);
     static size_t smem_set[64] = {};  // per device: the opt-in limit only ever needs raising
+    static int sm_count[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     dev &= 63;
+    if (sm_count[dev] == 0) cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+    // When the whole grid fits at w = ceil(CTAs / SMs) thread blocks per SM, ask for just enough shared memory that
+    // no SM can take more than w: the block scheduler otherwise packs some SMs to their limit and leaves others idle,
+    // and the streaming rate of an SM does not grow in proportion to the blocks it hosts.
+    {
+        constexpr size_t kSmemPerSm = 227 * 1024, kReserved = 1024;  // per-block reservation of the runtime
+        const long ncta = (long)split * cv.Hkv * cv.B;
+        const long w = (ncta + sm_count[dev] - 1) / std::max(sm_count[dev], 1);
+        if (w >= 1 && (size_t)(w + 1) * (smem + kReserved) <= kSmemPerSm)
+            smem = std::max(smem, kSmemPerSm / (size_t)(w + 1) + 1 - kReserved + 1024);
+    }
     if (smem > smem_set[dev]) {
         const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -450,13 +480,15 @@ static cudaError_t launch_decode_mma_t(const CacheView& cv, const void* q, const
     cfg.blockDim = dim3(kMmaWarps * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = split;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the kernel orders itself with griddepcontrol.wait
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     using T = __nv_bfloat16;
     return cudaLaunchKernelEx(&cfg, kern, cv, reinterpret_cast<const T*>(q), reinterpret_cast<const T*>(k),
                               reinterpret_cast<const T*>(v), reinterpret_cast<T*>(out), active, rows_cap);
