@@ -125,9 +125,13 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
                                    void* stream);
 
 /*
- * The same two calls with HOST tensors (pageable or pinned): inputs are copied to staging buffers inside the
- * workspace, the step runs, and the output is copied back, all enqueued on `stream`.  host_out is valid once
- * the stream has been synchronised.  Shapes as above.
+ * The same two calls with HOST tensors (pageable or page-locked), all enqueued on `stream`: host_out is valid,
+ * and the host inputs may be reused, once the stream has been synchronised.  Shapes as above.
+ * treekv_decode_step_host: when all four tensors are page-locked memory the GPU can address (cudaHostAlloc /
+ * cudaHostRegister, 16-byte aligned), the step's kernel reads q, k, v from them and writes the output to them
+ * directly across the bus - one launch, no staging copy; otherwise the inputs are copied to staging buffers
+ * inside the workspace, the step runs, and the output is copied back.
+ * treekv_prefill_chunk_host always stages through the workspace.
  */
 treekv_status treekv_decode_step_host(treekv_ctx* ctx, const void* host_q, const void* host_k, const void* host_v,
                                       void* host_out, const uint8_t* host_active, void* stream);

@@ -215,8 +215,8 @@ class TreeKV:
 
     def close(self):
         h, self._h = getattr(self, "_h", None), None
-        if h:
-            treekv_destroy(h)
+        if h and lib is not None and getattr(lib, "treekv_destroy", None) is not None:   # (names vanish at interpreter exit)
+            lib.treekv_destroy(h)
 
     def __del__(self):
         self.close()

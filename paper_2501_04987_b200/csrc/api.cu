@@ -106,6 +106,15 @@ int pick_decode_split(const treekv_ctx* ctx) {
     return s;
 }
 
+// Device-side alias of a host pointer when the GPU can address it directly (page-locked memory registered with
+// the CUDA runtime, or memory allocated by it), else nullptr.
+void* device_alias(const void* host_ptr) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host_ptr) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (at.type != cudaMemoryTypeHost && at.type != cudaMemoryTypeManaged && at.type != cudaMemoryTypeDevice) return nullptr;
+    return at.devicePointer;
+}
+
 }  // namespace
 
 extern "C" {
@@ -281,6 +290,16 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
 treekv_status treekv_decode_step_host(treekv_ctx* ctx, const void* host_q, const void* host_k, const void* host_v,
                                       void* host_out, const uint8_t* host_active, void* stream) {
     if (!ctx || !host_q || !host_k || !host_v || !host_out) return TREEKV_ERR_INVALID_ARG;
+    // Page-locked host tensors are read and written by the kernel itself across the bus (q, k, v are each read
+    // early in the kernel, under the cache stream; the output is written once): no copy, no staging, one launch.
+    {
+        void* dq = device_alias(host_q);
+        void* dk = dq ? device_alias(host_k) : nullptr;
+        void* dv = dk ? device_alias(host_v) : nullptr;
+        void* dout = dv ? device_alias(host_out) : nullptr;
+        if (dout && aligned16(dq) && aligned16(dk) && aligned16(dv) && aligned16(dout))
+            return treekv_decode_step(ctx, dq, dk, dv, dout, host_active, stream);
+    }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t qb = (size_t)ctx->cv.B * ctx->cv.Hq * ctx->cv.d * ctx->elem;
     const size_t kb = (size_t)ctx->cv.B * ctx->cv.Hkv * ctx->cv.d * ctx->elem;

@@ -12,7 +12,7 @@ struct treekv_ctx {
     int max_chunk;
     int G;
     size_t elem;
-    // staging for the *_host entry points
+    // staging for the *_host entry points (sized for a chunk)
     void *st_q, *st_k, *st_v, *st_out;
     // options
     int opt_decode_split;

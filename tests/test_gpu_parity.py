@@ -262,7 +262,9 @@ def test_bitwise_reproducible(gpu):
         assert torch.equal(x, y)
 
 
-def test_host_entry_points_match_device_entry_points(gpu):
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_entry_points_match_device_entry_points(gpu, pinned):
+    """Page-locked host tensors are read by the decode kernel directly; pageable ones go through staging copies."""
     import torch
 
     w = W.parity_slice(W.CONFIGS["cfg4"], layers=1, batch=2, n_heads=8, n_kv_heads=2, budget=64, chunk=32)
@@ -278,13 +280,54 @@ def test_host_entry_points_match_device_entry_points(gpu):
         assert torch.equal(od.cpu(), oh)
     q, k, v = W.tokens(w, 0, 128, 128 + 40)
     for s in range(40):
-        h = [torch.from_numpy(x[s]).bfloat16().pin_memory() for x in (q, k, v)]
-        oh = torch.empty_like(h[0]).pin_memory()
+        h = [torch.from_numpy(x[s]).bfloat16() for x in (q, k, v)]
+        oh = torch.empty_like(h[0])
+        if pinned:
+            h = [x.pin_memory() for x in h]
+            oh = oh.pin_memory()
         b.decode_step_host(h[0], h[1], h[2], oh)
         od = a.decode_step(*[x.cuda() for x in h])
         torch.cuda.synchronize()
         assert torch.equal(od.cpu(), oh)
     assert torch.equal(a.retained_positions()[0], b.retained_positions()[0])
+
+
+def test_host_decode_pipeline_without_intermediate_syncs(gpu):
+    """Many host-tensor decode steps over three contexts (layers), enqueued back to back on a side stream with no
+    synchronisation in between and mixed with device-tensor calls: every output and the final caches must equal
+    those of the device entry point."""
+    import torch
+
+    w = W.parity_slice(W.CONFIGS["cfg2"], layers=3, batch=2, n_heads=4, n_kv_heads=4, budget=48, chunk=0)
+    host = [gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, 0) for _ in range(w.layers)]
+    dev = [gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, 0) for _ in range(w.layers)]
+    steps = 150
+    ins = []
+    for layer in range(w.layers):
+        q, k, v = W.tokens(w, layer, 0, steps)
+        ins.append([torch.from_numpy(x).bfloat16().pin_memory() for x in (q, k, v)])
+    outs_h = [torch.zeros((steps, w.batch, w.n_heads, w.head_dim), dtype=torch.bfloat16).pin_memory() for _ in range(w.layers)]
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        for s in range(steps):
+            for layer in range(w.layers):
+                q, k, v = ins[layer]
+                if s % 7 == 3 and layer == 1:   # a device-tensor call in the middle of the pipeline, same stream
+                    o = host[layer].decode_step(q[s].cuda(non_blocking=True), k[s].cuda(non_blocking=True),
+                                                v[s].cuda(non_blocking=True))
+                    outs_h[layer][s].copy_(o, non_blocking=True)
+                else:
+                    host[layer].decode_step_host(q[s], k[s], v[s], outs_h[layer][s])
+    side.synchronize()
+    for layer in range(w.layers):
+        q, k, v = ins[layer]
+        for s in range(steps):
+            od = dev[layer].decode_step(q[s].cuda(), k[s].cuda(), v[s].cuda())
+            assert torch.equal(od.cpu(), outs_h[layer][s]), (layer, s)
+        assert torch.equal(dev[layer].retained_positions()[0], host[layer].retained_positions()[0])
+        assert torch.equal(dev[layer].scores(), host[layer].scores())
+        assert host[layer].stats()["device_error"] == 0
 
 
 def test_argument_and_state_errors(gpu):
