@@ -119,18 +119,26 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     unsigned char* pair_kv = reinterpret_cast<unsigned char*>(                   // [4][ROWB] K,V of the scope's two rows
         (reinterpret_cast<uintptr_t>(s_old + rows_cap) + 15) & ~uintptr_t(15));
     float* pair_s = reinterpret_cast<float*>(pair_kv + 4 * ROWB);          // [2] updated S of rows 2i, 2i+1 (split == 1)
+    unsigned char* tok = pair_kv + 4 * ROWB + 16;                          // [G+2][ROWB] this step's q heads, k, v
     float* o_warp = reinterpret_cast<float*>(ring);                        // [NW][G][D], aliases the ring after the loop
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const float scale = kLog2e * rsqrtf((float)D);
 
-    // ---- append (Algorithm 1: K <- K u {k}, V <- V u {v}); the step itself reads the new token from k_in / v_in
-    if (owns_new && warp == NW - 1) {
-        for (int e = lane; e < CHUNKS; e += 32) {
-            reinterpret_cast<uint4*>(Kc + (size_t)new_row * D)[e] = ld_plain(reinterpret_cast<const uint4*>(k_new) + e);
-            reinterpret_cast<uint4*>(Vc + (size_t)new_row * D)[e] = ld_plain(reinterpret_cast<const uint4*>(v_new) + e);
+    // ---- this step's inputs go to shared memory once per CTA (warp 0, one commit group of their own): the q rows of
+    //      the group's heads, and in the CTAs that use them the new key and value rows.  Everything that needs them
+    //      reads the copy, so q, k, v are fetched once, early, whether they live in HBM or in page-locked host memory.
+    const bool needs_kv = owns_new || rank == 0;
+    if (warp == 0) {
+        const T* qrow = q + ((size_t)b * cv.Hq + kh * G) * D;
+        for (int e = lane; e < (G + 2) * CPR; e += 32) {
+            const int r = e / CPR, cidx = e % CPR;
+            if (r >= G && !needs_kv) continue;
+            const T* srow = r < G ? qrow + (size_t)r * D : (r == G ? k_new : v_new);
+            cp_async_16(smem_u32(tok + r * ROWB + cidx * 16), reinterpret_cast<const unsigned char*>(srow) + cidx * 16, true);
         }
+        cp_async_commit();
     }
 
     const uint32_t ring_w = smem_u32(ring) + warp * NS * STAGE;
@@ -177,7 +185,6 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     //      the eviction scope (rows 2i and 2i+1; the new token's row comes from k_in / v_in)
     const bool will_evict = (N + 1 > cv.c);
     static_assert(NT % D == 0, "a thread always combines the same channel");
-    const float vnew_r = owns_new ? __bfloat162float(v_new[tid % D]) : 0.f;  // this thread's channel of the new value row
     int pos_l = 0, pos_r = 0;  // stream positions of the scope's two tokens (used by lane 0 of warp 0 in CTA 0)
     if (rank == 0 && will_evict && tid == 0) {
         pos_l = Pc[2 * i_cyc];
@@ -192,15 +199,38 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         for (int e = lane; e < 4 * CPR; e += 32) {
             const int which = e / CPR, cidx = e % CPR;   // 0: K left, 1: K right, 2: V left, 3: V right
             const int prow = 2 * i_cyc + (which & 1);
-            const T* srcrow = (prow == new_row) ? ((which < 2) ? k_new : v_new)
-                                                : ((which < 2) ? Kc : Vc) + (size_t)prow * D;
+            if (prow == new_row) continue;  // the appended row is taken from the staged inputs below
+            const T* srcrow = ((which < 2) ? Kc : Vc) + (size_t)prow * D;
             cp_async_16(smem_u32(pair_kv + which * ROWB + cidx * 16), reinterpret_cast<const unsigned char*>(srcrow) + cidx * 16, true);
         }
     }
 #pragma unroll
     for (int s = 0; s < NS; ++s) issue(warp + s * NW, s);
 
-    // ---- the new token's logit q.k_new (warp 0 of the owning CTA), computed while the first tiles are in flight
+    if (warp == 0) cp_async_wait<NS>();  // the staged inputs have landed (the NS tile groups may still be in flight)
+    __syncthreads();
+    const T* tq = reinterpret_cast<const T*>(tok);
+    const T* tk = reinterpret_cast<const T*>(tok + G * ROWB);
+    const T* tv = reinterpret_cast<const T*>(tok + (G + 1) * ROWB);
+    const float vnew_r = owns_new ? __bfloat162float(tv[tid % D]) : 0.f;  // this thread's channel of the new value row
+
+    // ---- append (Algorithm 1: K <- K u {k}, V <- V u {v}); the step itself uses the staged copy of the new token
+    if (warp == NW - 1) {
+        if (owns_new) {
+            for (int e = lane; e < CHUNKS; e += 32) {
+                reinterpret_cast<uint4*>(Kc + (size_t)new_row * D)[e] = reinterpret_cast<const uint4*>(tk)[e];
+                reinterpret_cast<uint4*>(Vc + (size_t)new_row * D)[e] = reinterpret_cast<const uint4*>(tv)[e];
+            }
+        }
+        if (rank == 0 && will_evict && new_row == 2 * i_cyc + 1) {  // the scope's right row is the appended one
+            for (int e = lane; e < CHUNKS; e += 32) {
+                reinterpret_cast<uint4*>(pair_kv + 1 * ROWB)[e] = reinterpret_cast<const uint4*>(tk)[e];
+                reinterpret_cast<uint4*>(pair_kv + 3 * ROWB)[e] = reinterpret_cast<const uint4*>(tv)[e];
+            }
+        }
+    }
+
+    // ---- the new token's logit q.k_new (warp 0 of the owning CTA)
     if (warp == 0) {
         float sn[G];
 #pragma unroll
@@ -209,8 +239,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
 #pragma unroll
             for (int h = 0; h < G; ++h) {
                 float a = 0.f;
-                for (int e = lane; e < D; e += 32)
-                    a += __bfloat162float(q[((size_t)b * cv.Hq + kh * G + h) * D + e]) * __bfloat162float(k_new[e]);
+                for (int e = lane; e < D; e += 32) a += __bfloat162float(tq[h * D + e]) * __bfloat162float(tk[e]);
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
                 sn[h] = a * scale;
@@ -231,7 +260,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     for (int kk = 0; kk < D / 16; ++kk) {
         qa[kk][0] = 0u; qa[kk][1] = 0u;
         if (g < G) {
-            const T* qh = q + ((size_t)b * cv.Hq + kh * G + g) * D + 16 * kk + 2 * t;
+            const T* qh = tq + g * D + 16 * kk + 2 * t;
             qa[kk][0] = *reinterpret_cast<const uint32_t*>(qh);
             qa[kk][1] = *reinterpret_cast<const uint32_t*>(qh + 8);
         }
@@ -445,7 +474,8 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
 size_t decode_mma_smem_bytes(int G, int D, int c, int split) {
     const size_t ring = (size_t)kMmaWarps * kMmaStages * 2 * kBlk * D * 2;
     return ring + sizeof(float) * ((size_t)G * mma_rows_cap(c, split) + (kMmaWarps + 1) * 2 * G + kMaxSplit * 2 * G +
-                                   (size_t)split * G * D + (size_t)mma_rows_cap(c, split) + 2) + 4 * (size_t)D * 2 + 16;
+                                   (size_t)split * G * D + (size_t)mma_rows_cap(c, split) + 2) + 4 * (size_t)D * 2 + 16 +
+           16 + (size_t)(G + 2) * D * 2;
 }
 
 template <int D, int G>
