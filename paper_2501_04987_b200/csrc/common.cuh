@@ -152,6 +152,32 @@ struct PrefillScratch {
 };
 constexpr int kQTileRows = 128;  // query rows (token x head-in-group) per prefill tile
 
+// ---- programmatic dependent launch.  A kernel launched with launch_pdl may be scheduled while the kernel before
+// it in the stream is still running; it calls pdl_wait() before it reads or writes anything of the cache or the
+// scratch, which returns once every earlier kernel in the stream has completed and its writes are visible, and
+// pdl_trigger() (first statement) lets the kernel after it be scheduled in turn.  Launch latency and block
+// scheduling thereby overlap the predecessor's tail.  Every block waits, also one that then finds nothing to
+// do, so that the order of the chain stays transitive.  Launched without the attribute, both are no-ops.
+#ifdef __CUDACC__
+__device__ inline void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ inline void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+#endif
+
 // ---- launchers implemented in the .cu files (each enqueues on `stream` and returns the launch status)
 size_t decode_smem_bytes(int G, int D, int c, int split);
 cudaError_t launch_decode(const CacheView& cv, treekv_dtype dt, const void* q, const void* k, const void* v, void* out,

@@ -84,9 +84,9 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     const int kh = blockIdx.y, b = blockIdx.z;
     // Programmatic dependent launch: the next kernel in the stream may be scheduled while this one runs (it does
     // the same), and nothing below the wait is read before the previous kernel's writes are complete and visible.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pdl_trigger();
+    pdl_wait();  // every block waits, also one of an inactive sequence
     if (!active.test(b)) return;  // the whole cluster shares b
-    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int unit = b * cv.Hkv + kh;
     const int N = cv.n_seen[unit];

@@ -394,8 +394,15 @@ static cudaError_t launch_prefill_tc_t(const CacheView& cv, const PrefillScratch
                                        int chunk_stride, int max_m, cudaStream_t stream) {
     auto kern = prefill_tc_kernel<G>;
     const size_t smem = prefill_tc_smem_bytes();
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    static bool smem_set[64] = {};  // per device: the opt-in is needed once
+    int dev = 0;
+    cudaGetDevice(&dev);
+    dev &= 63;
+    if (!smem_set[dev]) {
+        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        smem_set[dev] = true;
+    }
     dim3 grid((max_m * G + kQTileRows - 1) / kQTileRows, cv.B * cv.Hkv);
     kern<<<grid, kTcThreads, smem, stream>>>(tmQ, tmK, tmV, cv, ps, reinterpret_cast<__nv_bfloat16*>(out), lens, chunk_stride);
     return cudaGetLastError();

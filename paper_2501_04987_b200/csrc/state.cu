@@ -59,6 +59,8 @@ cudaError_t launch_scores(const CacheView& cv, float* sbar_out, cudaStream_t str
 template <typename T>
 __global__ void chunk_append_kernel(CacheView cv, const T* __restrict__ k, const T* __restrict__ v, ChunkLens lens,
                                     int chunk_stride) {
+    pdl_trigger();
+    pdl_wait();
     const int unit = blockIdx.y;
     const int b = unit / cv.Hkv, kh = unit % cv.Hkv;
     const int m = lens.m[b];
@@ -83,17 +85,17 @@ cudaError_t launch_chunk_append(const CacheView& cv, treekv_dtype dt, const void
                                 int chunk_stride, int max_m, cudaStream_t stream) {
     dim3 grid((max_m + 7) / 8, cv.B * cv.Hkv);
     if (dt == TREEKV_F32)
-        chunk_append_kernel<float><<<grid, 256, 0, stream>>>(cv, (const float*)k, (const float*)v, lens, chunk_stride);
-    else
-        chunk_append_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(cv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
-                                                                      lens, chunk_stride);
-    return cudaGetLastError();
+        return launch_pdl(chunk_append_kernel<float>, grid, dim3(256), 0, stream, cv, (const float*)k, (const float*)v, lens,
+                          chunk_stride);
+    return launch_pdl(chunk_append_kernel<__nv_bfloat16>, grid, dim3(256), 0, stream, cv, (const __nv_bfloat16*)k,
+                      (const __nv_bfloat16*)v, lens, chunk_stride);
 }
 
 // ---------------------------------------------------------------------------------------------------------
 // Chunk score update: S[row(lam)] += (sum over query tiles of the partial column sums) / G, tiles added in
 // a fixed order so the result does not depend on scheduling.
 __global__ void chunk_scores_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
+    pdl_trigger();  // launched in plain stream order itself; the eviction kernel behind it may be scheduled early
     const int unit = blockIdx.y;
     const int b = unit / cv.Hkv;
     const int m = lens.m[b];
@@ -126,6 +128,8 @@ cudaError_t launch_chunk_scores(const CacheView& cv, const PrefillScratch& ps, c
 // move goes through staging rows: gather (decide + copy out), then scatter (copy in) as a second launch.
 template <typename T>
 __global__ void chunk_evict_gather_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int seg) {
+    pdl_trigger();
+    pdl_wait();
     const int unit = blockIdx.y;
     const int b = unit / cv.Hkv;
     const int m = lens.m[b];
@@ -166,6 +170,8 @@ __global__ void chunk_evict_gather_kernel(CacheView cv, PrefillScratch ps, Chunk
 
 template <typename T>
 __global__ void chunk_evict_scatter_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int seg) {
+    pdl_trigger();
+    pdl_wait();
     const int unit = blockIdx.y;
     const int b = unit / cv.Hkv;
     const int m = lens.m[b];
@@ -193,24 +199,27 @@ cudaError_t launch_chunk_evict(const CacheView& cv, treekv_dtype dt, const Prefi
                                int seg, int max_items, cudaStream_t stream) {
     if (max_items <= 0) return cudaSuccess;
     dim3 grid((max_items + 7) / 8, cv.B * cv.Hkv);
+    cudaError_t e;
     if (dt == TREEKV_F32) {
-        chunk_evict_gather_kernel<float><<<grid, 256, 0, stream>>>(cv, ps, lens, seg);
-        chunk_evict_scatter_kernel<float><<<grid, 256, 0, stream>>>(cv, ps, lens, seg);
+        e = launch_pdl(chunk_evict_gather_kernel<float>, grid, dim3(256), 0, stream, cv, ps, lens, seg);
+        if (e == cudaSuccess) e = launch_pdl(chunk_evict_scatter_kernel<float>, grid, dim3(256), 0, stream, cv, ps, lens, seg);
     } else {
-        chunk_evict_gather_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(cv, ps, lens, seg);
-        chunk_evict_scatter_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(cv, ps, lens, seg);
+        e = launch_pdl(chunk_evict_gather_kernel<__nv_bfloat16>, grid, dim3(256), 0, stream, cv, ps, lens, seg);
+        if (e == cudaSuccess)
+            e = launch_pdl(chunk_evict_scatter_kernel<__nv_bfloat16>, grid, dim3(256), 0, stream, cv, ps, lens, seg);
     }
-    return cudaGetLastError();
+    return e;
 }
 
 __global__ void chunk_finalize_kernel(CacheView cv, ChunkLens lens) {
+    pdl_trigger();
+    pdl_wait();
     const int unit = blockIdx.x * blockDim.x + threadIdx.x;
     if (unit < cv.B * cv.Hkv) cv.n_seen[unit] += lens.m[unit / cv.Hkv];
 }
 cudaError_t launch_chunk_finalize(const CacheView& cv, const ChunkLens& lens, cudaStream_t stream) {
     const int units = cv.B * cv.Hkv;
-    chunk_finalize_kernel<<<(units + 255) / 256, 256, 0, stream>>>(cv, lens);
-    return cudaGetLastError();
+    return launch_pdl(chunk_finalize_kernel, dim3((units + 255) / 256), dim3(256), 0, stream, cv, lens);
 }
 
 }  // namespace treekv
