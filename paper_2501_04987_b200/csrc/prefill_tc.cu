@@ -16,9 +16,11 @@
 // log-sum-exp", with the probabilities used for the output and for the scores being the same numbers.
 //
 // Warp roles: warp 0 issues TMA, warp 1 issues MMA and owns the tensor-memory allocation, warps 2-9 are two
-// groups of four softmax warps (one tensor-memory lane quarter per warp); group g owns the S buffer, the P^T
-// buffer and the key tiles of parity g, so the two groups alternate tiles and overlap each other's latency.  All waits are bounded mbarrier waits; a wait that gives
-// up sets an error word and the CTA drains to its exit, where tensor memory is released.
+// groups of four softmax warps (one tensor-memory lane quarter per warp); group g takes the key tiles of parity
+// g and owns P^T buffer g, so the two groups alternate tiles and overlap each other's latency.  The S / S^T
+// accumulators are three tensor-memory buffers used round-robin by tile index, so the MMA warp can start a
+// tile's logits while both groups are still reading theirs.  All waits are bounded mbarrier waits; a wait that
+// gives up sets an error word and the CTA drains to its exit, where tensor memory is released.
 #include <type_traits>
 
 #include "common.cuh"
@@ -35,7 +37,8 @@ constexpr int kTcThreads = 320;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kD = 128;
 
-enum Bar { Q_FULL = 0, RING_FULL = 1, RING_EMPTY = 5, S_FULL = 9, S_FREE = 11, P_FULL = 13, P_FREE = 15, O_FULL = 17, N_BARS = 18 };
+constexpr int kSBufs = 3;     // S / S^T accumulators in tensor memory, used round-robin by tile index
+enum Bar { Q_FULL = 0, RING_FULL = 1, RING_EMPTY = 5, S_FULL = 9, S_FREE = 12, P_FULL = 15, P_FREE = 17, O_FULL = 19, N_BARS = 20 };
 
 struct KeyTiles {
     int i;     // cycle position: live rows [0,i) and [2i, ...)
@@ -95,10 +98,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (tid == 0) {
         mbar_init(bar(Q_FULL), 1);
         for (int s = 0; s < kRing; ++s) { mbar_init(bar(RING_FULL + s), 1); mbar_init(bar(RING_EMPTY + s), 1); }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_FREE + s), 4);
-            mbar_init(bar(P_FULL + s), 4); mbar_init(bar(P_FREE + s), 1);
-        }
+        for (int s = 0; s < kSBufs; ++s) { mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_FREE + s), 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar(P_FULL + s), 4); mbar_init(bar(P_FREE + s), 1); }
         mbar_init(bar(O_FULL), 1);
         mbar_fence_init();
     }
@@ -107,7 +108,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    const uint32_t tmS = tmem, tmO = tmem + 256;  // S / S^T double buffer at columns 0 and 128; O^T at 256
+    const uint32_t tmS = tmem, tmO = tmem + 128 * kSBufs;  // S / S^T buffers at columns 0, 128, 256; O^T at 384
 
     bool ok = true;
     if (warp == 0) {
@@ -147,10 +148,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, 1, 1);  // V^T and P^T: MN-major
             ok = mbar_wait(bar(Q_FULL), 0);
             tc_fence_after();
-            int use[2] = {0, 0};  // times each S buffer has been handed to the softmax warps (both passes)
+            int use[kSBufs] = {0, 0, 0};  // times each S buffer has been handed to the softmax warps (both passes)
             // ---- pass A: S = Q K^T
             for (int j = 0; j < NT && ok; ++j) {
-                const int ld = j, slot = ld % kRing, buf = j & 1;
+                const int ld = j, slot = ld % kRing, buf = j % kSBufs;
                 ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), (use[buf] & 1) ^ 1);
                 if (!ok) break;
                 tc_fence_after();
@@ -169,7 +170,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             //      owns buffer j & 1 finds S^T_{j+2} ready when it finishes tile j (its buffer is free as soon as
             //      it has read tile j into registers, long before P_j^T is complete)
             auto issue_st = [&](int j) {
-                const int ld = NT + (j < 3 ? j : 2 * j - 2), slot = ld % kRing, buf = j & 1;  // see the producer's load order
+                const int ld = NT + (j < 3 ? j : 2 * j - 2), slot = ld % kRing, buf = j % kSBufs;  // see the producer's load order
                 ok = mbar_wait(bar(RING_FULL + slot), (ld / kRing) & 1) && mbar_wait(bar(S_FREE + buf), (use[buf] & 1) ^ 1);
                 if (!ok) return;
                 tc_fence_after();
@@ -211,19 +212,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const int row = quarter * 32 + lane;   // pass A: query row; pass B: key of the tile; epilogue: channel
         const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
         const float sc2 = kLog2e * rsqrtf((float)kD);
-        const uint32_t tmSg = tmS + grp * 128 + lane_off;
         float* nlse = lse;                     // [128] minus the log2-domain log-sum-exp of every query row
         // per-group running (max, sum) of pass A, [2][128] each; they borrow the P^T area, which pass A does not use
         float* part_m = reinterpret_cast<float*>(base_ptr + (1 + kRing) * kSlot);
         float* part_l = part_m + 256;
         uint32_t va[32], vb[32];  // two chunks of 32 columns: the next one is in flight while this one is used
-        int use = 0;  // times this group's S buffer has been filled (both passes)
         // ---- pass A: row statistics over this group's tiles
         {
             const int tq = min(t0 + row / G, t1 - 1);  // rows past the chunk repeat the last real row: finite, unused
             float mrun = -INFINITY, lrun = 0.f;
             for (int j = grp; j < NT && ok; j += 2) {
-                if (!mbar_wait(bar(S_FULL + grp), use & 1)) { ok = false; break; }
+                const int buf = j % kSBufs;  // the buffer's fill number in this pass is j / kSBufs
+                const uint32_t tmSg = tmS + buf * 128 + lane_off;
+                if (!mbar_wait(bar(S_FULL + buf), (j / kSBufs) & 1)) { ok = false; break; }
                 tc_fence_after();
                 int lam0, row0, valid;
                 tile_of(kt, j, lam0, row0, valid);
@@ -274,9 +275,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 tmem_ld_wait_for(vb);
                 tc_fence_before();  // last read of this S buffer: hand it back before the arithmetic on it
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(S_FREE + grp));
+                if (lane == 0) mbar_arrive(bar(S_FREE + buf));
                 stats32(vb, 3);
-                ++use;
             }
             part_m[grp * 128 + row] = mrun;
             part_l[grp * 128 + row] = lrun;
@@ -295,7 +295,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         float* part = ps.colsum + ((size_t)unit * ps.QT + qt) * ps.n_max;
         int puse = 0;  // times this group's P^T buffer has been filled
         for (int j = grp; j < NT && ok; j += 2) {
-            if (!mbar_wait(bar(S_FULL + grp), use & 1)) { ok = false; break; }
+            const int buf = j % kSBufs;
+            const uint32_t tmSg = tmS + buf * 128 + lane_off;
+            const int fills_a = (NT + kSBufs - 1 - buf) / kSBufs;  // times pass A filled this buffer
+            if (!mbar_wait(bar(S_FULL + buf), (fills_a + j / kSBufs) & 1)) { ok = false; break; }
             tc_fence_after();
             int lam0, row0, valid;
             tile_of(kt, j, lam0, row0, valid);
@@ -305,8 +308,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const bool full = __all_sync(0xffffffffu, rmin == 0) && rmax == 128;
             float colsum = 0.f;
             unsigned char* prow = base_ptr + (1 + kRing) * kSlot + grp * kSlot + row * 128;
-            auto probs32 = [&](auto full_tag, const uint32_t (&v)[32], int cg) {
-                constexpr bool kFull = decltype(full_tag)::value;  // every (key, query) pair of the warp's rows is visible
+            auto probs32 = [&](auto full_tag, auto first_tag, const uint32_t (&v)[32], int cg) {
+                constexpr bool kFull = decltype(full_tag)::value;    // every (key, query) pair of the warp's rows is visible
+                constexpr bool kFirst = decltype(first_tag)::value;  // first chunk of the tile: the P^T buffer may still be read
+                uint4 pk[4];
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {  // 8 query columns -> one 16-byte chunk of the P^T row
                     float p[8];
@@ -326,38 +331,42 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         }
                     }
                     colsum += ((p[0] + p[1]) + (p[2] + p[3])) + ((p[4] + p[5]) + (p[6] + p[7]));
-                    uint4 pk;
                     __nv_bfloat162 t2;
-                    t2 = __floats2bfloat162_rn(p[0], p[1]); pk.x = *reinterpret_cast<uint32_t*>(&t2);
-                    t2 = __floats2bfloat162_rn(p[2], p[3]); pk.y = *reinterpret_cast<uint32_t*>(&t2);
-                    t2 = __floats2bfloat162_rn(p[4], p[5]); pk.z = *reinterpret_cast<uint32_t*>(&t2);
-                    t2 = __floats2bfloat162_rn(p[6], p[7]); pk.w = *reinterpret_cast<uint32_t*>(&t2);
+                    t2 = __floats2bfloat162_rn(p[0], p[1]); pk[q4].x = *reinterpret_cast<uint32_t*>(&t2);
+                    t2 = __floats2bfloat162_rn(p[2], p[3]); pk[q4].y = *reinterpret_cast<uint32_t*>(&t2);
+                    t2 = __floats2bfloat162_rn(p[4], p[5]); pk[q4].z = *reinterpret_cast<uint32_t*>(&t2);
+                    t2 = __floats2bfloat162_rn(p[6], p[7]); pk[q4].w = *reinterpret_cast<uint32_t*>(&t2);
+                }
+                if constexpr (kFirst) {
+                    // the O^T MMA of this group's previous tile must have read the P^T buffer; it has had the time of
+                    // the first loads and of this chunk's arithmetic to finish
+                    if (!mbar_wait(bar(P_FREE + grp), (puse & 1) ^ 1)) { ok = false; }
+                }
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
                     const int cidx = cg * 4 + q4;  // 16-byte chunk of the 128-query row: half = cidx / 8
-                    *reinterpret_cast<uint4*>(prow + (cidx >> 3) * kHalf + (((cidx & 7) ^ (row & 7)) << 4)) = pk;
+                    *reinterpret_cast<uint4*>(prow + (cidx >> 3) * kHalf + (((cidx & 7) ^ (row & 7)) << 4)) = pk[q4];
                 }
             };
             tmem_ld32(tmSg, va);
             tmem_ld_wait_for(va);
             tmem_ld32(tmSg + 32, vb);
-            // the P^T buffer is only needed now: the O^T MMA of two tiles ago has had the time of the loads to finish
-            if (!mbar_wait(bar(P_FREE + grp), (puse & 1) ^ 1)) { ok = false; }
-            if (full) probs32(std::true_type{}, va, 0); else probs32(std::false_type{}, va, 0);
+            if (full) probs32(std::true_type{}, std::true_type{}, va, 0); else probs32(std::false_type{}, std::true_type{}, va, 0);
             tmem_ld_wait_for(vb);
             tmem_ld32(tmSg + 64, va);
-            if (full) probs32(std::true_type{}, vb, 1); else probs32(std::false_type{}, vb, 1);
+            if (full) probs32(std::true_type{}, std::false_type{}, vb, 1); else probs32(std::false_type{}, std::false_type{}, vb, 1);
             tmem_ld_wait_for(va);
             tmem_ld32(tmSg + 96, vb);
-            if (full) probs32(std::true_type{}, va, 2); else probs32(std::false_type{}, va, 2);
+            if (full) probs32(std::true_type{}, std::false_type{}, va, 2); else probs32(std::false_type{}, std::false_type{}, va, 2);
             tmem_ld_wait_for(vb);
             tc_fence_before();  // last read of this S^T buffer
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(S_FREE + grp));
-            if (full) probs32(std::true_type{}, vb, 3); else probs32(std::false_type{}, vb, 3);
+            if (lane == 0) mbar_arrive(bar(S_FREE + buf));
+            if (full) probs32(std::true_type{}, std::false_type{}, vb, 3); else probs32(std::false_type{}, std::false_type{}, vb, 3);
             if (kvalid) part[lam] = colsum;
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(P_FULL + grp));
-            ++use;
             ++puse;
         }
         // keys this tile's queries cannot see contribute nothing
