@@ -53,6 +53,33 @@ def measured_peaks():
 
 
 # ------------------------------------------------------------------------------------------------------
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/, valid for the named workload's per-layer shape and only while the kernel's sources are the ones that
+# were profiled: a changed source file makes the entry stale and the reported traffic null.
+NCU_TRAFFIC = {
+    "decode_mma_kernel": {"workload": "cfg2", "bytes_per_launch": 143.36e6, "sources": ["decode_mma.cu", "common.cuh"],
+                          "sha1": "1afc9e2a4000719d6e71befc7dd9c1430dac6312", "profile": "profiles/decode_mma_cfg2_2layers.md"},
+    "prefill_tc_kernel": {"workload": "cfg5", "bytes_per_launch": 151.41e6, "sources": ["prefill_tc.cu", "tma.cuh", "common.cuh"],
+                          "sha1": "0e269cce2d0c159019cbd84d16fba047aa8b5588", "profile": "profiles/prefill_tc_cfg5_1layer.md"},
+}
+
+
+def measured_traffic(kernel, workload):
+    import hashlib
+
+    ent = NCU_TRAFFIC.get(kernel)
+    if ent is None or ent["workload"] != workload:
+        return None
+    h = hashlib.sha1()
+    try:
+        for f in ent["sources"]:
+            h.update(open(os.path.join(ROOT, "paper_2501_04987_b200", "csrc", f), "rb").read())
+    except OSError:
+        return None
+    return ent["bytes_per_launch"] if h.hexdigest() == ent["sha1"] else None
+
+
+# ------------------------------------------------------------------------------------------------------
 # algorithmic bytes / flops (what the method must move or compute)
 # ------------------------------------------------------------------------------------------------------
 def decode_bytes_per_unit(c, d, e, g):
@@ -380,7 +407,9 @@ def run_decode_leg(torch, binding, w, steps, warmup, e2e_steps, decode_split, de
     launch_ms = ms_total / (steps * w.layers)
     achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "frac": achieved / peaks["hbm_gbs"],
+                "traffic": measured_traffic("decode_mma_kernel" if w.dtype == "bf16" else "decode_kernel", w.name),
+                "peak_source": peaks["source"],
                 "kernel": "decode_mma_kernel" if w.dtype == "bf16" else "decode_kernel",
                 "bytes_per_launch": bytes_per_launch, "launch_us": launch_ms * 1e3, "frac_of_nominal_8TBs": achieved / 8000.0}
 
@@ -469,7 +498,8 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, world, rank, barrier, max
             "config": {"workload": pw.name, "layers": pw.layers, "batch_per_gpu": pw.batch, "n_heads": pw.n_heads,
                        "n_kv_heads": pw.n_kv_heads, "head_dim": pw.head_dim, "budget": c, "chunk": m},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                         "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " (sustained)",
+                         "frac": achieved / peak, "traffic": measured_traffic("prefill_tc_kernel", pw.name),
+                         "kernel": "prefill_tc_kernel", "peak_source": peaks["source"] + " (sustained)",
                          "flops_per_chunk_all_layers": flops_chunk}}
 
 
