@@ -15,12 +15,13 @@
 // Same three contractions and two exponentials per element as "attention, then recompute against the final
 // log-sum-exp", with the probabilities used for the output and for the scores being the same numbers.
 //
-// Warp roles: warp 0 issues TMA, warp 1 issues MMA and owns the tensor-memory allocation, warps 2-9 are two
-// groups of four softmax warps (one tensor-memory lane quarter per warp); group g takes the key tiles of parity
-// g and owns P^T buffer g, so the two groups alternate tiles and overlap each other's latency.  The S / S^T
-// accumulators are three tensor-memory buffers used round-robin by tile index, so the MMA warp can start a
-// tile's logits while both groups are still reading theirs.  All waits are bounded mbarrier waits; a wait that
-// gives up sets an error word and the CTA drains to its exit, where tensor memory is released.
+// Warp roles: warp 0 issues TMA, warp 1 issues MMA and owns the tensor-memory allocation, warps 2-17 are two
+// groups of eight softmax warps; inside a group a warp owns one tensor-memory lane quarter and one half of a
+// tile's 128 columns.  Group g takes the key tiles of parity g and owns P^T buffer g, so the two groups
+// alternate tiles and overlap each other's latency.  The S / S^T accumulators are three tensor-memory buffers
+// used round-robin by tile index, so the MMA warp can start a tile's logits while both groups are still reading
+// theirs.  All waits are bounded mbarrier waits; a wait that gives up sets an error word and the CTA drains to
+// its exit, where tensor memory is released.
 #include <type_traits>
 
 #include "common.cuh"
@@ -33,7 +34,7 @@ namespace {
 constexpr int kSlot = 32768;   // one tile: [2 halves of 64 channels or 64 queries][128 rows][128 bytes]
 constexpr int kHalf = 16384;
 constexpr int kRing = 4;       // K / V tiles in flight
-constexpr int kTcThreads = 320;
+constexpr int kTcThreads = 576;  // TMA warp, MMA warp, 2 groups x 8 softmax warps
 constexpr uint32_t kTmemCols = 512;
 constexpr int kD = 128;
 
@@ -98,8 +99,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (tid == 0) {
         mbar_init(bar(Q_FULL), 1);
         for (int s = 0; s < kRing; ++s) { mbar_init(bar(RING_FULL + s), 1); mbar_init(bar(RING_EMPTY + s), 1); }
-        for (int s = 0; s < kSBufs; ++s) { mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_FREE + s), 4); }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar(P_FULL + s), 4); mbar_init(bar(P_FREE + s), 1); }
+        for (int s = 0; s < kSBufs; ++s) { mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_FREE + s), 8); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar(P_FULL + s), 8); mbar_init(bar(P_FREE + s), 1); }
         mbar_init(bar(O_FULL), 1);
         mbar_fence_init();
     }
@@ -207,15 +208,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
     } else {
         // ================= softmax warps =================
-        const int grp = (warp - 2) >> 2;       // group 0: warps 2-5, group 1: warps 6-9; group g owns tiles j = g (mod 2)
+        const int sw = warp - 2;               // 0..15
+        const int grp = sw >> 3;               // group 0: warps 2-9, group 1: warps 10-17; group g owns tiles j = g (mod 2)
+        const int half = (sw >> 2) & 1;        // this warp handles columns [64*half, 64*half + 64) of a tile
         const int quarter = warp & 3;          // tensor-memory lanes [32*quarter, +32) belong to this warp
         const int row = quarter * 32 + lane;   // pass A: query row; pass B: key of the tile; epilogue: channel
         const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
         const float sc2 = kLog2e * rsqrtf((float)kD);
         float* nlse = lse;                     // [128] minus the log2-domain log-sum-exp of every query row
-        // per-group running (max, sum) of pass A, [2][128] each; they borrow the P^T area, which pass A does not use
+        // running (max, sum) of pass A per (group, column half), [4][128] each; they borrow the P^T area, which
+        // pass A does not use
         float* part_m = reinterpret_cast<float*>(base_ptr + (1 + kRing) * kSlot);
-        float* part_l = part_m + 256;
+        float* part_l = part_m + 512;
+        float* xch = lse + 128;                // [2][128] column sums handed from the upper to the lower column half
         uint32_t va[32], vb[32];  // two chunks of 32 columns: the next one is in flight while this one is used
         // ---- pass A: row statistics over this group's tiles
         {
@@ -262,34 +267,33 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         }
                     }
                 };
-                tmem_ld32(tmSg, va);
+                tmem_ld32(tmSg + 64 * half, va);
                 tmem_ld_wait_for(va);
-                tmem_ld32(tmSg + 32, vb);
-                stats32(va, 0);
-                tmem_ld_wait_for(vb);
-                tmem_ld32(tmSg + 64, va);
-                stats32(vb, 1);
-                tmem_ld_wait_for(va);
-                tmem_ld32(tmSg + 96, vb);
-                stats32(va, 2);
+                tmem_ld32(tmSg + 64 * half + 32, vb);
+                stats32(va, 2 * half);
                 tmem_ld_wait_for(vb);
                 tc_fence_before();  // last read of this S buffer: hand it back before the arithmetic on it
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(S_FREE + buf));
-                stats32(vb, 3);
+                stats32(vb, 2 * half + 1);
             }
-            part_m[grp * 128 + row] = mrun;
-            part_l[grp * 128 + row] = lrun;
+            part_m[(grp * 2 + half) * 128 + row] = mrun;
+            part_l[(grp * 2 + half) * 128 + row] = lrun;
         }
-        asm volatile("bar.sync 1, 256;" ::: "memory");  // both groups: the partial statistics are complete
-        if (grp == 0) {
-            const float m0 = part_m[row], m1 = part_m[128 + row];
-            const float M = fmaxf(m0, m1);
-            const float l = (m0 == -INFINITY ? 0.f : part_l[row] * ex2(m0 - M)) +
-                            (m1 == -INFINITY ? 0.f : part_l[128 + row] * ex2(m1 - M));
+        asm volatile("bar.sync 1, 512;" ::: "memory");  // all softmax warps: the partial statistics are complete
+        if (sw < 4) {
+            float M = -INFINITY;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) M = fmaxf(M, part_m[u * 128 + row]);
+            float l = 0.f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float mu = part_m[u * 128 + row];
+                if (mu != -INFINITY) l += part_l[u * 128 + row] * ex2(mu - M);
+            }
             nlse[row] = -(M + log2f(l));
         }
-        asm volatile("bar.sync 1, 256;" ::: "memory");  // nlse[] is complete
+        asm volatile("bar.sync 1, 512;" ::: "memory");  // nlse[] is complete
         // ---- pass B: probabilities, column sums, P^T for the tensor cores
         const int rmax = G * (t1 - t0);  // query columns [rmax, 128) are padding
         float* part = ps.colsum + ((size_t)unit * ps.QT + qt) * ps.n_max;
@@ -348,34 +352,38 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     *reinterpret_cast<uint4*>(prow + (cidx >> 3) * kHalf + (((cidx & 7) ^ (row & 7)) << 4)) = pk[q4];
                 }
             };
-            tmem_ld32(tmSg, va);
+            tmem_ld32(tmSg + 64 * half, va);
             tmem_ld_wait_for(va);
-            tmem_ld32(tmSg + 32, vb);
-            if (full) probs32(std::true_type{}, std::true_type{}, va, 0); else probs32(std::false_type{}, std::true_type{}, va, 0);
-            tmem_ld_wait_for(vb);
-            tmem_ld32(tmSg + 64, va);
-            if (full) probs32(std::true_type{}, std::false_type{}, vb, 1); else probs32(std::false_type{}, std::false_type{}, vb, 1);
-            tmem_ld_wait_for(va);
-            tmem_ld32(tmSg + 96, vb);
-            if (full) probs32(std::true_type{}, std::false_type{}, va, 2); else probs32(std::false_type{}, std::false_type{}, va, 2);
+            tmem_ld32(tmSg + 64 * half + 32, vb);
+            if (full) probs32(std::true_type{}, std::true_type{}, va, 2 * half); else probs32(std::false_type{}, std::true_type{}, va, 2 * half);
             tmem_ld_wait_for(vb);
             tc_fence_before();  // last read of this S^T buffer
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(S_FREE + buf));
-            if (full) probs32(std::true_type{}, std::false_type{}, vb, 3); else probs32(std::false_type{}, std::false_type{}, vb, 3);
-            if (kvalid) part[lam] = colsum;
+            if (full) probs32(std::true_type{}, std::false_type{}, vb, 2 * half + 1); else probs32(std::false_type{}, std::false_type{}, vb, 2 * half + 1);
+            // the key's column sum = lower half + upper half, added in that order.  The warp of the upper half hands
+            // its sum over through shared memory (named barrier of the two warps); it can only write the slot again
+            // after this tile's P^T has been consumed, which needs the lower half's arrival below.
+            const int pair_bar = 2 + grp * 4 + quarter;
+            if (half == 1) {
+                xch[grp * 128 + row] = colsum;
+                asm volatile("bar.arrive %0, 64;" ::"r"(pair_bar) : "memory");
+            } else {
+                asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+                if (kvalid) part[lam] = colsum + xch[grp * 128 + row];
+            }
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(P_FULL + grp));
             ++puse;
         }
         // keys this tile's queries cannot see contribute nothing
-        for (int lam = kt.nvis + (tid - 64); lam < n; lam += 256) part[lam] = 0.f;
-        // ---- epilogue: O^T (lane = channel, column = query row) -> out[token][head][channel]; each group half the columns
+        for (int lam = kt.nvis + (tid - 64); lam < n; lam += 512) part[lam] = 0.f;
+        // ---- epilogue: O^T (lane = channel, column = query row) -> out[token][head][channel]; 32 query columns per warp
         if (ok && mbar_wait(bar(O_FULL), 0)) {
             tc_fence_after();
-#pragma unroll 1
-            for (int cg = 2 * grp; cg < 2 * grp + 2; ++cg) {
+            {
+                const int cg = sw >> 2;  // one chunk of 32 query columns per warp
                 tmem_ld32(tmO + lane_off + cg * 32, va);
                 tmem_ld_wait_for(va);
 #pragma unroll
@@ -395,7 +403,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
-size_t prefill_tc_smem_bytes() { return 1024 + (size_t)(3 + kRing) * kSlot + 128 * sizeof(float); }
+size_t prefill_tc_smem_bytes() { return 1024 + (size_t)(3 + kRing) * kSlot + (128 + 256) * sizeof(float); }
 
 template <int G>
 static cudaError_t launch_prefill_tc_t(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ,
