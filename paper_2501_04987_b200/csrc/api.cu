@@ -232,17 +232,13 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
     if (chunk_stride < 1) return TREEKV_ERR_INVALID_ARG;
     ChunkLens lens;
     memset(&lens, 0, sizeof(lens));
-    int max_m = 0, max_seg = 0;
+    int max_m = 0;
     for (int b = 0; b < ctx->cv.B; ++b) {
         const int m = host_chunk_lens ? host_chunk_lens[b] : chunk_stride;
         if (m < 0 || m > chunk_stride || m > ctx->max_chunk) return TREEKV_ERR_INVALID_ARG;
         if (ctx->n_seen[b] + m >= 0x7fffffff - 1) return TREEKV_ERR_BAD_STATE;
         lens.m[b] = (uint16_t)m;
         if (m > max_m) max_m = m;
-        if (m > 0) {
-            const int ns = evict_segment(ctx->n_seen[b], m, ctx->cv.c, 0).nseg;
-            if (ns > max_seg) max_seg = ns;
-        }
     }
     if (max_m == 0) return TREEKV_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -260,23 +256,10 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
         e = launch_prefill_simt(ctx->cv, ctx->dt, ctx->ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = launch_chunk_scores(ctx->cv, ctx->ps, lens, max_m, s);
+    // score update, all eviction segments and the token counters in one launch
+    e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    ctx->launches += 3;
-    for (int seg = 0; seg < max_seg; ++seg) {
-        int max_items = 0;
-        for (int b = 0; b < ctx->cv.B; ++b) {
-            if (!lens.m[b]) continue;
-            const EvictSegment sg = evict_segment(ctx->n_seen[b], lens.m[b], ctx->cv.c, seg);
-            if (sg.E + sg.rebase > max_items) max_items = sg.E + sg.rebase;
-        }
-        e = launch_chunk_evict(ctx->cv, ctx->dt, ctx->ps, lens, seg, max_items, s);
-        if (e != cudaSuccess) return cuda_fail(ctx, e);
-        ctx->launches += 2;
-    }
-    e = launch_chunk_finalize(ctx->cv, lens, s);
-    if (e != cudaSuccess) return cuda_fail(ctx, e);
-    ctx->launches += 1;
+    ctx->launches += 3;  // append, attention, update + eviction
     for (int b = 0; b < ctx->cv.B; ++b) {
         const int64_t before = ctx->n_seen[b];
         ctx->n_seen[b] += lens.m[b];

@@ -197,6 +197,9 @@ cudaError_t launch_chunk_scores(const CacheView& cv, const PrefillScratch& ps, c
 cudaError_t launch_chunk_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
                                int seg, int max_items, cudaStream_t stream);  // gather + scatter: two launches
 cudaError_t launch_chunk_finalize(const CacheView& cv, const ChunkLens& lens, cudaStream_t stream);
+// score update + every eviction segment + n_seen update of a chunk in one launch (a cluster per unit)
+cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
+                                      cudaStream_t stream);
 
 size_t prefill_simt_smem_bytes(int G, int D, int n_max);
 cudaError_t launch_prefill_simt(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const void* q, void* out,

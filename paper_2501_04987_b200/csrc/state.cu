@@ -1,6 +1,8 @@
 // Cache-state kernels of the TreeKV library: initialisation, read-outs in cache order, and the per-chunk
 // steps around prefill attention: append, score update (Algorithm 1: S <- S + a, summed over the chunk),
 // repeated pair eviction with frozen scores, compaction.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace treekv {
@@ -209,6 +211,121 @@ cudaError_t launch_chunk_evict(const CacheView& cv, treekv_dtype dt, const Prefi
             e = launch_pdl(chunk_evict_scatter_kernel<__nv_bfloat16>, grid, dim3(256), 0, stream, cv, ps, lens, seg);
     }
     return e;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// The three steps above in one launch: score update, every eviction segment of the chunk, n_seen += m.
+// A cluster of kEvictCluster thread blocks owns one unit.  Inside a segment the pairs are taken in rounds of
+// increasing pair index; a round first reads everything it moves into registers (decision, survivor's K and V
+// rows, its S and position), the cluster synchronises, then the round writes.  That is enough because the
+// destination row i+p of pair p can only be a source row of an earlier pair ((p-i)/2 < p) - read in this round
+// or a previous one - and never of a later pair; rows moved down after a wrap follow the same rule.  A new
+// segment starts after a further cluster barrier, since its pairs read rows the previous one wrote.
+constexpr int kEvictCluster = 4;
+constexpr int kEvictThreads = 512;
+constexpr int kEvictItemsPerWarp = 4;
+
+template <typename T>
+__global__ void __cluster_dims__(kEvictCluster, 1, 1) __launch_bounds__(kEvictThreads)
+chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
+    pdl_trigger();
+    pdl_wait();
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int unit = blockIdx.y;
+    const int b = unit / cv.Hkv;
+    const int m = lens.m[b];
+    if (m == 0) return;  // the whole cluster shares the unit
+    const int rank = (int)cluster.block_rank();
+    const int G = cv.Hq / cv.Hkv;
+    const int N = cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv.c);
+    const int n = st.L + m;
+    const int N1 = N + m;
+    T* Kc = reinterpret_cast<T*>(cv.K) + (size_t)unit * cv.R * cv.d;
+    T* Vc = reinterpret_cast<T*>(cv.V) + (size_t)unit * cv.R * cv.d;
+    float* Sc = cv.S + (size_t)unit * cv.R;
+    int32_t* Pc = cv.pos + (size_t)unit * cv.R;
+
+    // ---- score update (Algorithm 1: S <- S + a, summed over the chunk's steps; group mean): tiles added in a
+    //      fixed order so the result does not depend on scheduling
+    {
+        const int qt = (m * G + kQTileRows - 1) / kQTileRows;
+        const float inv_g = 1.0f / (float)G;
+        for (int lam = rank * kEvictThreads + threadIdx.x; lam < n; lam += kEvictCluster * kEvictThreads) {
+            const float* part = ps.colsum + (size_t)unit * ps.QT * ps.n_max + lam;
+            float s = 0.f;
+            for (int t = 0; t < qt; ++t) s += part[(size_t)t * ps.n_max];
+            float* Sp = Sc + phys_row(lam, st.i);
+            *Sp = *Sp + s * inv_g;  // chunk rows were zeroed by the append
+        }
+    }
+    cluster.sync();  // every S of the unit is final; every block has read n_seen
+    if (rank == 0 && threadIdx.x == 0) cv.n_seen[unit] = N1;
+
+    // ---- eviction segments (Algorithm 1's "length > c" branch repeated with the scores frozen)
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gwarp = rank * (kEvictThreads / 32) + warp;
+    constexpr int kWarps = kEvictCluster * kEvictThreads / 32;
+    constexpr int kRound = kWarps * kEvictItemsPerWarp;
+    const int chunks = cv.d * (int)sizeof(T) / 16;  // 16-byte pieces per row: at most 32
+    const int nseg = evict_segment(N, m, cv.c, 0).nseg;
+    for (int seg = 0; seg < nseg; ++seg) {
+        const EvictSegment sg = evict_segment(N, m, cv.c, seg);
+        const int items = sg.E + sg.rebase;
+        for (int r0 = 0; r0 < items; r0 += kRound) {
+            uint4 kr[kEvictItemsPerWarp], vr[kEvictItemsPerWarp];
+            float sr[kEvictItemsPerWarp];
+            int32_t pr[kEvictItemsPerWarp];
+#pragma unroll
+            for (int u = 0; u < kEvictItemsPerWarp; ++u) {
+                const int item = r0 + u * kWarps + gwarp;
+                if (item >= items) continue;
+                int src;
+                if (item < sg.E) {
+                    const int l = 2 * (sg.i + item), r = l + 1;
+                    int evict_right = 0;
+                    if (lane == 0) {
+                        bool near_tie = false;
+                        evict_right = pair_evicts_right(Sc[l], N1 - Pc[l], Sc[r], N1 - Pc[r], cv.rule, &near_tie) ? 1 : 0;
+                        if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
+                    }
+                    evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
+                    src = evict_right ? l : r;
+                } else {
+                    src = 2 * cv.c + (item - sg.E);
+                }
+                if (lane < chunks) {
+                    kr[u] = reinterpret_cast<const uint4*>(Kc + (size_t)src * cv.d)[lane];
+                    vr[u] = reinterpret_cast<const uint4*>(Vc + (size_t)src * cv.d)[lane];
+                }
+                if (lane == 0) { sr[u] = Sc[src]; pr[u] = Pc[src]; }
+            }
+            cluster.sync();  // everything this round moves has been read
+#pragma unroll
+            for (int u = 0; u < kEvictItemsPerWarp; ++u) {
+                const int item = r0 + u * kWarps + gwarp;
+                if (item >= items) continue;
+                const int dst = item < sg.E ? sg.i + item : cv.c + (item - sg.E);
+                if (lane < chunks) {
+                    reinterpret_cast<uint4*>(Kc + (size_t)dst * cv.d)[lane] = kr[u];
+                    reinterpret_cast<uint4*>(Vc + (size_t)dst * cv.d)[lane] = vr[u];
+                }
+                if (lane == 0) { Sc[dst] = sr[u]; Pc[dst] = pr[u]; }
+            }
+        }
+        if (seg + 1 < nseg) cluster.sync();  // the next segment's pairs read rows this one wrote
+    }
+}
+
+cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
+                                      cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kEvictCluster, cv.B * cv.Hkv);
+    cfg.blockDim = dim3(kEvictThreads);
+    cfg.stream = stream;  // plain stream order behind the attention kernel; the kernel after it may be scheduled early
+    if (dt == TREEKV_F32) return cudaLaunchKernelEx(&cfg, chunk_update_evict_kernel<float>, cv, ps, lens);
+    return cudaLaunchKernelEx(&cfg, chunk_update_evict_kernel<__nv_bfloat16>, cv, ps, lens);
 }
 
 __global__ void chunk_finalize_kernel(CacheView cv, ChunkLens lens) {
