@@ -57,10 +57,10 @@ def measured_peaks():
 # profiles/, valid for the named workload's per-layer shape and only while the kernel's sources are the ones that
 # were profiled: a changed source file makes the entry stale and the reported traffic null.
 NCU_TRAFFIC = {
-    "decode_mma_kernel": {"workload": "cfg2", "bytes_per_launch": 143.36e6, "sources": ["decode_mma.cu", "common.cuh"],
-                          "sha1": "1afc9e2a4000719d6e71befc7dd9c1430dac6312", "profile": "profiles/decode_mma_cfg2_2layers.md"},
-    "prefill_tc_kernel": {"workload": "cfg5", "bytes_per_launch": 151.41e6, "sources": ["prefill_tc.cu", "tma.cuh", "common.cuh"],
-                          "sha1": "0e269cce2d0c159019cbd84d16fba047aa8b5588", "profile": "profiles/prefill_tc_cfg5_1layer.md"},
+    "decode_mma_kernel": {"workload": "cfg2", "bytes_per_launch": 143.23e6, "sources": ["decode_mma.cu", "common.cuh"],
+                          "sha1": "49abcff8fbecaaad30f01f1689169c5593e57236", "profile": "profiles/decode_mma_cfg2_2layers.md"},
+    "prefill_tc_kernel": {"workload": "cfg5", "bytes_per_launch": 154.19e6, "sources": ["prefill_tc.cu", "tma.cuh", "common.cuh"],
+                          "sha1": "e0784954221202f2447c9c9c85eda2331622d937", "profile": "profiles/prefill_tc_cfg5_1layer.md"},
 }
 
 
