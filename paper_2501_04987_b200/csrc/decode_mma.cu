@@ -184,7 +184,6 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     //      S of this CTA's rows (4-byte cp.async; they join the first commit group), and in CTA 0 the K/V rows of
     //      the eviction scope (rows 2i and 2i+1; the new token's row comes from k_in / v_in)
     const bool will_evict = (N + 1 > cv.c);
-    static_assert(NT % D == 0, "a thread always combines the same channel");
     int pos_l = 0, pos_r = 0;  // stream positions of the scope's two tokens (used by lane 0 of warp 0 in CTA 0)
     if (rank == 0 && will_evict && tid == 0) {
         pos_l = Pc[2 * i_cyc];
@@ -212,7 +211,6 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     const T* tq = reinterpret_cast<const T*>(tok);
     const T* tk = reinterpret_cast<const T*>(tok + G * ROWB);
     const T* tv = reinterpret_cast<const T*>(tok + (G + 1) * ROWB);
-    const float vnew_r = owns_new ? __bfloat162float(tv[tid % D]) : 0.f;  // this thread's channel of the new value row
 
     // ---- append (Algorithm 1: K <- K u {k}, V <- V u {v}); the step itself uses the staged copy of the new token
     if (warp == NW - 1) {
@@ -383,7 +381,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         }
         if (owns_new) {
             const float f = exp2_diff(wstat[(NW * 2) * G + h], M);
-            o += vnew_r * f;
+            o += __bfloat162float(tv[ch]) * f;
             l += f;
         }
         o_all0[(size_t)rank * G * D + idx] = o;

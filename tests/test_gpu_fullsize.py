@@ -194,3 +194,44 @@ def test_cfg5_full_layer_ragged_prefill(gpu):
     lens = [2 * 4096 + 1024 + 517, 2 * 4096 + 100, 10 * 1024, 2 * 4096 + 1]
     err = _prefill_fullsize(gpu, w, lens, decode_steps=24)
     print("cfg5 full layer: max sampled out err %.3g" % err)
+
+
+def test_large_budget_decode_through_eight_block_clusters(gpu):
+    """A budget of 16384 with one sequence and two KV heads (g = 4): the decode kernel runs as clusters of eight
+    blocks with 2049 rows each, close to the largest shared-memory footprint the library accepts.  The cache is
+    filled token by token, then steps across the first evictions are checked on every head against fp64 softmax
+    attention over the retained set, with the cache invariants."""
+    import torch
+
+    c, Hq, Hkv, d, B = 16384, 8, 2, 128, 1
+    g = Hq // Hkv
+    kv = gpu.TreeKV(c, Hq, Hkv, d, "bf16", B, 0)
+    gen = torch.Generator(device="cuda"); gen.manual_seed(20250111)
+    steps = c + 24
+    q = _draw(torch, gen, (steps, B, Hq, d))
+    k = _draw(torch, gen, (steps, B, Hkv, d))
+    v = _draw(torch, gen, (steps, B, Hkv, d))
+    kh64 = k[:, 0].float().cpu().numpy().astype(np.float64)   # [steps, Hkv, d]
+    vh64 = v[:, 0].float().cpu().numpy().astype(np.float64)
+    out = torch.empty((B, Hq, d), dtype=torch.bfloat16, device="cuda")
+    max_err = 0.0
+    for t in range(steps):
+        check = t >= c - 8 or t in (0, 1, 17, 4097)
+        if check:
+            pos_before, cnt_before = kv.retained_positions()
+            pos_before = pos_before.cpu().numpy(); cnt_before = cnt_before.cpu().numpy()
+        kv.decode_step(q[t], k[t], v[t], out)
+        if check:
+            o = out.float().cpu().numpy()
+            for kh in range(Hkv):
+                vis = np.concatenate([pos_before[0, kh, : cnt_before[0, kh]], [t]])
+                for hh in range(g):
+                    h = kh * g + hh
+                    ref = _softmax_rows(q[t, 0, h].float().cpu().numpy().astype(np.float64), kh64[vis, kh], vh64[vis, kh])
+                    err = float(np.abs(o[0, h] - ref).max())
+                    max_err = max(max_err, err)
+                    assert err <= 2e-2, (t, h, err)
+    _check_invariants(kv, [steps])
+    st = kv.stats()
+    assert st["device_error"] == 0 and st["evictions"] == steps - c
+    print("c=16384 decode: max out err %.3g" % max_err)
