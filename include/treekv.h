@@ -63,7 +63,8 @@ typedef enum { TREEKV_RULE_SCORES = 0, TREEKV_RULE_KEEP_LEFT = 1, TREEKV_RULE_EV
 /* Options for treekv_set_option. */
 typedef enum {
     TREEKV_OPT_DECODE_SPLIT = 0, /* thread blocks per (sequence, KV head) in decode: 0 = automatic, else 1,2,4,8 */
-    TREEKV_OPT_PREFILL_PATH = 1, /* 0 = automatic, 1 = CUDA-core kernel, 2 = tcgen05 tensor-core kernel (bf16, head_dim 128) */
+    TREEKV_OPT_PREFILL_PATH = 1, /* 0 = automatic, 1 = CUDA-core kernel, 2 / 3 = tcgen05 tensor-core kernel with 128 / 256
+                                    query rows per thread block (bf16, head_dim 128) */
     TREEKV_OPT_DECODE_PATH = 2   /* 0 = automatic, 1 = CUDA-core kernel, 2 = cp.async + mma.sync kernel (bf16 only) */
 } treekv_option;
 

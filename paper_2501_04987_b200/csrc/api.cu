@@ -251,7 +251,11 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
         const uint64_t strides[2] = {256ull, (uint64_t)ctx->cv.Hq * 256ull};
         const uint32_t box[3] = {64u, (uint32_t)ctx->G, (uint32_t)(128 / ctx->G)};
         if (!make_tensor_map_bf16(&tmQ, dev_q, 3, dims, strides, box)) return TREEKV_ERR_CUDA;
-        e = launch_prefill_tc(ctx->cv, ctx->ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s);
+        // two query tiles per CTA once the one-tile grid would cover the machine at least twice (or on request)
+        const long tiles = (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + kQTileRows - 1) / kQTileRows);
+        const bool two = ctx->opt_prefill_path == 3 || (ctx->opt_prefill_path == 0 && tiles >= 2L * ctx->sm_count);
+        e = two ? launch_prefill_tc2(ctx->cv, ctx->ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s)
+                : launch_prefill_tc(ctx->cv, ctx->ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s);
     } else {
         e = launch_prefill_simt(ctx->cv, ctx->dt, ctx->ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
     }
@@ -376,8 +380,8 @@ treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value) {
             ctx->opt_decode_split = 0;
             return TREEKV_OK;
         case TREEKV_OPT_PREFILL_PATH:
-            if (value < 0 || value > 2) return TREEKV_ERR_INVALID_ARG;
-            if (value == 2 && !ctx->has_tma) return TREEKV_ERR_UNSUPPORTED;
+            if (value < 0 || value > 3) return TREEKV_ERR_INVALID_ARG;
+            if (value >= 2 && !ctx->has_tma) return TREEKV_ERR_UNSUPPORTED;
             ctx->opt_prefill_path = value;
             return TREEKV_OK;
     }

@@ -205,6 +205,11 @@ size_t prefill_simt_smem_bytes(int G, int D, int n_max);
 cudaError_t launch_prefill_simt(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const void* q, void* out,
                                 const ChunkLens& lens, int chunk_stride, int max_m, cudaStream_t stream);
 
+size_t prefill_tc2_smem_bytes();
+cudaError_t launch_prefill_tc2(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                               const CUtensorMap& tmV, void* out, const ChunkLens& lens, int chunk_stride, int max_m,
+                               cudaStream_t stream);  // 256 query rows per CTA, for large grids
+
 size_t prefill_tc_smem_bytes();
 cudaError_t launch_prefill_tc(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                               const CUtensorMap& tmV, void* out, const ChunkLens& lens, int chunk_stride, int max_m,

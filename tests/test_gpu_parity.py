@@ -126,6 +126,25 @@ def test_cfg5_slice_ragged_gqa_prefill(gpu):
     print("cfg5 slice", rep)
 
 
+@pytest.mark.parametrize("g,lens,chunk,budget", [
+    (4, [2 * 1024 + 517, 2 * 1024 + 40], 512, 1024),   # GQA, ragged tails: a partial last tile and an empty second sub-tile
+    (1, [5 * 384 + 200, 3 * 384], 384, 512),           # MHA, 1.5 pairs of tiles per chunk, chunks that wrap the idx cycle
+    (8, [1300, 64], 256, 256),                         # eight heads per group: 16 tokens per sub-tile
+])
+def test_two_tile_tensor_core_prefill_kernel(gpu, g, lens, chunk, budget):
+    """The prefill kernel that gives a thread block two tiles of 128 query rows is only chosen for large grids;
+    here it is forced on small ragged cases and followed in lock-step like the one-tile kernel."""
+    w = W.parity_slice(W.CONFIGS["cfg5"], layers=1, batch=2, n_heads=g * 2, n_kv_heads=2, budget=budget, chunk=chunk)
+    kv, orc = _pair(gpu, w)
+    kv.set_option(gpu.OPT_PREFILL_PATH, 3)
+    rep = Report()
+    _run_prefill(kv, orc, w, rep, lens, chunk)
+    assert [kv.tokens_seen(b) for b in range(2)] == lens
+    _run_decode(kv, orc, w, 0, 8, rep, starts=lens)
+    assert kv.stats()["device_error"] == 0
+    print("two-tile prefill g=%d" % g, rep)
+
+
 # ---------------------------------------------------------------------------------------------------------
 # edge cases
 # ---------------------------------------------------------------------------------------------------------
