@@ -57,10 +57,10 @@ def measured_peaks():
 # profiles/, valid for the named workload's per-layer shape and only while the kernel's sources are the ones that
 # were profiled: a changed source file makes the entry stale and the reported traffic null.
 NCU_TRAFFIC = {
-    "decode_mma_kernel": {"workload": "cfg2", "bytes_per_launch": 143.23e6, "sources": ["decode_mma.cu", "common.cuh"],
-                          "sha1": "49abcff8fbecaaad30f01f1689169c5593e57236", "profile": "profiles/decode_mma_cfg2_2layers.md"},
-    "prefill_tc_kernel": {"workload": "cfg5", "bytes_per_launch": 154.19e6, "sources": ["prefill_tc.cu", "tma.cuh", "common.cuh"],
-                          "sha1": "e0784954221202f2447c9c9c85eda2331622d937", "profile": "profiles/prefill_tc_cfg5_1layer.md"},
+    "decode_mma_kernel": {"workload": "cfg2", "bytes_per_launch": 143.45e6, "sources": ["decode_mma.cu", "common.cuh"],
+                          "sha1": "6e49e213c0340309b66a4adb8c8f28a6f7959f9d", "profile": "profiles/decode_mma_cfg2_2layers.md"},
+    "prefill_tc2_kernel": {"workload": "cfg5", "bytes_per_launch": 150.25e6, "sources": ["prefill_tc2.cu", "tma.cuh", "common.cuh"],
+                           "sha1": "f16ca499efd5c223035411d1d369e3d0c875aba8", "profile": "profiles/prefill_tc2_cfg5_1layer.md"},
 }
 
 
@@ -488,6 +488,9 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, world, rank, barrier, max
     ms = max_over_ranks(ev0.elapsed_time(ev1))
     launches = sum(x.stats()["kernel_launches"] for x in ctxs) - launches0
     tok_s = whole_job_rate(world, n_chunks * m * pw.batch, ms)
+    # the library gives a thread block two 128-row query tiles once the one-tile grid covers the GPU at least twice
+    tiles = pw.batch * pw.n_kv_heads * ((m * pw.group + 127) // 128)
+    kernel = "prefill_tc2_kernel" if tiles >= 2 * torch.cuda.get_device_properties(dev).multi_processor_count else "prefill_tc_kernel"
     flops_chunk = pw.layers * pw.batch * pw.n_heads * prefill_flops_per_head_chunk(m, c, pw.head_dim)
     achieved = flops_chunk * n_chunks / (ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
@@ -498,8 +501,8 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, world, rank, barrier, max
             "config": {"workload": pw.name, "layers": pw.layers, "batch_per_gpu": pw.batch, "n_heads": pw.n_heads,
                        "n_kv_heads": pw.n_kv_heads, "head_dim": pw.head_dim, "budget": c, "chunk": m},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                         "frac": achieved / peak, "traffic": measured_traffic("prefill_tc_kernel", pw.name),
-                         "kernel": "prefill_tc_kernel", "peak_source": peaks["source"] + " (sustained)",
+                         "frac": achieved / peak, "traffic": measured_traffic(kernel, pw.name),
+                         "kernel": kernel, "peak_source": peaks["source"] + " (sustained)",
                          "flops_per_chunk_all_layers": flops_chunk}}
 
 
