@@ -90,14 +90,16 @@ size_t decode_smem_for(const treekv_ctx* ctx, int split) {
 
 // Thread blocks (cluster size) per unit.  The bf16 kernel keeps one CTA per unit once there are at least as many
 // units as SMs (its CTAs are small and several are resident per SM) and otherwise splits until the machine is
-// covered about twice; the CUDA-core kernel splits while a CTA keeps at least 128 rows.
+// covered about twice - but clusters of eight only while all CTAs fit one per SM: a cluster must be placed inside
+// one GPC, and with more CTAs than SMs some clusters of eight waited for a second wave.  The CUDA-core kernel
+// splits while a CTA keeps at least 128 rows.
 int pick_decode_split(const treekv_ctx* ctx) {
     const int c = ctx->cv.c, units = ctx->cv.B * ctx->cv.Hkv;
     int s = ctx->opt_decode_split;
     if (s == 0) {
         s = 1;
         if (use_mma_decode(ctx)) {
-            while (s < 8 && units * (2 * s) <= 2 * ctx->sm_count && (c + 1) / (2 * s) >= 64) s *= 2;
+            while (s < 8 && units * (2 * s) <= (2 * s == 8 ? 1 : 2) * ctx->sm_count && (c + 1) / (2 * s) >= 64) s *= 2;
         } else {
             while (s < 8 && units * s < 3 * ctx->sm_count && (c + 1) / (2 * s) >= 128) s *= 2;
         }

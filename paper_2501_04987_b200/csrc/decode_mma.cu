@@ -405,6 +405,26 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         for (int r = 0; r < nsplit; ++r) L += gstat[(r * 2 + 1) * G + h] * exp2_diff(gstat[(r * 2) * G + h], M);
         Mg[h] = M; invL[h] = 1.0f / L;
     }
+    // ---- in a cluster of several CTAs the scope's two updated scores go to CTA 0 first (remote shared-memory
+    //      stores), and the cluster barrier is split around the bulk of the global stores: arrive now - its release
+    //      only has these few stores to cover - and wait after the output and the score update have been issued.
+    //      Each value is computed with the same expression the bulk loop uses.
+    const int ncached = nrows - (owns_new ? 1 : 0);
+    auto updated_score = [&](int j) {  // j: index among this CTA's rows; the appended token starts from S = 0
+        float ps = 0.f;
+#pragma unroll
+        for (int h = 0; h < G; ++h) ps += exp2f(sl[h * rows_cap + j] - Mg[h]) * invL[h];
+        return (j < ncached ? s_old[j] : 0.f) + ps * (1.0f / G);
+    };
+    if (nsplit > 1) {
+        if (will_evict && tid < 2) {
+            const int lam = i_cyc + tid;  // live indices of physical rows 2i and 2i+1
+            if (lam >= lo && lam < hi) cluster.map_shared_rank(pair_s, 0)[tid] = updated_score(lam - lo);
+        }
+        __syncwarp();
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    }
+
     if (rank == 0) {
 #pragma unroll
         for (int h = 0; h < G; ++h) {
@@ -417,29 +437,25 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         }
     }
     // ---- normalised probabilities; score update (Algorithm 1: S <- (S u {0}) + a, group mean)
-    //      (a masked or padded logit is -inf and 2^-inf = 0, so exp2f needs no guard here: Mg is finite)
-    const int ncached = nrows - (owns_new ? 1 : 0);
+    //      (a masked or padded logit is -inf and 2^-inf = 0, so exp2f needs no guard here: Mg is finite).  The two
+    //      rows of the scope are left to the eviction below, which writes the survivor's score to its new row.
 #pragma unroll 4
     for (int j = tid; j < ncached; j += NT) {
-        float ps = 0.f;
-#pragma unroll
-        for (int h = 0; h < G; ++h) ps += exp2f(sl[h * rows_cap + j] - Mg[h]) * invL[h];
         const int ph = phys_row(lo + j, i_cyc);
-        const float s_new = s_old[j] + ps * (1.0f / G);
-        Sc[ph] = s_new;
-        if (nsplit == 1 && (ph >> 1) == i_cyc) pair_s[ph & 1] = s_new;  // the scope's scores stay on chip
+        const float s_new = updated_score(j);
+        if (!(will_evict && (ph >> 1) == i_cyc)) Sc[ph] = s_new;
+        else if (nsplit == 1) pair_s[ph & 1] = s_new;  // a single CTA takes the scope's scores from its own loop
     }
-    if (owns_new && tid == NT - 1) {  // the appended token starts from S = 0
-        float ps = 0.f;
-#pragma unroll
-        for (int h = 0; h < G; ++h) ps += exp2f(sl[h * rows_cap + ncached] - Mg[h]) * invL[h];
-        const float s_new = ps * (1.0f / G);
-        Sc[new_row] = s_new;
+    if (owns_new && tid == NT - 1) {
         Pc[new_row] = N;
-        if (nsplit == 1 && (new_row >> 1) == i_cyc) pair_s[new_row & 1] = s_new;
+        const float s_new = updated_score(ncached);
+        if (!(will_evict && (new_row >> 1) == i_cyc)) Sc[new_row] = s_new;
+        else if (nsplit == 1) pair_s[new_row & 1] = s_new;
     }
 
-    unit_barrier();  // (B) the appended row and every S update of the unit are complete
+    // (B) the scope's scores have arrived in CTA 0
+    if (nsplit > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    else __syncthreads();
 
     if (rank == 0 && warp == 0 && will_evict) {
         // ---- Algorithm 1, "length > c" branch: scope {idx, idx+1} = physical rows (2i, 2i+1)
@@ -448,12 +464,12 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         int evict_right = 0;
         if (lane == 0) {
             bool near_tie = false;
-            const float S_l = nsplit == 1 ? pair_s[0] : __ldcg(Sc + l);
-            const float S_r = nsplit == 1 ? pair_s[1] : __ldcg(Sc + r);
+            const float S_l = pair_s[0], S_r = pair_s[1];
             evict_right = pair_evicts_right(S_l, N1 - pos_l, S_r, N1 - pos_r, cv.rule, &near_tie) ? 1 : 0;
             if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
             const int src = evict_right ? l : r;
-            if (src != i_cyc) { Sc[i_cyc] = evict_right ? S_l : S_r; Pc[i_cyc] = evict_right ? pos_l : pos_r; }
+            Sc[i_cyc] = evict_right ? S_l : S_r;  // also when the survivor stays in place: the score update skipped the scope
+            Pc[i_cyc] = evict_right ? pos_l : pos_r;
         }
         evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
         const int src = evict_right ? l : r, dst = i_cyc;
