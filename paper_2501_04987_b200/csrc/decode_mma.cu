@@ -30,6 +30,16 @@ __device__ inline void cp_async_16(uint32_t dst, const void* src, bool valid) {
     const int sz = valid ? 16 : 0;  // src-size 0: the 16 destination bytes are zero-filled
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
 }
+// the same copy for data that is read once: its L2 lines are the first to be replaced
+__device__ inline void cp_async_16_stream(uint32_t dst, const void* src, bool valid, uint64_t policy) {
+    const int sz = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;" ::"r"(dst), "l"(src), "r"(sz), "l"(policy) : "memory");
+}
+__device__ inline uint64_t l2_evict_first_policy() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
 __device__ inline void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ inline void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
@@ -51,10 +61,15 @@ __device__ inline uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+// bulk L2 prefetch of a 16-byte aligned range whose size is a multiple of 16
+__device__ inline void l2_prefetch(const void* p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
 // 2^(a-b) with the convention 2^(-inf - anything) = 0, so empty partials (max = -inf) never produce NaN
 __device__ inline float exp2_diff(float a, float b) { return a == -INFINITY ? 0.f : exp2f(a - b); }
 
 constexpr int kBlk = 16;      // keys per pipeline stage
+constexpr int kPrefetchRows = 256;  // rows of K and of V a CTA asks L2 for before its stream-order wait (0 = none)
 constexpr int kMaxSplit = 8;  // largest cluster
 constexpr int kMmaWarps = 4;
 constexpr int kMmaStages = 2;
@@ -85,10 +100,34 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     // Programmatic dependent launch: the next kernel in the stream may be scheduled while this one runs (it does
     // the same), and nothing below the wait is read before the previous kernel's writes are complete and visible.
     pdl_trigger();
+    const int unit = b * cv.Hkv + kh;
+    // While the previous kernel of the stream drains, ask L2 for the first rows this CTA will stream.  This is a hint
+    // and nothing more: the token count is read before the wait and may be one step old (the rows then shift by one),
+    // no data reaches a register, and L2 is the point of coherence, so a line that the previous kernel still writes
+    // is simply up to date when it is read after the wait.
+    if (kPrefetchRows > 0 && threadIdx.x == 0 && active.test(b)) {
+        int Ns;
+        asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(Ns) : "l"(cv.n_seen + unit));
+        if (Ns >= 0) {
+            const UnitState ss = unit_state(Ns, cv.c);
+            const int blk_all = (ss.L + 1 + kBlk - 1) / kBlk, per = (blk_all + nsplit - 1) / nsplit;
+            const int lo_s = min(rank * per * kBlk, ss.L), hi_s = min(min(lo_s + per * kBlk, ss.L), lo_s + kPrefetchRows);
+            const unsigned char* Kb = reinterpret_cast<const unsigned char*>(cv.K) + (size_t)unit * cv.R * ROWB;
+            const unsigned char* Vb = reinterpret_cast<const unsigned char*>(cv.V) + (size_t)unit * cv.R * ROWB;
+            const int a1 = min(hi_s, max(lo_s, ss.i));  // live indices [lo_s, a1) sit at row = index, [a1, hi_s) at index + i
+            if (a1 > lo_s) {
+                l2_prefetch(Kb + (size_t)lo_s * ROWB, (uint32_t)(a1 - lo_s) * ROWB);
+                l2_prefetch(Vb + (size_t)lo_s * ROWB, (uint32_t)(a1 - lo_s) * ROWB);
+            }
+            if (hi_s > a1) {
+                l2_prefetch(Kb + (size_t)(a1 + ss.i) * ROWB, (uint32_t)(hi_s - a1) * ROWB);
+                l2_prefetch(Vb + (size_t)(a1 + ss.i) * ROWB, (uint32_t)(hi_s - a1) * ROWB);
+            }
+        }
+    }
     pdl_wait();  // every block waits, also one of an inactive sequence
     if (!active.test(b)) return;  // the whole cluster shares b
 
-    const int unit = b * cv.Hkv + kh;
     const int N = cv.n_seen[unit];
     const UnitState st = unit_state(N, cv.c);
     const int n = st.L + 1;  // live rows including the token appended by this step
@@ -149,6 +188,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     const int c_rsub = lane / CPR, c_cidx = lane % CPR;
     const uint32_t c_lane_off = c_rsub * ITERS * ROWB;  // lane's first row = rsub * ITERS
     const int c_row7 = (c_rsub * ITERS) & 7;            // (row & 7) of iteration `it` is c_row7 + it (no carry)
+    const uint64_t stream_policy = l2_evict_first_policy();  // K and V rows are read once per step
     auto issue = [&](int blk, int stage) {
         if (blk < nblk) {
             const uint32_t kst = ring_w + stage * STAGE, vst = kst + kBlk * ROWB;
@@ -162,8 +202,8 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
 #pragma unroll
                 for (int it = 0; it < ITERS; ++it) {
                     const uint32_t off = c_lane_off + it * ROWB + ((c_cidx ^ (c_row7 + it)) << 4);
-                    cp_async_16(kst + off, ks + it * ROWB, true);
-                    cp_async_16(vst + off, vs + it * ROWB, true);
+                    cp_async_16_stream(kst + off, ks + it * ROWB, true, stream_policy);
+                    cp_async_16_stream(vst + off, vs + it * ROWB, true, stream_policy);
                 }
             } else {
 #pragma unroll
@@ -173,8 +213,8 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
                     const bool valid = lam < hi && lam != n - 1;  // the new token is merged separately
                     const size_t ro = valid ? (size_t)phys_row(lam, i_cyc) * ROWB : 0;
                     const uint32_t off = c_lane_off + it * ROWB + ((c_cidx ^ (c_row7 + it)) << 4);
-                    cp_async_16(kst + off, reinterpret_cast<const unsigned char*>(Kc) + ro + c_cidx * 16, valid);
-                    cp_async_16(vst + off, reinterpret_cast<const unsigned char*>(Vc) + ro + c_cidx * 16, valid);
+                    cp_async_16_stream(kst + off, reinterpret_cast<const unsigned char*>(Kc) + ro + c_cidx * 16, valid, stream_policy);
+                    cp_async_16_stream(vst + off, reinterpret_cast<const unsigned char*>(Vc) + ro + c_cidx * 16, valid, stream_policy);
                 }
             }
         }
