@@ -22,7 +22,6 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
               T* __restrict__ out, ActiveMask active, int rows_cap) {
     constexpr int VEC = Elem<T>::kVec;
     constexpr int LPR = D / VEC;   // lanes per row
-    constexpr int RPW = 32 / LPR;  // rows per warp-wide load
     constexpr int CHUNKS = D * (int)sizeof(T) / 16;
     static_assert(LPR >= 1 && LPR <= 32 && (32 % LPR) == 0, "row must map onto a warp");
 
@@ -57,7 +56,7 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
     float* o_warp = o_part + G * D;            // [kDecodeWarps][G][D]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sub = lane % LPR, rsub = lane / LPR;
+    const int sub = lane % LPR;
 
     // ---- append (Algorithm 1: K <- K u {k}, V <- V u {v}).  This step itself reads the new token from
     //      k_in / v_in, so the slab row is not read back before the cluster barrier below.

@@ -281,6 +281,44 @@ def test_bitwise_reproducible(gpu):
         assert torch.equal(x, y)
 
 
+@pytest.mark.parametrize("shape", ["one_block_per_unit", "clusters"])
+def test_chained_launches_match_synchronised_launches(gpu, shape):
+    """The kernels of consecutive calls overlap at their edges (programmatic dependent launch; the decode kernel also
+    prefetches into L2 with a token count that may be one step old).  A stream of prefill chunks and decode steps
+    enqueued without any synchronisation must give the same bits as the same calls with a device synchronisation
+    after each one - on a batch large enough for one block per unit and on a small one that runs as clusters."""
+    import torch
+
+    if shape == "one_block_per_unit":
+        w = W.parity_slice(W.CONFIGS["cfg2"], layers=1, batch=20, n_heads=8, n_kv_heads=8, budget=160, chunk=64)
+    else:
+        w = W.parity_slice(W.CONFIGS["cfg4"], layers=1, batch=1, n_heads=8, n_kv_heads=2, budget=1024, chunk=256)
+    n_chunks, steps = w.budget // w.chunk + 3, 200
+    qs, ks, vs = W.tokens(w, 0, 0, n_chunks * w.chunk + steps)
+    dev = [torch.from_numpy(x).cuda().bfloat16() for x in (qs, ks, vs)]          # [T, B, H, d]
+    chunks = [[x[c * w.chunk:(c + 1) * w.chunk].transpose(0, 1).contiguous() for x in dev] for c in range(n_chunks)]
+    t0 = n_chunks * w.chunk
+    results = []
+    for sync in (False, True):
+        kv = gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, w.chunk)
+        outs_p = [torch.empty_like(chunks[0][0]) for _ in range(n_chunks)]
+        outs_d = torch.empty((steps, w.batch, w.n_heads, w.head_dim), dtype=torch.bfloat16, device="cuda")
+        torch.cuda.synchronize()
+        for c in range(n_chunks):
+            kv.prefill_chunk(*chunks[c], out=outs_p[c])
+            if sync:
+                torch.cuda.synchronize()
+        for s in range(steps):
+            kv.decode_step(dev[0][t0 + s], dev[1][t0 + s], dev[2][t0 + s], out=outs_d[s])
+            if sync:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        assert kv.stats()["device_error"] == 0
+        results.append((torch.stack(outs_p).clone(), outs_d.clone(), kv.scores().clone(), kv.retained_positions()[0].clone()))
+    for x, y in zip(*results):
+        assert torch.equal(x, y)
+
+
 @pytest.mark.parametrize("pinned", [True, False])
 def test_host_entry_points_match_device_entry_points(gpu, pinned):
     """Page-locked host tensors are read by the decode kernel directly; pageable ones go through staging copies."""
