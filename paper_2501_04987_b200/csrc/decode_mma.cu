@@ -65,6 +65,12 @@ __device__ inline uint32_t pack_bf16(float lo, float hi) {
 __device__ inline void l2_prefetch(const void* p, uint32_t bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
+// 2^x in one special-function instruction (about 2 ulp; arguments here are <= 0, results below 2^-126 flush to zero)
+__device__ inline float ex2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 // 2^(a-b) with the convention 2^(-inf - anything) = 0, so empty partials (max = -inf) never produce NaN
 __device__ inline float exp2_diff(float a, float b) { return a == -INFINITY ? 0.f : exp2f(a - b); }
 
@@ -453,7 +459,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     auto updated_score = [&](int j) {  // j: index among this CTA's rows; the appended token starts from S = 0
         float ps = 0.f;
 #pragma unroll
-        for (int h = 0; h < G; ++h) ps += exp2f(sl[h * rows_cap + j] - Mg[h]) * invL[h];
+        for (int h = 0; h < G; ++h) ps += ex2_fast(sl[h * rows_cap + j] - Mg[h]) * invL[h];
         return (j < ncached ? s_old[j] : 0.f) + ps * (1.0f / G);
     };
     if (nsplit > 1) {
@@ -479,7 +485,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     // ---- normalised probabilities; score update (Algorithm 1: S <- (S u {0}) + a, group mean)
     //      (a masked or padded logit is -inf and 2^-inf = 0, so exp2f needs no guard here: Mg is finite).  The two
     //      rows of the scope are left to the eviction below, which writes the survivor's score to its new row.
-#pragma unroll 4
+#pragma unroll 8
     for (int j = tid; j < ncached; j += NT) {
         const int ph = phys_row(lo + j, i_cyc);
         const float s_new = updated_score(j);
