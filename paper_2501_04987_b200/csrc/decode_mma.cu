@@ -72,7 +72,7 @@ __device__ inline float ex2_fast(float x) {
     return y;
 }
 // 2^(a-b) with the convention 2^(-inf - anything) = 0, so empty partials (max = -inf) never produce NaN
-__device__ inline float exp2_diff(float a, float b) { return a == -INFINITY ? 0.f : exp2f(a - b); }
+__device__ inline float exp2_diff(float a, float b) { return a == -INFINITY ? 0.f : ex2_fast(a - b); }
 
 constexpr int kBlk = 16;      // keys per pipeline stage
 constexpr int kPrefetchRows = 256;  // rows of K and of V a CTA asks L2 for before its stream-order wait (0 = none)
