@@ -531,32 +531,42 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     if (rank == 0 && tid == 0) cv.n_seen[unit] = N + 1;
 }
 
-size_t decode_mma_smem_bytes(int G, int D, int c, int split) {
-    const size_t ring = (size_t)kMmaWarps * kMmaStages * 2 * kBlk * D * 2;
+static size_t decode_mma_smem_bytes_ns(int G, int D, int c, int split, int stages) {
+    const size_t ring = (size_t)kMmaWarps * stages * 2 * kBlk * D * 2;
     return ring + sizeof(float) * ((size_t)G * mma_rows_cap(c, split) + (kMmaWarps + 1) * 2 * G + kMaxSplit * 2 * G +
                                    (size_t)split * G * D + (size_t)mma_rows_cap(c, split) + 2) + 4 * (size_t)D * 2 + 16 +
            16 + (size_t)(G + 2) * D * 2;
 }
 
-template <int D, int G>
-static cudaError_t launch_decode_mma_t(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
-                                       const ActiveMask& active, int split, cudaStream_t stream) {
-    auto kern = decode_mma_kernel<D, G, kMmaWarps, kMmaStages>;
-    const int rows_cap = mma_rows_cap(cv.c, split);
-    size_t smem = decode_mma_smem_bytes(G, D, cv.c, split);
-    static size_t smem_set[64] = {};  // per device: the opt-in limit only ever needs raising
+size_t decode_mma_smem_bytes(int G, int D, int c, int split) { return decode_mma_smem_bytes_ns(G, D, c, split, kMmaStages); }
+
+static int decode_sm_count() {
     static int sm_count[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     dev &= 63;
     if (sm_count[dev] == 0) cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+    return std::max(sm_count[dev], 1);
+}
+
+template <int D, int G, int NS>
+static cudaError_t launch_decode_mma_ns(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+                                        const ActiveMask& active, int split, cudaStream_t stream) {
+    auto kern = decode_mma_kernel<D, G, kMmaWarps, NS>;
+    const int rows_cap = mma_rows_cap(cv.c, split);
+    size_t smem = decode_mma_smem_bytes_ns(G, D, cv.c, split, NS);
+    static size_t smem_set[64] = {};  // per device: the opt-in limit only ever needs raising
+    int dev = 0;
+    cudaGetDevice(&dev);
+    dev &= 63;
+    const int sms = decode_sm_count();
     // When the whole grid fits at w = ceil(CTAs / SMs) thread blocks per SM, ask for just enough shared memory that
     // no SM can take more than w: the block scheduler otherwise packs some SMs to their limit and leaves others idle,
     // and the streaming rate of an SM does not grow in proportion to the blocks it hosts.
     {
         constexpr size_t kSmemPerSm = 227 * 1024, kReserved = 1024;  // per-block reservation of the runtime
         const long ncta = (long)split * cv.Hkv * cv.B;
-        const long w = (ncta + sm_count[dev] - 1) / std::max(sm_count[dev], 1);
+        const long w = (ncta + sms - 1) / sms;
         if (w >= 1 && (size_t)(w + 1) * (smem + kReserved) <= kSmemPerSm)
             smem = std::max(smem, kSmemPerSm / (size_t)(w + 1) + 1 - kReserved + 1024);
     }
@@ -582,6 +592,17 @@ static cudaError_t launch_decode_mma_t(const CacheView& cv, const void* q, const
     using T = __nv_bfloat16;
     return cudaLaunchKernelEx(&cfg, kern, cv, reinterpret_cast<const T*>(q), reinterpret_cast<const T*>(k),
                               reinterpret_cast<const T*>(v), reinterpret_cast<T*>(out), active, rows_cap);
+}
+
+// A thread block that has an SM to itself keeps three tiles per warp in flight instead of two (when they fit): one
+// block of four warps per SM is otherwise short of bytes in flight.
+template <int D, int G>
+static cudaError_t launch_decode_mma_t(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+                                       const ActiveMask& active, int split, cudaStream_t stream) {
+    const long ncta = (long)split * cv.Hkv * cv.B;
+    if (ncta <= decode_sm_count() && decode_mma_smem_bytes_ns(G, D, cv.c, split, 3) <= 227 * 1024)
+        return launch_decode_mma_ns<D, G, 3>(cv, q, k, v, out, active, split, stream);
+    return launch_decode_mma_ns<D, G, kMmaStages>(cv, q, k, v, out, active, split, stream);
 }
 
 template <int D>
