@@ -27,6 +27,10 @@
  *     n_kv_heads); the weight a cached token receives in a step is the mean
  *     over the query heads of its group (equal to Algorithm 1 when the group
  *     size is 1).
+ *   - Calls on one context execute in the order in which they were made when they are made on one stream;
+ *     the kernels of consecutive calls may overlap at their edges (programmatic dependent launch) and order
+ *     their own memory accesses.  Calls made on different streams, or from several host threads at once,
+ *     for the same context are the caller's to order.
  *   - Errors are returned, never thrown or trapped.  Argument and state errors
  *     are detected before anything is enqueued.  Asynchronous CUDA errors
  *     surface on a later call or in treekv_get_stats.
@@ -80,7 +84,7 @@ typedef struct {
  * Bytes of device workspace a context of this shape needs (0 if the shape is unsupported).
  * The workspace holds, per (sequence, KV head): K and V slabs of 2*budget + max_chunk rows, the score sums
  * S and the stream positions of the cached tokens; plus per-call scratch for chunked prefill (partial
- * column sums, staging rows for compaction) and staging buffers for the *_host entry points.
+ * column sums) and staging buffers for the *_host entry points.
  * max_chunk = 0 makes a decode-only context.
  */
 size_t treekv_workspace_bytes(int budget, int n_heads, int n_kv_heads, int head_dim, treekv_dtype dtype,

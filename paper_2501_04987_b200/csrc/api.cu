@@ -17,7 +17,7 @@ constexpr size_t kSmemLimit = 227 * 1024;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, S, pos, n_seen, stats, colsum, stage_K, stage_V, stage_S, stage_pos, st_q, st_k, st_v, st_out, total;
+    size_t K, V, S, pos, n_seen, stats, colsum, st_q, st_k, st_v, st_out, total;
     int R, QT, n_max;
 };
 
@@ -54,10 +54,6 @@ Layout make_layout(int budget, int n_heads, int n_kv_heads, int head_dim, treekv
     L.n_seen = take(units * 4);
     L.stats = take(sizeof(DevStats));
     L.colsum = take(units * L.QT * L.n_max * 4);
-    L.stage_K = take(units * max_chunk * head_dim * e);
-    L.stage_V = take(units * max_chunk * head_dim * e);
-    L.stage_S = take(units * max_chunk * 4);
-    L.stage_pos = take(units * max_chunk * 4);
     const size_t mc = max_chunk > 0 ? max_chunk : 1;
     L.st_q = take((size_t)batch * mc * n_heads * head_dim * e);
     L.st_k = take((size_t)batch * mc * n_kv_heads * head_dim * e);
@@ -148,10 +144,8 @@ treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_
     ctx->cv.c = budget; ctx->cv.R = L.R; ctx->cv.Hq = n_heads; ctx->cv.Hkv = n_kv_heads; ctx->cv.B = batch;
     ctx->cv.d = head_dim; ctx->cv.rule = TREEKV_RULE_SCORES;
     ctx->ps.colsum = reinterpret_cast<float*>(base + L.colsum);
-    ctx->ps.stage_K = base + L.stage_K;
-    ctx->ps.stage_V = base + L.stage_V;
-    ctx->ps.stage_S = reinterpret_cast<float*>(base + L.stage_S);
-    ctx->ps.stage_pos = reinterpret_cast<int32_t*>(base + L.stage_pos);
+    // (rows in flight during compaction stay in registers: the context has no staging rows; PrefillScratch's
+    //  staging pointers are only used by the entry point that brings its own scratch)
     ctx->ps.QT = L.QT; ctx->ps.n_max = L.n_max; ctx->ps.max_chunk = max_chunk;
     ctx->st_q = base + L.st_q; ctx->st_k = base + L.st_k; ctx->st_v = base + L.st_v; ctx->st_out = base + L.st_out;
     ctx->dt = dtype; ctx->max_chunk = max_chunk; ctx->G = n_heads / n_kv_heads;

@@ -1,7 +1,8 @@
 // treekv_prefill_chunk_static_scratch: the prefill-chunk call for callers that must not allocate.
 //
-// The regular call keeps its per-call scratch (partial column sums, staging rows used while compacting the
-// cache) in the workspace the caller sized and allocated at creation.  Some callers can only hand over the
+// The regular call keeps its per-call scratch (the partial column sums) in the workspace the caller sized and
+// allocated at creation.  This variant runs the kernels that need nothing but global scratch: CUDA-core attention
+// and the three-step score update / eviction, whose compaction goes through staging rows.  Some callers can only hand over the
 // tensors of the call itself: they run where device allocation is off the table (an inference server that
 // froze its memory pool at start-up, a plug-in living inside another framework's allocator, a latency-bound
 // loop that cannot afford cudaMalloc's implicit device-wide synchronisation), so whatever scratch a call needs
