@@ -135,7 +135,9 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
  * treekv_decode_step_host: when all four tensors are page-locked memory the GPU can address (cudaHostAlloc /
  * cudaHostRegister, 16-byte aligned), the step's kernel reads q, k, v from them and writes the output to them
  * directly across the bus - one launch, no staging copy; otherwise the inputs are copied to staging buffers
- * inside the workspace, the step runs, and the output is copied back.
+ * inside the workspace, the step runs, and the output is copied back.  host_q, host_k, host_v must hold their
+ * final values when the call is made (the CPU filled them): on the direct path the kernel may fetch them
+ * before earlier work in `stream` has finished.  The cache and host_out are touched only after it.
  * treekv_prefill_chunk_host always stages through the workspace.
  */
 treekv_status treekv_decode_step_host(treekv_ctx* ctx, const void* host_q, const void* host_k, const void* host_v,

@@ -188,8 +188,11 @@ treekv_status treekv_reset(treekv_ctx* ctx, void* stream) {
 
 void treekv_destroy(treekv_ctx* ctx) { delete ctx; }
 
-treekv_status treekv_decode_step(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v, void* dev_out,
-                                 const uint8_t* host_active, void* stream) {
+}  // extern "C"
+
+namespace {
+treekv_status decode_step_impl(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v, void* dev_out,
+                               const uint8_t* host_active, void* stream, int inputs_final) {
     if (!ctx || !dev_q || !dev_k || !dev_v || !dev_out) return TREEKV_ERR_INVALID_ARG;
     if (!aligned16(dev_q) || !aligned16(dev_k) || !aligned16(dev_v) || !aligned16(dev_out)) return TREEKV_ERR_INVALID_ARG;
     ActiveMask mask;
@@ -205,7 +208,7 @@ treekv_status treekv_decode_step(treekv_ctx* ctx, const void* dev_q, const void*
     if (n_active == 0) return TREEKV_OK;
     const cudaError_t e =
         use_mma_decode(ctx)
-            ? launch_decode_mma(ctx->cv, dev_q, dev_k, dev_v, dev_out, mask, pick_decode_split(ctx),
+            ? launch_decode_mma(ctx->cv, dev_q, dev_k, dev_v, dev_out, mask, pick_decode_split(ctx), inputs_final,
                                 static_cast<cudaStream_t>(stream))
             : launch_decode(ctx->cv, ctx->dt, dev_q, dev_k, dev_v, dev_out, mask, pick_decode_split(ctx),
                             static_cast<cudaStream_t>(stream));
@@ -218,6 +221,15 @@ treekv_status treekv_decode_step(treekv_ctx* ctx, const void* dev_q, const void*
         }
     }
     return TREEKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+treekv_status treekv_decode_step(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v, void* dev_out,
+                                 const uint8_t* host_active, void* stream) {
+    return decode_step_impl(ctx, dev_q, dev_k, dev_v, dev_out, host_active, stream, 0);
 }
 
 treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v, void* dev_out,
@@ -281,7 +293,7 @@ treekv_status treekv_decode_step_host(treekv_ctx* ctx, const void* host_q, const
         void* dv = dk ? device_alias(host_v) : nullptr;
         void* dout = dv ? device_alias(host_out) : nullptr;
         if (dout && aligned16(dq) && aligned16(dk) && aligned16(dv) && aligned16(dout))
-            return treekv_decode_step(ctx, dq, dk, dv, dout, host_active, stream);
+            return decode_step_impl(ctx, dq, dk, dv, dout, host_active, stream, 1);
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t qb = (size_t)ctx->cv.B * ctx->cv.Hq * ctx->cv.d * ctx->elem;

@@ -184,8 +184,9 @@ cudaError_t launch_decode(const CacheView& cv, treekv_dtype dt, const void* q, c
                           const ActiveMask& active, int split, cudaStream_t stream);
 
 size_t decode_mma_smem_bytes(int G, int D, int c, int split);
+// inputs_final: q, k, v held their final values before the launch (they may then be read ahead of the stream-order wait)
 cudaError_t launch_decode_mma(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
-                              const ActiveMask& active, int split, cudaStream_t stream);
+                              const ActiveMask& active, int split, int inputs_final, cudaStream_t stream);
 
 cudaError_t launch_init_state(const CacheView& cv, cudaStream_t stream);
 cudaError_t launch_retained_positions(const CacheView& cv, int32_t* pos_out, int32_t* count_out, cudaStream_t stream);

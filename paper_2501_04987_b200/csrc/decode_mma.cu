@@ -91,7 +91,7 @@ template <int D, int G, int NW, int NS>
 __global__ void __launch_bounds__(NW * 32)
 decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_in,
                   const __nv_bfloat16* __restrict__ v_in, __nv_bfloat16* __restrict__ out, ActiveMask active,
-                  int rows_cap) {
+                  int rows_cap, int inputs_final) {
     using T = __nv_bfloat16;
     constexpr int NT = NW * 32;
     constexpr int ROWB = D * 2;             // bytes per row
@@ -107,6 +107,41 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     // the same), and nothing below the wait is read before the previous kernel's writes are complete and visible.
     pdl_trigger();
     const int unit = b * cv.Hkv + kh;
+    const T* k_new = k_in + (size_t)unit * D;
+    const T* v_new = v_in + (size_t)unit * D;
+
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* ring = smem_raw;                                        // [NW][NS][STAGE]
+    float* sl = reinterpret_cast<float*>(ring + (size_t)NW * NS * STAGE);  // [G][rows_cap] logits (log2 units)
+    float* wstat = sl + (size_t)G * rows_cap;                              // [NW+1][2][G] per-warp (max, sum); slot NW = new token
+    float* gstat = wstat + (NW + 1) * 2 * G;                               // [nsplit][2][G] every CTA's (max, sum), pushed by its owner
+    float* o_all = gstat + kMaxSplit * 2 * G;                              // [nsplit][G][D] partial outputs, pushed into CTA 0 only
+    float* s_old = o_all + (size_t)nsplit * G * D;                         // [rows_cap] S of this CTA's rows, prefetched
+    unsigned char* pair_kv = reinterpret_cast<unsigned char*>(                   // [4][ROWB] K,V of the scope's two rows
+        (reinterpret_cast<uintptr_t>(s_old + rows_cap) + 15) & ~uintptr_t(15));
+    float* pair_s = reinterpret_cast<float*>(pair_kv + 4 * ROWB);          // [2] updated S of rows 2i, 2i+1 (split == 1)
+    unsigned char* tok = pair_kv + 4 * ROWB + 16;                          // [G+2][ROWB] this step's q heads, k, v
+    float* o_warp = reinterpret_cast<float*>(ring);                        // [NW][G][D], aliases the ring after the loop
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const float scale = kLog2e * rsqrtf((float)D);
+
+    // ---- this step's inputs go to shared memory once per CTA (warp 0, one commit group of their own): the q rows of
+    //      the group's heads and the new key and value rows.  Everything that needs them reads the copy, so q, k, v
+    //      are fetched once, early, whether they live in HBM or in page-locked host memory.  When the caller
+    //      guarantees that the inputs held their final values before the launch (host tensors filled by the CPU),
+    //      the fetch starts before the stream-order wait and its latency hides behind the previous kernel's tail.
+    auto stage_inputs = [&]() {
+        const T* qrow = q + ((size_t)b * cv.Hq + kh * G) * D;
+        for (int e = lane; e < (G + 2) * CPR; e += 32) {
+            const int r = e / CPR, cidx = e % CPR;
+            const T* srow = r < G ? qrow + (size_t)r * D : (r == G ? k_new : v_new);
+            cp_async_16(smem_u32(tok + r * ROWB + cidx * 16), reinterpret_cast<const unsigned char*>(srow) + cidx * 16, true);
+        }
+        cp_async_commit();
+    };
+    if (inputs_final && warp == 0 && active.test(b)) stage_inputs();
     // While the previous kernel of the stream drains, ask L2 for the first rows this CTA will stream.  This is a hint
     // and nothing more: the token count is read before the wait and may be one step old (the rows then shift by one),
     // no data reaches a register, and L2 is the point of coherence, so a line that the previous kernel still writes
@@ -150,41 +185,9 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     T* Vc = reinterpret_cast<T*>(cv.V) + (size_t)unit * cv.R * D;
     float* Sc = cv.S + (size_t)unit * cv.R;
     int32_t* Pc = cv.pos + (size_t)unit * cv.R;
-    const T* k_new = k_in + (size_t)unit * D;
-    const T* v_new = v_in + (size_t)unit * D;
     const int new_row = st.L + i_cyc;
 
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* ring = smem_raw;                                        // [NW][NS][STAGE]
-    float* sl = reinterpret_cast<float*>(ring + (size_t)NW * NS * STAGE);  // [G][rows_cap] logits (log2 units)
-    float* wstat = sl + (size_t)G * rows_cap;                              // [NW+1][2][G] per-warp (max, sum); slot NW = new token
-    float* gstat = wstat + (NW + 1) * 2 * G;                               // [nsplit][2][G] every CTA's (max, sum), pushed by its owner
-    float* o_all = gstat + kMaxSplit * 2 * G;                              // [nsplit][G][D] partial outputs, pushed into CTA 0 only
-    float* s_old = o_all + (size_t)nsplit * G * D;                         // [rows_cap] S of this CTA's rows, prefetched
-    unsigned char* pair_kv = reinterpret_cast<unsigned char*>(                   // [4][ROWB] K,V of the scope's two rows
-        (reinterpret_cast<uintptr_t>(s_old + rows_cap) + 15) & ~uintptr_t(15));
-    float* pair_s = reinterpret_cast<float*>(pair_kv + 4 * ROWB);          // [2] updated S of rows 2i, 2i+1 (split == 1)
-    unsigned char* tok = pair_kv + 4 * ROWB + 16;                          // [G+2][ROWB] this step's q heads, k, v
-    float* o_warp = reinterpret_cast<float*>(ring);                        // [NW][G][D], aliases the ring after the loop
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int g = lane >> 2, t = lane & 3;
-    const float scale = kLog2e * rsqrtf((float)D);
-
-    // ---- this step's inputs go to shared memory once per CTA (warp 0, one commit group of their own): the q rows of
-    //      the group's heads, and in the CTAs that use them the new key and value rows.  Everything that needs them
-    //      reads the copy, so q, k, v are fetched once, early, whether they live in HBM or in page-locked host memory.
-    const bool needs_kv = owns_new || rank == 0;
-    if (warp == 0) {
-        const T* qrow = q + ((size_t)b * cv.Hq + kh * G) * D;
-        for (int e = lane; e < (G + 2) * CPR; e += 32) {
-            const int r = e / CPR, cidx = e % CPR;
-            if (r >= G && !needs_kv) continue;
-            const T* srow = r < G ? qrow + (size_t)r * D : (r == G ? k_new : v_new);
-            cp_async_16(smem_u32(tok + r * ROWB + cidx * 16), reinterpret_cast<const unsigned char*>(srow) + cidx * 16, true);
-        }
-        cp_async_commit();
-    }
+    if (!inputs_final && warp == 0) stage_inputs();
 
     const uint32_t ring_w = smem_u32(ring) + warp * NS * STAGE;
     // Copy of one 16-row block: lane (half = lane / CPR... ) moves 16-byte chunk `cidx` of rows rsub*(16/RPI) + it.
@@ -551,7 +554,7 @@ static int decode_sm_count() {
 
 template <int D, int G, int NS>
 static cudaError_t launch_decode_mma_ns(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
-                                        const ActiveMask& active, int split, cudaStream_t stream) {
+                                        const ActiveMask& active, int split, int inputs_final, cudaStream_t stream) {
     auto kern = decode_mma_kernel<D, G, kMmaWarps, NS>;
     const int rows_cap = mma_rows_cap(cv.c, split);
     size_t smem = decode_mma_smem_bytes_ns(G, D, cv.c, split, NS);
@@ -591,36 +594,36 @@ static cudaError_t launch_decode_mma_ns(const CacheView& cv, const void* q, cons
     cfg.numAttrs = 2;
     using T = __nv_bfloat16;
     return cudaLaunchKernelEx(&cfg, kern, cv, reinterpret_cast<const T*>(q), reinterpret_cast<const T*>(k),
-                              reinterpret_cast<const T*>(v), reinterpret_cast<T*>(out), active, rows_cap);
+                              reinterpret_cast<const T*>(v), reinterpret_cast<T*>(out), active, rows_cap, inputs_final);
 }
 
 // A thread block that has an SM to itself keeps three tiles per warp in flight instead of two (when they fit): one
 // block of four warps per SM is otherwise short of bytes in flight.
 template <int D, int G>
 static cudaError_t launch_decode_mma_t(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
-                                       const ActiveMask& active, int split, cudaStream_t stream) {
+                                       const ActiveMask& active, int split, int inputs_final, cudaStream_t stream) {
     const long ncta = (long)split * cv.Hkv * cv.B;
     if (ncta <= decode_sm_count() && decode_mma_smem_bytes_ns(G, D, cv.c, split, 3) <= 227 * 1024)
-        return launch_decode_mma_ns<D, G, 3>(cv, q, k, v, out, active, split, stream);
-    return launch_decode_mma_ns<D, G, kMmaStages>(cv, q, k, v, out, active, split, stream);
+        return launch_decode_mma_ns<D, G, 3>(cv, q, k, v, out, active, split, inputs_final, stream);
+    return launch_decode_mma_ns<D, G, kMmaStages>(cv, q, k, v, out, active, split, inputs_final, stream);
 }
 
 template <int D>
 static cudaError_t launch_decode_mma_g(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
-                                       const ActiveMask& active, int split, cudaStream_t stream) {
+                                       const ActiveMask& active, int split, int inputs_final, cudaStream_t stream) {
     switch (cv.Hq / cv.Hkv) {
-        case 1: return launch_decode_mma_t<D, 1>(cv, q, k, v, out, active, split, stream);
-        case 2: return launch_decode_mma_t<D, 2>(cv, q, k, v, out, active, split, stream);
-        case 4: return launch_decode_mma_t<D, 4>(cv, q, k, v, out, active, split, stream);
-        case 8: return launch_decode_mma_t<D, 8>(cv, q, k, v, out, active, split, stream);
+        case 1: return launch_decode_mma_t<D, 1>(cv, q, k, v, out, active, split, inputs_final, stream);
+        case 2: return launch_decode_mma_t<D, 2>(cv, q, k, v, out, active, split, inputs_final, stream);
+        case 4: return launch_decode_mma_t<D, 4>(cv, q, k, v, out, active, split, inputs_final, stream);
+        case 8: return launch_decode_mma_t<D, 8>(cv, q, k, v, out, active, split, inputs_final, stream);
     }
     return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_decode_mma(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
-                              const ActiveMask& active, int split, cudaStream_t stream) {
-    if (cv.d == 64) return launch_decode_mma_g<64>(cv, q, k, v, out, active, split, stream);
-    if (cv.d == 128) return launch_decode_mma_g<128>(cv, q, k, v, out, active, split, stream);
+                              const ActiveMask& active, int split, int inputs_final, cudaStream_t stream) {
+    if (cv.d == 64) return launch_decode_mma_g<64>(cv, q, k, v, out, active, split, inputs_final, stream);
+    if (cv.d == 128) return launch_decode_mma_g<128>(cv, q, k, v, out, active, split, inputs_final, stream);
     return cudaErrorInvalidValue;
 }
 
