@@ -186,6 +186,23 @@ treekv_status treekv_retained_positions(treekv_ctx* ctx, int32_t* dev_pos, int32
  */
 treekv_status treekv_scores(treekv_ctx* ctx, float* dev_sbar, void* stream);
 
+/*
+ * State image: everything Algorithm 1 carries from one step to the next, in cache order, so that a context of the
+ * same shape can continue the stream elsewhere or later (the paper has no counterpart; idx and the counters C follow
+ * from the tokens seen and the stored positions).  Layout of the image, each part starting on a 256-byte boundary:
+ *   K   [batch][n_kv_heads][budget][head_dim]  dtype     V    the same
+ *   S   [batch][n_kv_heads][budget] float (sums, not averages)      pos  [batch][n_kv_heads][budget] int32
+ *   tokens seen [batch] int32
+ * Slots beyond a sequence's cache length are zero (pos: -1).
+ * treekv_export_state enqueues the copy and writes the host-side token counts to host_tokens_seen[batch] before
+ * returning; treekv_import_state replaces the context's state by the image (enqueued on `stream`) and takes the
+ * same counts back - they must be the ones exported with the image.
+ */
+size_t treekv_state_bytes(const treekv_ctx* ctx);
+treekv_status treekv_export_state(treekv_ctx* ctx, void* dev_image, int64_t* host_tokens_seen, void* stream);
+treekv_status treekv_import_state(treekv_ctx* ctx, const void* dev_image, const int64_t* host_tokens_seen,
+                                  void* stream);
+
 /* Counters and error words.  Synchronises `stream` to read the device-side counters. */
 treekv_status treekv_get_stats(treekv_ctx* ctx, treekv_stats* host_out, void* stream);
 

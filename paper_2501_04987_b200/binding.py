@@ -24,6 +24,7 @@ EXPORTS = [
     "treekv_decode_step_host", "treekv_prefill_chunk_host", "treekv_prefill_chunk_static_scratch", "treekv_retained_positions", "treekv_scores",
     "treekv_get_stats", "treekv_tokens_seen", "treekv_set_rule", "treekv_set_option", "treekv_reset",
     "treekv_destroy", "treekv_status_string", "treekv_version",
+    "treekv_state_bytes", "treekv_export_state", "treekv_import_state",
 ]
 
 
@@ -85,6 +86,12 @@ def _load():
     lib.treekv_status_string.argtypes = [i32]
     lib.treekv_version.restype = C.c_char_p
     lib.treekv_version.argtypes = []
+    lib.treekv_state_bytes.restype = C.c_size_t
+    lib.treekv_state_bytes.argtypes = [vp]
+    lib.treekv_export_state.restype = i32
+    lib.treekv_export_state.argtypes = [vp, vp, C.POINTER(C.c_int64), vp]
+    lib.treekv_import_state.restype = i32
+    lib.treekv_import_state.argtypes = [vp, vp, C.POINTER(C.c_int64), vp]
     return lib
 
 
@@ -175,6 +182,21 @@ def treekv_set_option(ctx, opt, value) -> int:
 
 def treekv_reset(ctx, stream=0) -> int:
     return lib.treekv_reset(ctx, stream)
+
+
+def treekv_state_bytes(ctx) -> int:
+    return lib.treekv_state_bytes(ctx)
+
+
+def treekv_export_state(ctx, dev_image, batch, stream=0):
+    seen = (C.c_int64 * batch)()
+    st = lib.treekv_export_state(ctx, dev_image, seen, stream)
+    return st, list(seen)
+
+
+def treekv_import_state(ctx, dev_image, tokens_seen, stream=0) -> int:
+    seen = (C.c_int64 * len(tokens_seen))(*[int(x) for x in tokens_seen])
+    return lib.treekv_import_state(ctx, dev_image, seen, stream)
 
 
 def treekv_destroy(ctx) -> None:
@@ -289,3 +311,19 @@ class TreeKV:
 
     def reset(self):
         _check(treekv_reset(self._h, self._stream()), "treekv_reset")
+
+    def export_state(self):
+        """(image, tokens_seen): a uint8 CUDA tensor holding the state image and the per-sequence token counts."""
+        n = treekv_state_bytes(self._h)
+        image = self.torch.empty(n + 256, dtype=self.torch.uint8, device=self.device)
+        off = (-image.data_ptr()) % 256
+        image = image[off:off + n]
+        st, seen = treekv_export_state(self._h, image.data_ptr(), self.batch, self._stream())
+        _check(st, "treekv_export_state")
+        return image, seen
+
+    def import_state(self, image, tokens_seen):
+        if not (image.is_cuda and image.dtype == self.torch.uint8 and image.numel() >= treekv_state_bytes(self._h)
+                and image.data_ptr() % 16 == 0):
+            raise ValueError("expected a uint8 CUDA tensor of at least treekv_state_bytes, 16-byte aligned")
+        _check(treekv_import_state(self._h, image.data_ptr(), tokens_seen, self._stream()), "treekv_import_state")

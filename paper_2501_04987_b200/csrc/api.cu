@@ -345,6 +345,51 @@ treekv_status treekv_scores(treekv_ctx* ctx, float* dev_sbar, void* stream) {
     return TREEKV_OK;
 }
 
+static size_t state_image_layout(const treekv_ctx* ctx, void* base, StateImage* img) {
+    const size_t units = (size_t)ctx->cv.B * ctx->cv.Hkv, slots = units * ctx->cv.c;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    const size_t oK = take(slots * ctx->cv.d * ctx->elem), oV = take(slots * ctx->cv.d * ctx->elem);
+    const size_t oS = take(slots * 4), oP = take(slots * 4), oN = take((size_t)ctx->cv.B * 4);
+    if (img) {
+        char* p = static_cast<char*>(base);
+        img->K = p + oK; img->V = p + oV;
+        img->S = reinterpret_cast<float*>(p + oS); img->pos = reinterpret_cast<int32_t*>(p + oP);
+        img->seen = reinterpret_cast<int32_t*>(p + oN);
+    }
+    return off;
+}
+
+size_t treekv_state_bytes(const treekv_ctx* ctx) { return ctx ? state_image_layout(ctx, nullptr, nullptr) : 0; }
+
+treekv_status treekv_export_state(treekv_ctx* ctx, void* dev_image, int64_t* host_tokens_seen, void* stream) {
+    if (!ctx || !dev_image || !host_tokens_seen || !aligned16(dev_image)) return TREEKV_ERR_INVALID_ARG;
+    StateImage img;
+    state_image_layout(ctx, dev_image, &img);
+    const cudaError_t e = launch_export_state(ctx->cv, ctx->dt, img, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    for (int b = 0; b < ctx->cv.B; ++b) host_tokens_seen[b] = ctx->n_seen[b];
+    return TREEKV_OK;
+}
+
+treekv_status treekv_import_state(treekv_ctx* ctx, const void* dev_image, const int64_t* host_tokens_seen, void* stream) {
+    if (!ctx || !dev_image || !host_tokens_seen || !aligned16(dev_image)) return TREEKV_ERR_INVALID_ARG;
+    for (int b = 0; b < ctx->cv.B; ++b)
+        if (host_tokens_seen[b] < 0 || host_tokens_seen[b] >= 0x7fffffff - 1) return TREEKV_ERR_INVALID_ARG;
+    StateImage img;
+    state_image_layout(ctx, const_cast<void*>(dev_image), &img);
+    const cudaError_t e = launch_import_state(ctx->cv, ctx->dt, img, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    ctx->evictions = 0;
+    for (int b = 0; b < ctx->cv.B; ++b) {
+        ctx->n_seen[b] = host_tokens_seen[b];
+        if (host_tokens_seen[b] > ctx->cv.c) ctx->evictions += (uint64_t)(host_tokens_seen[b] - ctx->cv.c);
+    }
+    return TREEKV_OK;
+}
+
 treekv_status treekv_get_stats(treekv_ctx* ctx, treekv_stats* host_out, void* stream) {
     if (!ctx || !host_out) return TREEKV_ERR_INVALID_ARG;
     DevStats ds;

@@ -189,6 +189,16 @@ cudaError_t launch_decode_mma(const CacheView& cv, const void* q, const void* k,
                               const ActiveMask& active, int split, int inputs_final, cudaStream_t stream);
 
 cudaError_t launch_init_state(const CacheView& cv, cudaStream_t stream);
+// state image in cache order (see treekv_export_state): pointers into the caller's buffer
+struct StateImage {
+    void* K;
+    void* V;
+    float* S;
+    int32_t* pos;
+    int32_t* seen;  // [B]
+};
+cudaError_t launch_export_state(const CacheView& cv, treekv_dtype dt, const StateImage& img, cudaStream_t stream);
+cudaError_t launch_import_state(const CacheView& cv, treekv_dtype dt, const StateImage& img, cudaStream_t stream);
 cudaError_t launch_retained_positions(const CacheView& cv, int32_t* pos_out, int32_t* count_out, cudaStream_t stream);
 cudaError_t launch_scores(const CacheView& cv, float* sbar_out, cudaStream_t stream);
 cudaError_t launch_chunk_append(const CacheView& cv, treekv_dtype dt, const void* k, const void* v, const ChunkLens& lens,

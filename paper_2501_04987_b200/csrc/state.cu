@@ -56,6 +56,55 @@ cudaError_t launch_scores(const CacheView& cv, float* sbar_out, cudaStream_t str
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// State image: the live rows of every unit in cache order.  One warp per (unit, slot).
+template <typename T, bool kImport>
+__global__ void state_image_kernel(CacheView cv, StateImage img) {
+    const int unit = blockIdx.y;
+    const int b = unit / cv.Hkv;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lam = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (lam >= cv.c) return;
+    const int N = kImport ? img.seen[b] : cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv.c);
+    const int chunks = cv.d * (int)sizeof(T) / 16;
+    const size_t slot = (size_t)unit * cv.c + lam;
+    uint4* ki = reinterpret_cast<uint4*>(reinterpret_cast<T*>(img.K) + slot * cv.d);
+    uint4* vi = reinterpret_cast<uint4*>(reinterpret_cast<T*>(img.V) + slot * cv.d);
+    if (lam < st.L) {
+        const size_t row = (size_t)unit * cv.R + phys_row(lam, st.i);
+        uint4* kc = reinterpret_cast<uint4*>(reinterpret_cast<T*>(cv.K) + row * cv.d);
+        uint4* vc = reinterpret_cast<uint4*>(reinterpret_cast<T*>(cv.V) + row * cv.d);
+        if (kImport) {
+            for (int e = lane; e < chunks; e += 32) { kc[e] = ki[e]; vc[e] = vi[e]; }
+            if (lane == 0) { cv.S[row] = img.S[slot]; cv.pos[row] = img.pos[slot]; }
+        } else {
+            for (int e = lane; e < chunks; e += 32) { ki[e] = kc[e]; vi[e] = vc[e]; }
+            if (lane == 0) { img.S[slot] = cv.S[row]; img.pos[slot] = cv.pos[row]; }
+        }
+    } else if (!kImport) {
+        for (int e = lane; e < chunks; e += 32) { ki[e] = make_uint4(0, 0, 0, 0); vi[e] = make_uint4(0, 0, 0, 0); }
+        if (lane == 0) { img.S[slot] = 0.f; img.pos[slot] = -1; }
+    }
+    if (lam == 0 && lane == 0) {
+        if (kImport) cv.n_seen[unit] = N;
+        else if (unit % cv.Hkv == 0) img.seen[b] = N;
+    }
+}
+template <bool kImport>
+static cudaError_t launch_state_image(const CacheView& cv, treekv_dtype dt, const StateImage& img, cudaStream_t stream) {
+    dim3 grid((cv.c + 7) / 8, cv.B * cv.Hkv);
+    if (dt == TREEKV_F32) state_image_kernel<float, kImport><<<grid, 256, 0, stream>>>(cv, img);
+    else state_image_kernel<__nv_bfloat16, kImport><<<grid, 256, 0, stream>>>(cv, img);
+    return cudaGetLastError();
+}
+cudaError_t launch_export_state(const CacheView& cv, treekv_dtype dt, const StateImage& img, cudaStream_t stream) {
+    return launch_state_image<false>(cv, dt, img, stream);
+}
+cudaError_t launch_import_state(const CacheView& cv, treekv_dtype dt, const StateImage& img, cudaStream_t stream) {
+    return launch_state_image<true>(cv, dt, img, stream);
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Chunk append: chunk token t of sequence b goes to physical row L + i + t of every KV head's slab.
 // One warp per (token, unit); k,v are [B][chunk_stride][Hkv][d].
 template <typename T>
