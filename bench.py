@@ -57,10 +57,10 @@ def measured_peaks():
 # profiles/, valid for the named workload's per-layer shape and only while the kernel's sources are the ones that
 # were profiled: a changed source file makes the entry stale and the reported traffic null.
 NCU_TRAFFIC = {
-    "decode_mma_kernel": {"workload": "cfg2", "bytes_per_launch": 140.86e6, "sources": ["decode_mma.cu", "common.cuh"],
-                          "sha1": "9bea501157962fd2b13bccebc1fd521bd138ded7", "profile": "profiles/decode_mma_cfg2_2layers.md"},
-    "prefill_tc2_kernel": {"workload": "cfg5", "bytes_per_launch": 150.11e6, "sources": ["prefill_tc2.cu", "tma.cuh", "common.cuh"],
-                           "sha1": "d768b8273558fc7bfe853816dc25c3917002369e", "profile": "profiles/prefill_tc2_cfg5_1layer.md"},
+    "decode_mma_kernel": {"workload": "cfg2", "bytes_per_launch": 141.16e6, "sources": ["decode_mma.cu", "common.cuh"],
+                          "sha1": "d588789f54b63eefdcc6510a26c23f77377158e2", "profile": "profiles/decode_mma_cfg2_2layers.md"},
+    "prefill_tc2_kernel": {"workload": "cfg5", "bytes_per_launch": 149.87e6, "sources": ["prefill_tc2.cu", "tma.cuh", "common.cuh"],
+                           "sha1": "b9140f2051a2ccaeac53170c2d4270cdd2053141", "profile": "profiles/prefill_tc2_cfg5_1layer.md"},
 }
 
 
