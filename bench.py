@@ -4,8 +4,9 @@
 
 Headline (value): decode steps/s on the Llama-2-7B-shaped configuration (32 layers, batch 8, 32 heads, d=128,
 bf16, budget 1024) with every cache full, one step = all 32 layers in order, inputs resident in HBM.
-`e2e`: the same step through the *_host entry points: host->device copies of q,k,v and the device->host copy
-of the output are inside the timed region, every step.
+`e2e`: the same step through treekv_decode_step_host with page-locked host tensors: q, k, v cross the bus to the
+GPU and the output crosses it back inside the timed region, every layer of every step (the kernel reads and writes
+the host tensors itself; h2d / d2h bytes are counted from the tensors).
 `prefill`: chunked-prefill tokens/s (through all layers) on the Llama-3-8B-shaped prefill configuration (batch 4,
 chunks of 1024 to budget 4096), steady state with full chunks, with its own tensor roofline entry.
 `decode_alt` / `prefill_alt`: the same two measurements on the other decode (Llama-3-8B GQA, batch 32, budget 2048)
