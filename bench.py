@@ -251,8 +251,9 @@ def run_reference(args, w):
         "metric": "treekv_decode_steps_per_s", "value": val, "unit": "steps/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1000.0 / val, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
-        "config": {"workload": w.name, "layers": w.layers, "batch": w.batch, "n_heads": w.n_heads,
-                   "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "budget": w.budget},
+        "config": {"workload": w.name, "layers": w.layers, "batch_per_gpu": w.batch, "n_heads": w.n_heads,
+                   "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "budget": w.budget,
+                   "parallelism": "oracle on the host cores of rank 0"},
         "cpu_baseline": {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": val, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
