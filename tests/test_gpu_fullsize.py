@@ -196,14 +196,15 @@ def test_cfg5_full_layer_ragged_prefill(gpu):
     print("cfg5 full layer: max sampled out err %.3g" % err)
 
 
-def test_large_budget_decode_through_eight_block_clusters(gpu):
-    """A budget of 16384 with one sequence and two KV heads (g = 4): the decode kernel runs as clusters of eight
-    blocks with 2049 rows each, close to the largest shared-memory footprint the library accepts.  The cache is
-    filled token by token, then steps across the first evictions are checked on every head against fp64 softmax
-    attention over the retained set, with the cache invariants."""
+@pytest.mark.parametrize("c,Hq,Hkv", [(16384, 8, 2), (65536, 1, 1)])
+def test_large_budget_decode_through_eight_block_clusters(gpu, c, Hq, Hkv):
+    """Budgets of 16384 (one sequence, two KV heads, g = 4) and of 65536, the largest the library accepts (one head):
+    the decode kernel runs as clusters of eight blocks with 2049 / 8193 rows each, close to the largest shared-memory
+    footprint.  The cache is filled token by token, then steps across the first evictions are checked on every head
+    against fp64 softmax attention over the retained set, with the cache invariants."""
     import torch
 
-    c, Hq, Hkv, d, B = 16384, 8, 2, 128, 1
+    d, B = 128, 1
     g = Hq // Hkv
     kv = gpu.TreeKV(c, Hq, Hkv, d, "bf16", B, 0)
     gen = torch.Generator(device="cuda"); gen.manual_seed(20250111)
@@ -234,4 +235,4 @@ def test_large_budget_decode_through_eight_block_clusters(gpu):
     _check_invariants(kv, [steps])
     st = kv.stats()
     assert st["device_error"] == 0 and st["evictions"] == steps - c
-    print("c=16384 decode: max out err %.3g" % max_err)
+    print("c=%d decode: max out err %.3g" % (c, max_err))
