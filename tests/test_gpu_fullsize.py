@@ -110,7 +110,7 @@ def test_cfg2_full_layer_decode_sampled_units(gpu):
     print("cfg2 full layer: max out err %.3g, near-ties %d, flips %d" % (max_err, near, flips))
 
 
-def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6):
+def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_chunk=None):
     import torch
 
     B, Hq, Hkv, d, m, c = w.batch, w.n_heads, w.n_kv_heads, w.head_dim, w.chunk, w.budget
@@ -119,15 +119,18 @@ def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6):
     gen = torch.Generator(device="cuda"); gen.manual_seed(w.seed)
     rs = np.random.default_rng(w.seed)
     seq_scale = torch.from_numpy(W.seq_key_scales(w)).cuda() if w.key_scale else None
-    sampled = [(0, 0), (B - 1, Hkv - 1), (B // 2, Hkv // 2)]
+    sampled = sorted(set([(0, 0), (B - 1, Hkv - 1), (B // 2, Hkv // 2)]))
     hist_k = {u: np.zeros((0, d)) for u in sampled}   # full key / value streams of the sampled units (fp64)
     hist_v = {u: np.zeros((0, d)) for u in sampled}
     seen = [0] * B
     lens_total = list(lens_total)
-    n_calls = (max(lens_total) + m - 1) // m
+    # call boundaries: chunks of m, optionally after a shorter first chunk
+    bounds = [0] + ([first_chunk] if first_chunk else [])
+    while bounds[-1] < max(lens_total):
+        bounds.append(bounds[-1] + m)
     max_err = 0.0
-    for call in range(n_calls):
-        lens = [max(0, min(m, L - call * m)) for L in lens_total]
+    for call in range(len(bounds) - 1):
+        lens = [max(0, min(bounds[call + 1], L) - bounds[call]) for L in lens_total]
         q = _draw(torch, gen, (B, m, Hq, d))
         k = _draw(torch, gen, (B, m, Hkv, d), seq_scale=seq_scale)
         v = _draw(torch, gen, (B, m, Hkv, d))
@@ -236,3 +239,30 @@ def test_large_budget_decode_through_eight_block_clusters(gpu, c, Hq, Hkv):
     st = kv.stats()
     assert st["device_error"] == 0 and st["evictions"] == steps - c
     print("c=%d decode: max out err %.3g" % (c, max_err))
+
+
+@pytest.mark.parametrize("path", [1, 2, 3])
+def test_maximum_chunk_with_many_wraps(gpu, path):
+    """The longest chunk the library accepts (8192 tokens) into a budget of 1024: one call evicts through eight wraps of
+    the idx cycle, with a rebase of the not yet paired rows after each.  Run with the CUDA-core kernel and with both
+    tensor-core kernels; sampled output rows against fp64 attention over [retained before the call | chunk so far]."""
+    import torch
+
+    w = W.parity_slice(W.CONFIGS["cfg5"], layers=1, batch=1, n_heads=2, n_kv_heads=1, budget=1024, chunk=8192, key_scale=False)
+    kv_holder = {}
+
+    class _Forced:
+        """binding.TreeKV with the prefill path fixed at creation."""
+        def __getattr__(self, name):
+            return getattr(gpu, name)
+
+        def TreeKV(self, *a, **k):
+            kv = gpu.TreeKV(*a, **k)
+            kv.set_option(gpu.OPT_PREFILL_PATH, path)
+            kv_holder["kv"] = kv
+            return kv
+
+    err = _prefill_fullsize(_Forced(), w, [700 + 2 * 8192], decode_steps=6, n_sample_rows=5, first_chunk=700)
+    st = kv_holder["kv"].stats()
+    assert st["evictions"] == 700 + 2 * 8192 + 6 - 1024 and st["device_error"] == 0
+    print("m=8192 into c=1024, path %d: max sampled out err %.3g" % (path, err))
