@@ -158,6 +158,27 @@ def test_shapes_and_group_sizes(gpu, dtype, d, hq, hkv):
     _run_decode(kv, orc, w, 0, 60, rep, starts=[40, 33, 16])
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_maximum_batch_with_changing_active_sets(gpu, dtype):
+    """1024 sequences (the largest batch), a different random subset of them stepping each time: sequences drift apart,
+    so every step mixes units that are still filling with units at different points of their eviction cycle."""
+    w = W.parity_slice(W.CONFIGS["cfg1"], dtype=dtype, head_dim=64, n_heads=2, n_kv_heads=2, batch=1024, budget=12, chunk=0,
+                       n_outliers=2)
+    kv, orc = _pair(gpu, w)
+    rep = Report()
+    rs = np.random.default_rng(7)
+    seen = np.zeros(w.batch, np.int64)
+    for step in range(36):
+        active = rs.random(w.batch) < (0.9 if step < 6 else 0.6)
+        active[step % w.batch] = True
+        q, k, v = W.tokens_at(w, 0, seen, 1)
+        step_decode(kv, orc, q[0], k[0], v[0], w.dtype, rep, active=active.astype(np.uint8), check_scores=(step % 6 == 5))
+        seen += active
+    assert [kv.tokens_seen(b) for b in (0, 511, 1023)] == [int(seen[b]) for b in (0, 511, 1023)]
+    assert kv.stats()["evictions"] == int(np.maximum(seen - w.budget, 0).sum())
+    print("batch 1024", dtype, rep)
+
+
 @pytest.mark.parametrize("c", [2, 3, 5])
 def test_tiny_budgets(gpu, c):
     w = W.parity_slice(W.CONFIGS["cfg1"], budget=c, chunk=7, batch=2)
