@@ -62,6 +62,8 @@ NCU_TRAFFIC = {
                           "sha1": "d588789f54b63eefdcc6510a26c23f77377158e2", "profile": "profiles/decode_mma_cfg2_2layers.md"},
     "prefill_tc2_kernel": {"workload": "cfg5", "bytes_per_launch": 149.87e6, "sources": ["prefill_tc2.cu", "tma.cuh", "common.cuh"],
                            "sha1": "b9140f2051a2ccaeac53170c2d4270cdd2053141", "profile": "profiles/prefill_tc2_cfg5_1layer.md"},
+    "prefill_tc_kernel": {"workload": "cfg3", "bytes_per_launch": 46.60e6, "sources": ["prefill_tc.cu", "tma.cuh", "common.cuh"],
+                          "sha1": "026cc9d2ef69ada63b6fe549d1ae7c7e09da95fd", "profile": "profiles/prefill_tc_cfg3_2layers.md"},
 }
 
 
