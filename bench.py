@@ -503,7 +503,9 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, world, rank, barrier, max
     return {"metric": "treekv_prefill_tokens_per_s", "value": tok_s, "unit": "tokens/s", "chunks": n_chunks,
             "ms_per_chunk_all_layers": ms / n_chunks, "gpu_launches": int(launches),
             "config": {"workload": pw.name, "layers": pw.layers, "batch_per_gpu": pw.batch, "n_heads": pw.n_heads,
-                       "n_kv_heads": pw.n_kv_heads, "head_dim": pw.head_dim, "budget": c, "chunk": m},
+                       "n_kv_heads": pw.n_kv_heads, "head_dim": pw.head_dim, "budget": c, "chunk": m,
+                       "l2": "no flush: a chunk reads %.0f MB of K/V per layer and a layer is revisited %d layers later (126 MB L2)"
+                             % (2 * pw.batch * pw.n_kv_heads * (c + m) * pw.head_dim * 2 / 1e6, pw.layers)},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                          "frac": achieved / peak, "traffic": measured_traffic(kernel, pw.name),
                          "kernel": kernel, "peak_source": peaks["source"] + " (sustained)",
