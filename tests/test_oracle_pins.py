@@ -494,19 +494,90 @@ def test_ragged_batch_and_inactive_sequences(oracle_lib):
         assert ob.idx(b) == os_[b].idx(0)
 
 
+def _adversarial_hint(before, after, c):
+    """The retained set that keeps the token a decision dropped and drops the one it kept, everything else alike:
+    `before` are the c+1 positions ahead of the eviction, `after` the c positions it left."""
+    dropped = [p for p in before if p not in set(after)]
+    assert len(dropped) == 1
+    j = list(before).index(dropped[0])
+    return dropped[0], j
+
+
 def test_near_tie_hint_is_only_used_at_near_ties(oracle_lib):
-    c, d, T = 4, 4, 9
-    q, k, v = _stream(24, T, 1, 1, d, peaked=True)
-    a = Oracle(c, 1, 1, d, 1)
-    b = Oracle(c, 1, 1, d, 1)
+    """The near-tie hint (a test device, not part of Algorithm 1) may only change a decision whose relative score gap
+    is below the tolerance.  A twin oracle plays Algorithm 1 unaided; the oracle under test gets, at every eviction,
+    the hint that asks for the OPPOSITE of the twin's decision in every unit (it contains the loser of the scope
+    and not the winner).  With the working tolerance of 1e-4 and well-separated scores nothing may flip."""
+    c, d, T, B, Hq, Hkv = 6, 4, 42, 2, 4, 2
+    q, k, v = _stream(24, T, Hq, Hkv, d, B, peaked=True)
+    a = Oracle(c, Hq, Hkv, d, B)
+    b = Oracle(c, Hq, Hkv, d, B)
+    decisions = 0
     for t in range(T):
-        a.decode_step(q[t], k[t], v[t])
+        a.decode_attend(q[t], k[t], v[t])
         b.decode_attend(q[t], k[t], v[t])
-        # a hint that asks for the opposite of every decision must be ignored when the gap is large
-        hint = np.full((1, 1, c), -1, np.int32); cnt = np.zeros((1, 1), np.int32)
+        before = {(s, kh): list(a.positions(s, kh)) for s in range(B) for kh in range(Hkv)}
+        idx = a.idx(0)
+        a.evict()
+        if t < c:
+            b.evict()
+            continue
+        hint = np.full((B, Hkv, c), -1, np.int32)
+        cnt = np.full((B, Hkv), c, np.int32)
+        for (s, kh), bef in before.items():
+            aft = list(a.positions(s, kh))
+            lost, j = _adversarial_hint(bef, aft, c)
+            assert j in (idx - 1, idx)                               # the dropped slot is a member of the scope
+            kept = bef[idx - 1] if j == idx else bef[idx]
+            h = sorted((set(bef) - {kept}))                          # keeps the loser, drops the winner
+            assert len(h) == c and lost in h and kept not in h
+            hint[s, kh] = h
         b.evict(hint, cnt, near_tie_tol=1e-4)
-        assert b.last_hint_flips == 0
-        assert list(a.positions(0, 0)) == list(b.positions(0, 0))
+        assert b.last_min_gap >= 1e-4, "the stream was meant to have well-separated scores"
+        assert b.last_near_ties == 0 and b.last_hint_flips == 0
+        decisions += B * Hkv
+        for s in range(B):
+            for kh in range(Hkv):
+                assert list(a.positions(s, kh)) == list(b.positions(s, kh)), (t, s, kh)
+    assert decisions == (T - c) * B * Hkv and b.total_hint_flips == 0
+
+
+def test_near_tie_hint_decides_real_near_ties(oracle_lib):
+    """The other direction: with q = 0 every weight is 1/len, so tokens that arrived after the cache filled have
+    equal averaged scores up to rounding (relative gap ~1e-16).  There the adversarial hint must win, every time
+    the two members of the scope both arrived after the fill."""
+    c, d, T = 4, 4, 30
+    r = _rng(25)
+    k = r.standard_normal((T, 1, 1, d)); v = r.standard_normal((T, 1, 1, d)); q = np.zeros((T, 1, 1, d))
+    b = Oracle(c, 1, 1, d, 1)
+    flips = 0
+    for t in range(T):
+        b.decode_attend(q[t], k[t], v[t])
+        if t < c:
+            b.evict()
+            continue
+        bef = list(b.positions(0, 0))
+        idx = b.idx(0)
+        l, rr = bef[idx - 1], bef[idx]
+        # what Algorithm 1 does unaided on this state
+        pos, S, C, sb = b.unit(0, 0)
+        unaided_evicts_right = sb[idx - 1] > sb[idx]
+        kept = l if unaided_evicts_right else rr
+        h = sorted(set(bef) - {kept})
+        gap = abs(sb[idx - 1] - sb[idx]) / max(abs(sb[idx - 1]), abs(sb[idx]))
+        b.evict(np.array([[h]], np.int32), np.array([[c]], np.int32), near_tie_tol=1e-4)
+        if gap < 1e-4:
+            assert b.last_near_ties == 1 and b.last_hint_flips == 1
+            assert list(b.positions(0, 0)) == h
+            flips += 1
+        else:
+            assert b.last_hint_flips == 0 and kept in list(b.positions(0, 0))
+    assert flips >= 5
+
+
+def test_near_tie_hint_with_absurd_tolerance(oracle_lib):
+    c, d = 4, 4
+    q, k, v = _stream(24, c + 1, 1, 1, d, peaked=True)
     # with an absurdly large tolerance every decision is a "near-tie" and the hint decides
     b2 = Oracle(c, 1, 1, d, 1)
     for t in range(c + 1):
