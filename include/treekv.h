@@ -150,10 +150,11 @@ treekv_status treekv_prefill_chunk_host(treekv_ctx* ctx, const void* host_q, con
  * treekv_prefill_chunk for callers that cannot allocate device memory.  (The paper has no counterpart: this
  * is a deployment variant of the call above, not a different computation.)
  *
- * Same arguments, same effect on the cache and the same dev_out as treekv_prefill_chunk, but none of the
- * call's scratch (partial column sums, rows staged during compaction) is taken from the workspace: it lives
- * in a fixed 16 MiB area that is part of the library image on every GPU that has loaded the library, from
- * load until the process exits.  It is meant for code that may not call cudaMalloc at the point where it
+ * Same arguments and the same result as treekv_prefill_chunk within the library's tolerances (it always runs the
+ * CUDA-core attention kernel, so against a context that runs the tensor-core kernel outputs and scores agree to
+ * rounding, and against one forced to the CUDA-core kernel bit for bit), but none of the call's scratch (partial
+ * column sums, rows staged during compaction) is taken from the workspace: it lives in a fixed 16 MiB area that is
+ * part of the library image and stays on every GPU that has used this entry point until the process exits.  It is meant for code that may not call cudaMalloc at the point where it
  * runs - a server that has frozen its memory pool, a plug-in inside another framework's allocator, a loop
  * that cannot take cudaMalloc's device-wide synchronisation - and so cannot size scratch per call.  The
  * entry point itself calls no allocating routine.
@@ -162,7 +163,12 @@ treekv_status treekv_prefill_chunk_host(treekv_ctx* ctx, const void* host_q, con
  *     bytes (each of the five parts rounded up to 256); beyond 16 MiB it returns TREEKV_ERR_UNSUPPORTED and
  *     enqueues nothing.
  *   - The first call on a device looks up the area's device address (once per device, with that device
- *     current); make that first call outside any stream capture.
+ *     current).  That lookup is also the moment the CUDA runtime loads the part of the library that holds the
+ *     area, i.e. when the GPU commits the 16 MiB; it may synchronise the device and can fail when no memory is
+ *     left.  So make one warm-up call per device at start-up - before a memory pool is frozen and outside any
+ *     stream capture; every later call only reads the cached address.
+ *   - The device that is current at the call must be the one the context was created on (where its workspace
+ *     lives); otherwise TREEKV_ERR_BAD_STATE.
  *   - Every context of the process shares the one area of its GPU, and the area keeps whatever the last call
  *     left.  A call never reads a slot it has not itself written first, so nothing needs clearing between
  *     calls; but two calls that overlap on the GPU (issued on different streams, whether for the same context
@@ -203,8 +209,20 @@ treekv_status treekv_export_state(treekv_ctx* ctx, void* dev_image, int64_t* hos
 treekv_status treekv_import_state(treekv_ctx* ctx, const void* dev_image, const int64_t* host_tokens_seen,
                                   void* stream);
 
-/* Counters and error words.  Synchronises `stream` to read the device-side counters. */
+/* Counters and error words.  Synchronises `stream` to read the device-side counters.  *host_out is filled
+ * whenever the read itself succeeded; the return value is TREEKV_ERR_TIMEOUT when device_error is non-zero, i.e.
+ * when a kernel's bounded wait gave up (bits: 4 TMA producer, 8 MMA issuer, 16 softmax / epilogue warps of the
+ * tensor-core prefill kernels, 32 misaligned shared memory, 64 the self-test below).  treekv_reset clears it. */
 treekv_status treekv_get_stats(treekv_ctx* ctx, treekv_stats* host_out, void* stream);
+
+/*
+ * Self-test of the give-up path (the paper has no counterpart).  Enqueues a kernel of one thread block that waits,
+ * for at most `attempts` polls (1..4096), on a barrier that nothing signals - with the helper every bounded wait of
+ * the library uses - and then records the give-up in the context's device error word, as a real kernel would.  The
+ * cache is not touched.  Afterwards treekv_get_stats returns TREEKV_ERR_TIMEOUT with device_error = 64 until
+ * treekv_reset.  Healthy runs never take this path, so this call is how the status plumbing is exercised.
+ */
+treekv_status treekv_selftest_wait_giveup(treekv_ctx* ctx, int attempts, void* stream);
 
 /* Tokens seen so far by sequence b according to the host-side record (-1 on bad arguments). */
 int64_t treekv_tokens_seen(const treekv_ctx* ctx, int b);

@@ -24,7 +24,7 @@ EXPORTS = [
     "treekv_decode_step_host", "treekv_prefill_chunk_host", "treekv_prefill_chunk_static_scratch", "treekv_retained_positions", "treekv_scores",
     "treekv_get_stats", "treekv_tokens_seen", "treekv_set_rule", "treekv_set_option", "treekv_reset",
     "treekv_destroy", "treekv_status_string", "treekv_version",
-    "treekv_state_bytes", "treekv_export_state", "treekv_import_state",
+    "treekv_state_bytes", "treekv_export_state", "treekv_import_state", "treekv_selftest_wait_giveup",
 ]
 
 
@@ -92,6 +92,8 @@ def _load():
     lib.treekv_export_state.argtypes = [vp, vp, C.POINTER(C.c_int64), vp]
     lib.treekv_import_state.restype = i32
     lib.treekv_import_state.argtypes = [vp, vp, C.POINTER(C.c_int64), vp]
+    lib.treekv_selftest_wait_giveup.restype = i32
+    lib.treekv_selftest_wait_giveup.argtypes = [vp, i32, vp]
     return lib
 
 
@@ -199,6 +201,10 @@ def treekv_import_state(ctx, dev_image, tokens_seen, stream=0) -> int:
     return lib.treekv_import_state(ctx, dev_image, seen, stream)
 
 
+def treekv_selftest_wait_giveup(ctx, attempts, stream=0) -> int:
+    return lib.treekv_selftest_wait_giveup(ctx, attempts, stream)
+
+
 def treekv_destroy(ctx) -> None:
     lib.treekv_destroy(ctx)
 
@@ -269,6 +275,19 @@ class TreeKV:
                                     stride, self._stream()), "treekv_prefill_chunk")
         return out
 
+    def prefill_chunk_static_scratch(self, q, k, v, out=None, chunk_lens=None):
+        """prefill_chunk through the entry point whose scratch is the library's fixed device area (no allocation)."""
+        B, Hq, Hkv, d = self.batch, self.n_heads, self.n_kv_heads, self.head_dim
+        stride = q.shape[1]
+        self._chk(q, (B, stride, Hq, d)); self._chk(k, (B, stride, Hkv, d)); self._chk(v, (B, stride, Hkv, d))
+        if out is None:
+            out = self.torch.empty_like(q)
+        self._chk(out, (B, stride, Hq, d))
+        _check(treekv_prefill_chunk_static_scratch(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                                   chunk_lens, stride, self._stream()),
+               "treekv_prefill_chunk_static_scratch")
+        return out
+
     def decode_step_host(self, q, k, v, out, active=None):
         """q,k,v,out: CPU tensors (pinned for asynchronous copies)."""
         _check(treekv_decode_step_host(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), active,
@@ -294,10 +313,13 @@ class TreeKV:
         _check(treekv_scores(self._h, sb.data_ptr(), self._stream()), "treekv_scores")
         return sb
 
-    def stats(self):
+    def stats(self, check=True):
+        """Counters as a dict.  With check=False a device-side give-up (TREEKV_ERR_TIMEOUT) is reported through
+        'device_error' and 'status' instead of raising."""
         st, s = treekv_get_stats(self._h, self._stream())
-        _check(st, "treekv_get_stats")
-        return {"evictions": s.evictions, "near_ties": s.near_ties, "kernel_launches": s.kernel_launches,
+        if check or st not in (TREEKV_OK, 6):
+            _check(st, "treekv_get_stats")
+        return {"status": st, "evictions": s.evictions, "near_ties": s.near_ties, "kernel_launches": s.kernel_launches,
                 "device_error": s.device_error, "last_cuda_error": s.last_cuda_error}
 
     def tokens_seen(self, b=0):

@@ -156,6 +156,7 @@ treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
             sms = 148;
         ctx->sm_count = sms;
+        ctx->device = dev;
     }
     ctx->has_tma = false;
     if (dtype == TREEKV_BF16 && head_dim == 128 && max_chunk > 0) {

@@ -112,10 +112,12 @@ template <> struct Elem<__nv_bfloat16> {
     __device__ static __nv_bfloat16 from_float(float x) { return __float2bfloat16_rn(x); }
 };
 
-// 128-bit read-only load that bypasses L1 allocation; only for rows no thread writes while they are being read
+// 128-bit streaming load of a cache row: served from L2, no L1 allocation.  Deliberately not the non-coherent
+// (.nc) form: the kernel that streams a slab also writes rows of it (the appended token, the survivor's move), and
+// .nc is only defined for data nobody writes while the kernel runs.
 __device__ inline uint4 ld_stream(const void* p) {
     uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
     return r;
 }
 __device__ inline uint4 ld_plain(const void* p) { return *reinterpret_cast<const uint4*>(p); }

@@ -19,6 +19,7 @@ struct treekv_ctx {
     int opt_prefill_path;
     int opt_decode_path;
     int sm_count;
+    int device;  // ordinal of the device that was current at creation: the workspace lives there
     // host-side record
     int64_t n_seen[treekv::kMaxBatch];
     uint64_t evictions;

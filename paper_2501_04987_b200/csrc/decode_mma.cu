@@ -168,6 +168,10 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     }
     pdl_wait();  // every block waits, also one of an inactive sequence
     if (!active.test(b)) return;  // the whole cluster shares b
+    // Remote shared-memory stores below need every CTA of the cluster to have started.  Arrive here (relaxed: nothing
+    // is published yet) and wait just before the first remote store; the whole streaming loop lies between the two,
+    // so the barrier costs nothing.  A cluster of one has no remote stores and stays barrier-free.
+    if (nsplit > 1) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 
     const int N = cv.n_seen[unit];
     const UnitState st = unit_state(N, cv.c);
@@ -417,6 +421,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
 
     // ---- CTA partial: (max, sum) per head and the output relative to the CTA max, pushed with remote stores
     //      (statistics into every CTA of the cluster, the output into CTA 0): nobody waits on a remote load
+    if (nsplit > 1) asm volatile("barrier.cluster.wait.aligned;" ::: "memory");  // every CTA of the cluster is running
     float* o_all0 = cluster.map_shared_rank(o_all, 0);
     for (int idx = tid; idx < G * D; idx += NT) {
         const int h = idx / D, ch = idx % D;

@@ -14,6 +14,8 @@
 // with that device current) and passes that pointer to the kernels.
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "ctx.cuh"
 
@@ -26,13 +28,17 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 
 constexpr int kMaxDevices = 64;
 void* g_scratch_addr[kMaxDevices];  // device address of g_static_scratch, per device ordinal; 0 = not looked up yet
+std::mutex g_scratch_mutex;         // host threads may make their first calls at the same time
 
-// Device address of the static scratch on the current device.  The first call on a device performs the lookup.
-cudaError_t static_scratch_address(void** out) {
+// Device address of the static scratch on the current device.  The first call on a device performs the lookup
+// (the runtime loads the module that holds the array at that moment, which is when the device commits its 16 MiB).
+cudaError_t static_scratch_address(void** out, int* dev_out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    *dev_out = dev;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
     if (!g_scratch_addr[dev]) {
         void* p = nullptr;
         e = cudaGetSymbolAddress(&p, g_static_scratch);
@@ -84,8 +90,11 @@ extern "C" treekv_status treekv_prefill_chunk_static_scratch(treekv_ctx* ctx, co
     if (b_col + 2 * b_row + 2 * b_scalar > kStaticScratchBytes) return TREEKV_ERR_UNSUPPORTED;  // beyond the 16 MiB limit
     if (prefill_simt_smem_bytes(ctx->G, ctx->cv.d, ps.n_max) > 227 * 1024) return TREEKV_ERR_UNSUPPORTED;
     void* base_v = nullptr;
-    cudaError_t e = static_scratch_address(&base_v);
+    int dev = -1;
+    cudaError_t e = static_scratch_address(&base_v, &dev);
     if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; return TREEKV_ERR_CUDA; }
+    // the area is per device: the kernels of this call must run where the context's workspace lives
+    if (dev != ctx->device) return TREEKV_ERR_BAD_STATE;
     unsigned char* base = static_cast<unsigned char*>(base_v);
     ps.colsum = reinterpret_cast<float*>(base);
     ps.stage_K = base + b_col;

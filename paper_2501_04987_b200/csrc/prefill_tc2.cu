@@ -16,41 +16,17 @@
 // that gives up sets an error word and the CTA drains to its exit, where tensor memory is released.
 #include <type_traits>
 
-#include "common.cuh"
-#include "tma.cuh"
+#include "prefill_tc_common.cuh"
 
 namespace treekv {
 
 namespace {
 
-constexpr int kSlot = 32768;   // one tile: [2 halves of 64 channels or 64 queries][128 rows][128 bytes]
-constexpr int kHalf = 16384;
+using namespace tc;
+
 constexpr int kRing = 3;       // K / V tiles in flight
-constexpr int kThreads = 576;  // TMA warp, MMA warp, 2 groups x 8 softmax warps
-constexpr uint32_t kTmemCols = 512;
-constexpr int kD = 128;
 
 enum Bar { Q_FULL = 0, RING_FULL = 1, RING_EMPTY = 4, S_FULL = 7, S_FREE = 11, P_FULL = 15, P_FREE = 17, O_FULL = 19, N_BARS = 20 };
-
-struct KeyTiles {
-    int i;     // cycle position: live rows [0,i) and [2i, ...)
-    int L;     // cached rows before the chunk
-    int nvis;  // live indices [0, nvis) are visible to at least one query of this CTA
-    int nA;    // tiles over the old segment [0, i)
-    int NT;    // all tiles
-};
-// key tile j: first live index, first physical row, rows that exist
-__device__ inline void tile_of(const KeyTiles& kt, int j, int& lam0, int& row0, int& valid) {
-    if (j < kt.nA) { lam0 = j * 128; row0 = lam0; valid = min(128, kt.i - lam0); }
-    else { lam0 = kt.i + (j - kt.nA) * 128; row0 = lam0 + kt.i; valid = min(128, kt.nvis - lam0); }
-}
-
-// 2^x on the special-function unit, one instruction (inputs here are <= ~0; results below 2^-126 flush to zero)
-__device__ inline float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 
 }  // namespace
 

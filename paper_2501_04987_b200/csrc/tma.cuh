@@ -33,12 +33,13 @@ __device__ inline bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// bounded wait for the phase with the given parity; false = gave up
-__device__ inline bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it)
+// bounded wait for the phase with the given parity, at most `limit` attempts; false = gave up
+__device__ inline bool mbar_wait_limit(uint32_t bar, uint32_t parity, uint32_t limit) {
+    for (uint32_t it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+__device__ inline bool mbar_wait(uint32_t bar, uint32_t parity) { return mbar_wait_limit(bar, parity, kSpinLimit); }
 // orders earlier generic-proxy accesses to shared memory before later async-proxy (TMA, tcgen05.mma) accesses
 __device__ inline void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 

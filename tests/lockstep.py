@@ -8,6 +8,8 @@ element by element within the stated tolerances.
 """
 from __future__ import annotations
 
+import os
+
 import numpy as np
 
 OUT_TOL = {"bf16": 2e-2, "f32": 1e-4}   # max abs error of attention outputs
@@ -16,18 +18,40 @@ SCORE_ATOL = 1e-12                       # floor for weights that underflow in f
 NEAR_TIE = 1e-4
 
 
+REPORTS = []   # every Report of the session, in creation order; the terminal summary prints them (conftest.py)
+
+
 class Report:
-    def __init__(self):
+    """Tallies of one lock-step run.  `decisions` counts pair decisions (evictions x KV heads) the oracle took,
+    `near_ties` those whose relative gap was below NEAR_TIE, `flips` those where the oracle followed the library."""
+
+    def __init__(self, label=None):
+        self.label = label or os.environ.get("PYTEST_CURRENT_TEST", "?").split(" ")[0]
         self.calls = 0
         self.max_out_err = 0.0
         self.max_score_rel = 0.0
         self.near_ties = 0
         self.flips = 0
         self.decisions = 0
+        REPORTS.append(self)
+
+    def tally(self, orc, evicted_before, near_ties, flips):
+        """Add one oracle eviction call: `evicted_before` = sum of n_evicted over sequences before the call."""
+        after = sum(orc.n_evicted(b) for b in range(orc.B))
+        self.decisions += (after - evicted_before) * orc.Hkv
+        self.near_ties += near_ties
+        self.flips += flips
+        self.calls += 1
+        # a flip is only possible at a near-tie: anything else means the oracle followed the library where it must not
+        assert self.flips <= self.near_ties <= self.decisions, repr(self)
 
     def __repr__(self):
-        return ("calls=%d max_out_err=%.3g max_score_rel=%.3g near_ties=%d flips=%d" %
-                (self.calls, self.max_out_err, self.max_score_rel, self.near_ties, self.flips))
+        return ("calls=%d max_out_err=%.3g max_score_rel=%.3g decisions=%d near_ties=%d flips=%d" %
+                (self.calls, self.max_out_err, self.max_score_rel, self.decisions, self.near_ties, self.flips))
+
+
+def evicted_total(orc):
+    return sum(orc.n_evicted(b) for b in range(orc.B))
 
 
 def _to_dev(torch, a, tdtype):
@@ -70,8 +94,9 @@ def step_decode(kv, orc, q, k, v, dtype, rep, active=None, check_scores=True):
     out_g = kv.decode_step(_to_dev(torch, q, kv.tdtype), _to_dev(torch, k, kv.tdtype), _to_dev(torch, v, kv.tdtype),
                            active=active)
     pos_g, cnt_g = kv.retained_positions()
+    ev0 = evicted_total(orc)
     nt, fl = orc.evict(pos_g.cpu().numpy(), cnt_g.cpu().numpy(), NEAR_TIE)
-    rep.near_ties += nt; rep.flips += fl; rep.calls += 1
+    rep.tally(orc, ev0, nt, fl)
     og = out_g.float().cpu().numpy().astype(np.float64)
     sel = slice(None) if active is None else np.asarray(active, bool)
     err = float(np.abs(og[sel] - out_o[sel]).max()) if np.size(og[sel]) else 0.0
@@ -80,18 +105,19 @@ def step_decode(kv, orc, q, k, v, dtype, rep, active=None, check_scores=True):
     compare_state(kv, orc, rep, check_scores)
 
 
-def step_prefill(kv, orc, q, k, v, dtype, rep, chunk_lens=None, check_scores=True):
-    """q [B,m,Hq,d], k,v [B,m,Hkv,d] float32 numpy holding dtype-rounded values."""
+def step_prefill(kv, orc, q, k, v, dtype, rep, chunk_lens=None, check_scores=True, method="prefill_chunk"):
+    """q [B,m,Hq,d], k,v [B,m,Hkv,d] float32 numpy holding dtype-rounded values; `method` names the wrapper's call."""
     import torch
 
     B, m = q.shape[0], q.shape[1]
     lens = [m] * B if chunk_lens is None else [int(x) for x in chunk_lens]
     out_o = orc.prefill_attend(q, k, v, lens)
-    out_g = kv.prefill_chunk(_to_dev(torch, q, kv.tdtype), _to_dev(torch, k, kv.tdtype), _to_dev(torch, v, kv.tdtype),
-                             chunk_lens=lens)
+    out_g = getattr(kv, method)(_to_dev(torch, q, kv.tdtype), _to_dev(torch, k, kv.tdtype),
+                                _to_dev(torch, v, kv.tdtype), chunk_lens=lens)
     pos_g, cnt_g = kv.retained_positions()
+    ev0 = evicted_total(orc)
     nt, fl = orc.evict(pos_g.cpu().numpy(), cnt_g.cpu().numpy(), NEAR_TIE)
-    rep.near_ties += nt; rep.flips += fl; rep.calls += 1
+    rep.tally(orc, ev0, nt, fl)
     og = out_g.float().cpu().numpy().astype(np.float64)
     err = 0.0
     for b in range(B):

@@ -3,10 +3,14 @@
 One layer of each configuration is run at its full batch / head count / budget / chunk size.  The oracle cannot
 follow every unit at these sizes, so:
   * decode (configuration 2's shape): single-head oracles follow sampled (sequence, head) units in lock-step;
-  * chunked prefill (configurations 4 and 5): sampled output rows are recomputed one by one in fp64 as plain
-    softmax attention over [tokens retained before the chunk | chunk tokens up to the row's own] from the raw
-    input stream, and the cache invariants that hold at any size are checked after every call (length = min(seen,
-    budget), strictly increasing positions, every averaged score in [0, 1]).
+  * chunked prefill (configurations 4 and 5, and the maximum chunk): an oracle with one KV head and the group's g
+    query heads follows every sampled (sequence, KV head) unit in lock-step through prefill_attend + evict(hint) -
+    retained positions exactly, averaged scores within 1e-3, every output row of the unit within 2e-2, after every
+    call - at the launch shape the library picks by itself (the two-tile tensor-core kernel on 512 and more CTAs);
+    beside it, sampled output rows are recomputed one by one in fp64 as plain softmax attention over [tokens
+    retained before the chunk | chunk tokens up to the row's own] from the raw input stream, and the cache
+    invariants that hold at any size are checked after every call (length = min(seen, budget), strictly increasing
+    positions, every averaged score in [0, 1]).
 Inputs are seeded Gaussians drawn with torch on the device (keys with the configuration's outlier channels or
 per-sequence scale; no rotary embedding here - the lock-step tests on slices use the full recipe).
 """
@@ -16,6 +20,7 @@ import numpy as np
 import pytest
 
 import workloads as W
+from lockstep import NEAR_TIE, OUT_TOL, SCORE_ATOL, SCORE_RTOL, Report, evicted_total
 
 pytestmark = pytest.mark.gpu
 
@@ -79,7 +84,7 @@ def test_cfg2_full_layer_decode_sampled_units(gpu):
     sampled = [(0, 0), (3, 17), (7, 31)]
     orcs = [Oracle(w.budget, 1, 1, w.head_dim, 1) for _ in sampled]
     steps = w.budget + 1024 + 60
-    flips = near = 0
+    reps = [Report() for _ in sampled]
     max_err = 0.0
     for t in range(steps):
         q = _draw(torch, gen, (w.batch, w.n_heads, w.head_dim))
@@ -87,16 +92,17 @@ def test_cfg2_full_layer_decode_sampled_units(gpu):
         v = _draw(torch, gen, (w.batch, w.n_kv_heads, w.head_dim))
         out = kv.decode_step(q, k, v)
         pos, cnt = kv.retained_positions()
-        for (b, h), orc in zip(sampled, orcs):
+        for (b, h), orc, rep in zip(sampled, orcs, reps):
             qo = q[b, h].float().cpu().numpy()[None, None]
             ko = k[b, h].float().cpu().numpy()[None, None]
             vo = v[b, h].float().cpu().numpy()[None, None]
             ref = orc.decode_attend(qo, ko, vo)
             hp = pos[b, h].cpu().numpy()[None, None]; hc = cnt[b, h].cpu().numpy()[None, None]
-            nt, fl = orc.evict(hp, hc, 1e-4)
-            near += nt; flips += fl
+            ev0 = evicted_total(orc)
+            nt, fl = orc.evict(hp, hc, NEAR_TIE)
+            rep.tally(orc, ev0, nt, fl)
             err = float(np.abs(out[b, h].float().cpu().numpy() - ref[0, 0]).max())
-            max_err = max(max_err, err)
+            max_err = max(max_err, err); rep.max_out_err = max(rep.max_out_err, err)
             assert err <= 2e-2, (t, b, h, err)
             assert np.array_equal(orc.retained_positions()[0][0, 0], hp[0, 0]), (t, b, h)
         if t % 97 == 0 or t == steps - 1:
@@ -107,11 +113,60 @@ def test_cfg2_full_layer_decode_sampled_units(gpu):
     _check_invariants(kv, [steps] * w.batch)
     st = kv.stats()
     assert st["device_error"] == 0 and st["evictions"] == w.batch * (steps - w.budget)
-    print("cfg2 full layer: max out err %.3g, near-ties %d, flips %d" % (max_err, near, flips))
+    print("cfg2 full layer: max out err %.3g" % max_err, reps)
+
+
+def _lockstep_sampled(orc, rep, sampled, q, k, v, out, lens, pos_g, cnt_g, sb_g, decode):
+    """One call of the single-KV-head oracle (sequence s of the oracle = sampled unit s) beside the library's call.
+    q,k,v,out: the call's device tensors; pos_g, cnt_g, sb_g: the library's read-outs after the call (numpy)."""
+    g = orc.Hq
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    if decode:
+        qs = np.stack([f64(q[b, kh * g:(kh + 1) * g]) for (b, kh) in sampled])            # [S, g, d]
+        ks = np.stack([f64(k[b, kh:kh + 1]) for (b, kh) in sampled])
+        vs = np.stack([f64(v[b, kh:kh + 1]) for (b, kh) in sampled])
+        out_o = orc.decode_attend(qs, ks, vs)
+        out_g = np.stack([f64(out[b, kh * g:(kh + 1) * g]) for (b, kh) in sampled])
+        err = float(np.abs(out_g - out_o).max())
+    else:
+        qs = np.stack([f64(q[b, :, kh * g:(kh + 1) * g]) for (b, kh) in sampled])         # [S, m, g, d]
+        ks = np.stack([f64(k[b, :, kh:kh + 1]) for (b, kh) in sampled])
+        vs = np.stack([f64(v[b, :, kh:kh + 1]) for (b, kh) in sampled])
+        ls = [lens[b] for (b, kh) in sampled]
+        out_o = orc.prefill_attend(qs, ks, vs, ls)
+        err = 0.0
+        for s, (b, kh) in enumerate(sampled):
+            if ls[s]:
+                err = max(err, float(np.abs(f64(out[b, :ls[s], kh * g:(kh + 1) * g]) - out_o[s, :ls[s]]).max()))
+    rep.max_out_err = max(rep.max_out_err, err)
+    assert err <= OUT_TOL["bf16"], "sampled units' outputs off by %.3g" % err
+    hp = np.stack([pos_g[b, kh] for (b, kh) in sampled])[:, None, :].astype(np.int32)
+    hc = np.array([[cnt_g[b, kh]] for (b, kh) in sampled], np.int32)
+    ev0 = evicted_total(orc)
+    nt, fl = orc.evict(hp, hc, NEAR_TIE)
+    rep.tally(orc, ev0, nt, fl)
+    pos_o, cnt_o = orc.retained_positions()
+    assert np.array_equal(cnt_o, hc), "retained counts differ from the oracle's"
+    if not np.array_equal(pos_o, hp):
+        bad = np.argwhere(pos_o != hp)[0]
+        raise AssertionError("retained positions differ at sampled unit %s slot %d: library %d oracle %d" %
+                             (sampled[bad[0]], bad[2], hp[tuple(bad)], pos_o[tuple(bad)]))
+    so = orc.scores()[:, 0, :]
+    sg = np.stack([sb_g[b, kh] for (b, kh) in sampled]).astype(np.float64)
+    e = np.abs(sg - so)
+    lim = SCORE_RTOL * np.abs(so) + SCORE_ATOL
+    if not np.all(e <= lim):
+        bad = np.argwhere(e > lim)[0]
+        raise AssertionError("score differs at sampled unit %s slot %d: library %.9g oracle %.9g" %
+                             (sampled[bad[0]], bad[1], sg[tuple(bad)], so[tuple(bad)]))
+    with np.errstate(divide="ignore", invalid="ignore"):
+        rel = np.where(so > 1e-9, e / so, 0.0)
+    rep.max_score_rel = max(rep.max_score_rel, float(rel.max()))
 
 
 def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_chunk=None):
     import torch
+    from oracle import Oracle
 
     B, Hq, Hkv, d, m, c = w.batch, w.n_heads, w.n_kv_heads, w.head_dim, w.chunk, w.budget
     g = Hq // Hkv
@@ -120,6 +175,8 @@ def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_c
     rs = np.random.default_rng(w.seed)
     seq_scale = torch.from_numpy(W.seq_key_scales(w)).cuda() if w.key_scale else None
     sampled = sorted(set([(0, 0), (B - 1, Hkv - 1), (B // 2, Hkv // 2)]))
+    orc = Oracle(c, g, 1, d, len(sampled))   # sequence s of the oracle follows sampled unit s (one KV head, g query heads)
+    rep = Report()
     hist_k = {u: np.zeros((0, d)) for u in sampled}   # full key / value streams of the sampled units (fp64)
     hist_v = {u: np.zeros((0, d)) for u in sampled}
     seen = [0] * B
@@ -156,7 +213,8 @@ def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_c
                     max_err = max(max_err, err)
                     assert err <= 2e-2, (call, b, t, h, err)
         seen = [s + l for s, l in zip(seen, lens)]
-        _check_invariants(kv, seen)
+        pos_g, cnt_g = _check_invariants(kv, seen)
+        _lockstep_sampled(orc, rep, sampled, q, k, v, out, lens, pos_g, cnt_g, kv.scores().cpu().numpy(), decode=False)
     assert [kv.tokens_seen(b) for b in range(B)] == seen
     # batched decode steps at ragged stream positions: sampled rows against brute force over the retained set
     for step in range(decode_steps):
@@ -177,8 +235,12 @@ def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_c
                 max_err = max(max_err, err)
                 assert err <= 2e-2, (step, b, h, err)
         seen = [s + 1 for s in seen]
+        pos_g, cnt_g = kv.retained_positions()
+        _lockstep_sampled(orc, rep, sampled, q, k, v, out, None, pos_g.cpu().numpy(), cnt_g.cpu().numpy(),
+                          kv.scores().cpu().numpy(), decode=True)
     _check_invariants(kv, seen)
     assert kv.stats()["device_error"] == 0
+    print(rep)
     return max_err
 
 

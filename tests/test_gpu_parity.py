@@ -232,8 +232,6 @@ def test_score_free_rules_match_closed_structure(gpu, rule):
         pb = b.retained_positions()[0].cpu().numpy()
         assert np.array_equal(pa, pb)
         assert np.array_equal(pa, orc.retained_positions()[0])
-    if rule == 2:  # evict-left closed form: offsets from the newest token
-        pass
 
 
 def test_inactive_sequences_are_untouched(gpu):
@@ -429,3 +427,30 @@ def test_argument_and_state_errors(gpu):
     kv.reset()
     assert kv.tokens_seen(0) == 0
     assert kv.retained_positions()[1].cpu().numpy().tolist() == [[0] * 4] * 2
+
+
+def test_device_side_give_up_surfaces_as_timeout_status(gpu):
+    """A bounded wait that gives up must reach the caller as TREEKV_ERR_TIMEOUT and be cleared by a reset.  No real
+    kernel ever gives up in a healthy run, so the library's self-test kernel makes one wait run out: a few dozen
+    polls of a barrier that nothing signals, nothing asynchronous outstanding, the cache untouched."""
+    import torch
+
+    kv = gpu.TreeKV(16, 4, 4, 64, "f32", 2, 0)
+    x = torch.randn((2, 4, 64), device="cuda")
+    kv.decode_step(x, x, x)
+    assert kv.stats()["device_error"] == 0
+    assert gpu.treekv_selftest_wait_giveup(kv._h, 0) == 1 and gpu.treekv_selftest_wait_giveup(kv._h, 5000) == 1
+    assert gpu.treekv_selftest_wait_giveup(kv._h, 48) == 0
+    st = kv.stats(check=False)
+    assert st["status"] == 6 and st["device_error"] == 64
+    assert gpu.status_string(6) == "device-side wait timed out"
+    with pytest.raises(gpu.TreeKVError):
+        kv.stats()
+    # the context and the GPU stay usable: the cache was not touched, and a reset clears the error word
+    assert kv.tokens_seen(0) == 1 and kv.retained_positions()[1].cpu().numpy().tolist() == [[1] * 4] * 2
+    kv.reset()
+    st = kv.stats()
+    assert st["device_error"] == 0 and st["status"] == 0
+    kv.decode_step(x, x, x)
+    torch.cuda.synchronize()
+    assert kv.stats()["device_error"] == 0 and kv.tokens_seen(0) == 1

@@ -93,4 +93,4 @@ def test_reference_arm_line_on_rank_zero():
     assert line["impl"] == "reference" and line["metric"] == "treekv_decode_steps_per_s" and line["unit"] == "steps/s"
     assert line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
     assert line["e2e"] == {"value": line["value"], "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
-    assert line["higher_is_better"] is True and line["config"]["workload"] == "cfg2"
+    assert line["higher_is_better"] is True and line["config"]["workload"] == "cfg4"
