@@ -31,7 +31,15 @@
  *     chunk attends to every slot whose pos <= its own, S and C are advanced
  *     for all m steps at once, then Algorithm 1's eviction branch is repeated
  *     with those frozen scores until the length is back to c.
- *   PARITY UNPINNED: the last two readings are not fixed by anything the paper
+ *   - protected tokens (Section 5.2, "4 initial tokens, 508 recent tokens, and 512 method-selected tokens"; the
+ *     paper does not say how the three parts interact): the first n_sink tokens of the stream and the newest
+ *     n_recent cached tokens are never in an eviction scope.  Algorithm 1 runs on the region between them, whose
+ *     size is c_mid = c - n_sink - n_recent: the scope is slots {n_sink + idx, n_sink + idx + 1} of the whole
+ *     cache and idx cycles 1..c_mid.  A token becomes eligible in the step in which it stops being one of the
+ *     n_recent newest (it is then the last slot of the middle region, exactly where Algorithm 1 appends).  S and
+ *     C of every cached token, protected or not, advance as in Algorithm 1 from the token's arrival.  With
+ *     n_sink = n_recent = 0 this is Algorithm 1 unchanged.
+ *   PARITY UNPINNED: the last three readings are not fixed by anything the paper
  *   prints; the tests constrain them (m=1 equals a decode step, mass
  *   conservation, score-free rules give identical retained sets) but cannot
  *   pin them to the paper.
@@ -58,6 +66,7 @@ typedef struct {
 
 typedef struct {
     int c, Hq, Hkv, d, B, g;
+    int n_sink, n_recent; /* protected tokens at both ends (Section 5.2); 0, 0 = Algorithm 1 as printed */
     int rule, idx_mode;
     int64_t *n_seen;    /* [B] */
     int64_t *n_evicted; /* [B] */
@@ -109,6 +118,15 @@ void tkvo_destroy(tkvo *o) {
 }
 
 void tkvo_set_rule(tkvo *o, int rule) { o->rule = rule; }
+
+/* Section 5.2: keep the first n_sink tokens and the newest n_recent tokens out of every eviction scope.
+ * Only valid before the first token; the middle region must keep room for a scope. Returns 0 on success. */
+int tkvo_set_protection(tkvo *o, int n_sink, int n_recent) {
+    if (n_sink < 0 || n_recent < 0 || o->c - n_sink - n_recent < 2) return -1;
+    for (int b = 0; b < o->B; ++b) if (o->n_seen[b] != 0) return -2;
+    o->n_sink = n_sink; o->n_recent = n_recent;
+    return 0;
+}
 void tkvo_set_idx_mode(tkvo *o, int mode) { o->idx_mode = mode; }
 
 /* Append one token to every KV head of sequence b (Alg. 1, the two append
@@ -254,12 +272,13 @@ static int in_sorted(const int32_t *a, int n, int64_t x) {
 void tkvo_evict(tkvo *o, const int32_t *hint_pos, const int32_t *hint_cnt, double near_tie_tol) {
     o->last_near_ties = 0; o->last_hint_flips = 0; o->last_min_gap = INFINITY;
     const int c = o->c, d = o->d;
+    const int c_mid = c - o->n_sink - o->n_recent; /* size of the region Algorithm 1 runs on (= c without protection) */
     for (int b = 0; b < o->B; ++b) {
         while (o->u[b * o->Hkv].len > c) {
-            const int idx = o->idx[b]; /* 1-based: scope is slots idx, idx+1 */
+            const int idx = o->idx[b]; /* 1-based within the middle region: scope is its slots idx, idx+1 */
             for (int kh = 0; kh < o->Hkv; ++kh) {
                 tkvo_unit *u = &o->u[b * o->Hkv + kh];
-                const int l = idx - 1, r = idx; /* 0-based slots */
+                const int l = o->n_sink + idx - 1, r = o->n_sink + idx; /* 0-based slots of the whole cache */
                 int evict_right;
                 if (o->rule == TKVO_RULE_KEEP_LEFT) evict_right = 1;
                 else if (o->rule == TKVO_RULE_EVICT_LEFT) evict_right = 0;
@@ -286,8 +305,8 @@ void tkvo_evict(tkvo *o, const int32_t *hint_pos, const int32_t *hint_cnt, doubl
                 }
                 unit_remove(u, d, evict_right ? r : l); /* Alg. 1: evict one of the pair */
             }
-            if (o->idx_mode == TKVO_IDX_LITERAL) o->idx[b] = (idx + 1) % c + 1;
-            else o->idx[b] = (idx % c) + 1; /* idx update, as the prose of Section 4.1 reads */
+            if (o->idx_mode == TKVO_IDX_LITERAL) o->idx[b] = (idx + 1) % c_mid + 1;
+            else o->idx[b] = (idx % c_mid) + 1; /* idx update, as the prose of Section 4.1 reads */
             o->n_evicted[b] += 1;
         }
     }

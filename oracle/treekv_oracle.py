@@ -46,6 +46,8 @@ def _load():
     lib.tkvo_destroy.argtypes = [vp]
     lib.tkvo_set_rule.argtypes = [vp, C.c_int]
     lib.tkvo_set_idx_mode.argtypes = [vp, C.c_int]
+    lib.tkvo_set_protection.argtypes = [vp, C.c_int, C.c_int]
+    lib.tkvo_set_protection.restype = C.c_int
     for name in ("tkvo_decode_attend", "tkvo_decode_step"):
         getattr(lib, name).argtypes = [vp, dp, dp, dp, dp, C.POINTER(C.c_uint8)]
         getattr(lib, name).restype = None
@@ -88,7 +90,8 @@ def _dp(a):
 class Oracle:
     """One TreeKV cache policy (one attention layer) for `batch` sequences."""
 
-    def __init__(self, budget, n_heads, n_kv_heads, head_dim, batch=1, rule=RULE_SCORES, idx_mode=IDX_CYCLE):
+    def __init__(self, budget, n_heads, n_kv_heads, head_dim, batch=1, rule=RULE_SCORES, idx_mode=IDX_CYCLE,
+                 n_sink=0, n_recent=0):
         self._lib = _load()
         self._h = self._lib.tkvo_create(budget, n_heads, n_kv_heads, head_dim, batch)
         if not self._h:
@@ -96,6 +99,9 @@ class Oracle:
         self.c, self.Hq, self.Hkv, self.d, self.B = budget, n_heads, n_kv_heads, head_dim, batch
         self._lib.tkvo_set_rule(self._h, rule)
         self._lib.tkvo_set_idx_mode(self._h, idx_mode)
+        self.n_sink, self.n_recent = n_sink, n_recent
+        if (n_sink or n_recent) and self._lib.tkvo_set_protection(self._h, n_sink, n_recent) != 0:
+            raise ValueError("bad protection: the region between sinks and recent tokens needs at least 2 slots")
 
     def __del__(self):
         h, self._h = getattr(self, "_h", None), None
