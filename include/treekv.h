@@ -228,6 +228,18 @@ treekv_status treekv_selftest_wait_giveup(treekv_ctx* ctx, int attempts, void* s
 int64_t treekv_tokens_seen(const treekv_ctx* ctx, int b);
 
 treekv_status treekv_set_rule(treekv_ctx* ctx, treekv_rule rule);
+
+/*
+ * Protected tokens (Section 5.2: the language-modelling runs keep "4 initial tokens, 508 recent tokens, and 512
+ * method-selected tokens" in a cache of 1024).  The first n_sink tokens of every sequence and its n_recent newest
+ * cached tokens are never in an eviction scope; Algorithm 1 runs on the budget - n_sink - n_recent slots between
+ * them (idx cycles over that many slots), and a token becomes eligible in the step in which it stops being one of
+ * the n_recent newest.  S and C of every cached token advance from its arrival as in Algorithm 1.  The paper gives
+ * the split, not these mechanics.  (0, 0) - the default - is Algorithm 1 as printed.
+ * Needs n_sink + n_recent <= budget - 2 (TREEKV_ERR_INVALID_ARG) and a context that has not seen a token yet
+ * (after creation or treekv_reset; else TREEKV_ERR_BAD_STATE).  Host-side only, nothing is enqueued.
+ */
+treekv_status treekv_set_protection(treekv_ctx* ctx, int n_sink, int n_recent);
 treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value);
 
 /* Back to the empty cache (idx = 1, nothing seen).  Enqueued on `stream`. */

@@ -25,6 +25,7 @@ EXPORTS = [
     "treekv_get_stats", "treekv_tokens_seen", "treekv_set_rule", "treekv_set_option", "treekv_reset",
     "treekv_destroy", "treekv_status_string", "treekv_version",
     "treekv_state_bytes", "treekv_export_state", "treekv_import_state", "treekv_selftest_wait_giveup",
+    "treekv_set_protection",
 ]
 
 
@@ -92,6 +93,8 @@ def _load():
     lib.treekv_export_state.argtypes = [vp, vp, C.POINTER(C.c_int64), vp]
     lib.treekv_import_state.restype = i32
     lib.treekv_import_state.argtypes = [vp, vp, C.POINTER(C.c_int64), vp]
+    lib.treekv_set_protection.restype = i32
+    lib.treekv_set_protection.argtypes = [vp, i32, i32]
     lib.treekv_selftest_wait_giveup.restype = i32
     lib.treekv_selftest_wait_giveup.argtypes = [vp, i32, vp]
     return lib
@@ -176,6 +179,10 @@ def treekv_tokens_seen(ctx, b) -> int:
 
 def treekv_set_rule(ctx, rule) -> int:
     return lib.treekv_set_rule(ctx, rule)
+
+
+def treekv_set_protection(ctx, n_sink, n_recent) -> int:
+    return lib.treekv_set_protection(ctx, n_sink, n_recent)
 
 
 def treekv_set_option(ctx, opt, value) -> int:
@@ -327,6 +334,9 @@ class TreeKV:
 
     def set_rule(self, rule):
         _check(treekv_set_rule(self._h, rule), "treekv_set_rule")
+
+    def set_protection(self, n_sink, n_recent):
+        _check(treekv_set_protection(self._h, n_sink, n_recent), "treekv_set_protection")
 
     def set_option(self, opt, value):
         _check(treekv_set_option(self._h, opt, value), "treekv_set_option")

@@ -17,7 +17,7 @@ constexpr size_t kSmemLimit = 227 * 1024;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, S, pos, n_seen, stats, colsum, st_q, st_k, st_v, st_out, total;
+    size_t K, V, S, pos, n_seen, w0, stats, colsum, st_q, st_k, st_v, st_out, total;
     int R, QT, n_max;
 };
 
@@ -52,6 +52,7 @@ Layout make_layout(int budget, int n_heads, int n_kv_heads, int head_dim, treekv
     L.S = take(units * L.R * 4);
     L.pos = take(units * L.R * 4);
     L.n_seen = take(units * 4);
+    L.w0 = take(units * 4);
     L.stats = take(sizeof(DevStats));
     L.colsum = take(units * L.QT * L.n_max * 4);
     const size_t mc = max_chunk > 0 ? max_chunk : 1;
@@ -140,9 +141,11 @@ treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_
     ctx->cv.S = reinterpret_cast<float*>(base + L.S);
     ctx->cv.pos = reinterpret_cast<int32_t*>(base + L.pos);
     ctx->cv.n_seen = reinterpret_cast<int32_t*>(base + L.n_seen);
+    ctx->cv.w0 = reinterpret_cast<int32_t*>(base + L.w0);
     ctx->cv.stats = reinterpret_cast<DevStats*>(base + L.stats);
     ctx->cv.c = budget; ctx->cv.R = L.R; ctx->cv.Hq = n_heads; ctx->cv.Hkv = n_kv_heads; ctx->cv.B = batch;
     ctx->cv.d = head_dim; ctx->cv.rule = TREEKV_RULE_SCORES;
+    ctx->cv.ns = 0; ctx->cv.nr = 0; ctx->cv.cm = budget;
     ctx->ps.colsum = reinterpret_cast<float*>(base + L.colsum);
     // (rows in flight during compaction stay in registers: the context has no staging rows; PrefillScratch's
     //  staging pointers are only used by the entry point that brings its own scratch)
@@ -416,6 +419,15 @@ treekv_status treekv_set_rule(treekv_ctx* ctx, treekv_rule rule) {
     if (rule != TREEKV_RULE_SCORES && rule != TREEKV_RULE_KEEP_LEFT && rule != TREEKV_RULE_EVICT_LEFT)
         return TREEKV_ERR_INVALID_ARG;
     ctx->cv.rule = (int)rule;
+    return TREEKV_OK;
+}
+
+treekv_status treekv_set_protection(treekv_ctx* ctx, int n_sink, int n_recent) {
+    if (!ctx) return TREEKV_ERR_INVALID_ARG;
+    if (n_sink < 0 || n_recent < 0 || (long long)n_sink + n_recent > ctx->cv.c - 2) return TREEKV_ERR_INVALID_ARG;
+    for (int b = 0; b < ctx->cv.B; ++b)
+        if (ctx->n_seen[b] != 0) return TREEKV_ERR_BAD_STATE;  // the layout of a cache in use cannot change
+    ctx->cv.ns = n_sink; ctx->cv.nr = n_recent; ctx->cv.cm = ctx->cv.c - n_sink - n_recent;
     return TREEKV_OK;
 }
 

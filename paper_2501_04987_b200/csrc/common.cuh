@@ -9,6 +9,17 @@
 //     [0, i)  and  [2i, L + i)            (both in stream order, the first entirely older than the second)
 // and the next token is appended at row L + i.  While the cache is still filling, i = 0 and the live rows
 // are [0, L).  "Live index" lambda in [0, L) maps to the physical row  lambda < i ? lambda : lambda + i.
+//
+// Protected tokens (Section 5.2 of the paper keeps 4 initial and 508 recent tokens beside 512 selected ones): the
+// first n_sink tokens of the stream and the newest n_recent cached tokens are never in a scope, and Algorithm 1
+// runs on the c_mid = c - n_sink - n_recent slots between them.  In the slab the sinks are rows [0, n_sink) and
+// the cycle sequence [middle region at cycle start | every later token] starts at row n_sink: pairs are rows
+// (n_sink + 2p, n_sink + 2p + 1), p = 0..c_mid-1, the survivor of pair p moves to row n_sink + p, and the live
+// rows are
+//     [0, a)  and  [a + i, L + i)     with the split point a = n_sink + i
+// - again two contiguous segments; without protection a = i and this is the layout above.  When a cycle ends
+// (i reaches c_mid) the n_recent rows that follow the last pair, [n_sink + 2 c_mid, ...), are moved down to
+// [n_sink + c_mid, ...) so that the next cycle starts from a contiguous cache ("re-base").
 #pragma once
 
 #include <cuda.h>
@@ -38,11 +49,15 @@ struct CacheView {
     float* S;         // [units][R]   sum of attention received
     int32_t* pos;     // [units][R]   0-based stream index of the token in the row
     int32_t* n_seen;  // [units]      tokens fed so far (kept per unit so a kernel only reads what it alone writes)
+    int32_t* w0;      // [units]      stream step at which scoring started: C_j = tokens seen - max(pos_j, w0); 0 = Algorithm 1
     DevStats* stats;
     int c;            // budget
     int R;            // rows per slab
     int Hq, Hkv, B, d;
     int rule;
+    int ns;           // protected initial tokens (sinks)
+    int nr;           // protected newest tokens (recent window)
+    int cm;           // c - ns - nr: slots Algorithm 1 runs on = evictions per cycle
 };
 
 struct ActiveMask {
@@ -54,17 +69,23 @@ struct ActiveMask {
 struct UnitState {
     int L;  // cached tokens
     int i;  // evictions done in the current cycle (idx - 1)
+    int a;  // split point n_sink + i: live indices below it sit at row = index, the others at index + i
 };
-__host__ __device__ inline UnitState unit_state(long long n_seen, int c) {
+__host__ __device__ inline UnitState unit_state(long long n_seen, int c, int cm, int ns) {
     UnitState s;
     if (n_seen <= c) { s.L = (int)n_seen; s.i = 0; }
-    else { s.L = c; s.i = (int)((n_seen - c) % c); }
+    else { s.L = c; s.i = (int)((n_seen - c) % cm); }
+    s.a = ns + s.i;
     return s;
 }
-__host__ __device__ inline int phys_row(int lambda, int i) { return lambda < i ? lambda : lambda + i; }
+__host__ __device__ inline UnitState unit_state(long long n_seen, const CacheView& cv) {
+    return unit_state(n_seen, cv.c, cv.cm, cv.ns);
+}
+__host__ __device__ inline int phys_row(int lambda, const UnitState& st) { return lambda < st.a ? lambda : lambda + st.i; }
 
-// One segment of a chunk's eviction: E pairs (2(i+p), 2(i+p)+1) -> row i+p, then, if the cycle wraps with
-// tokens still above budget, `rebase` rows [2c, 2c+rebase) move down to [c, c+rebase).
+// One segment of a chunk's eviction: E pairs (ns + 2(i+p), ns + 2(i+p) + 1) -> row ns + i + p, then, if the cycle
+// wraps, the `rebase` rows that follow the last pair, [ns + 2 cm, ns + 2 cm + rebase), move down to
+// [ns + cm, ns + cm + rebase): the protected recent tokens and whatever is still above budget.
 struct EvictSegment {
     int i;       // cycle position at segment start
     int len;     // live rows at segment start
@@ -72,17 +93,18 @@ struct EvictSegment {
     int rebase;  // rows moved down after a wrap
     int nseg;    // total number of segments for this chunk
 };
-__host__ __device__ inline EvictSegment evict_segment(long long n_seen_before, int m, int c, int seg) {
-    UnitState st = unit_state(n_seen_before, c);
+__host__ __device__ inline EvictSegment evict_segment(long long n_seen_before, int m, const CacheView& cv, int seg) {
+    const int c = cv.c, cm = cv.cm;
+    UnitState st = unit_state(n_seen_before, cv);
     EvictSegment cur;
     cur.i = st.i; cur.len = st.L + m; cur.E = 0; cur.rebase = 0; cur.nseg = 0;
     int i = st.i, len = st.L + m;
     int s = 0;
     while (len > c) {
-        const int E = len - c < c - i ? len - c : c - i;
+        const int E = len - c < cm - i ? len - c : cm - i;
         const int len2 = len - E;
         int i2 = i + E, rebase = 0;
-        if (i2 == c) { i2 = 0; if (len2 > c) rebase = len2 - c; }
+        if (i2 == cm) { i2 = 0; rebase = len2 - (cv.ns + cm); }
         if (s == seg) { cur.i = i; cur.len = len; cur.E = E; cur.rebase = rebase; }
         i = i2; len = len2; ++s;
     }
@@ -121,6 +143,11 @@ __device__ inline uint4 ld_stream(const void* p) {
     return r;
 }
 __device__ inline uint4 ld_plain(const void* p) { return *reinterpret_cast<const uint4*>(p); }
+
+// Algorithm 1's counter C of the token at stream position `pos` once `n_seen` tokens have been fed: the steps in
+// which the token was scored.  That is every step since its arrival, except after a one-shot prefill, where the
+// tokens older than the observation window were only scored from the window's first query (w0) on.
+__host__ __device__ inline int score_count(int n_seen, int pos, int w0) { return n_seen - (pos > w0 ? pos : w0); }
 
 // Algorithm 1's comparison on the averaged scores; returns true when the right member of the pair is evicted.
 // Also reports whether the decision was a near-tie (relative gap below kNearTieRel).

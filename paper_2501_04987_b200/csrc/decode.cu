@@ -33,7 +33,7 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
 
     const int unit = b * cv.Hkv + kh;
     const int N = cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
+    const UnitState st = unit_state(N, cv);
     const int n = st.L + 1;  // live rows including the token appended by this step
     const int i_cyc = st.i;
     const int per = (n + nsplit - 1) / nsplit;
@@ -82,7 +82,7 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
 
     // ---- K phase: logits (in log2 units) of this CTA's rows
     float mx[G];
-    k_phase<T, D, G, U>(Kc, lo, hi, i_cyc, n - 1, k_new, qr, sl, rows_cap, mx);
+    k_phase<T, D, G, U>(Kc, lo, hi, st, n - 1, k_new, qr, sl, rows_cap, mx);
     block_reduce<G>(mx, red, true);  // includes the barrier that publishes sl
 
     // ---- e = 2^(s - max), local sum
@@ -127,7 +127,7 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
             ps += p;
         }
         const int lam = lo + j;
-        const int ph = phys_row(lam, i_cyc);
+        const int ph = phys_row(lam, st);
         const float s_old = (lam == n - 1) ? 0.f : Sc[ph];
         Sc[ph] = s_old + ps * (1.0f / G);
         if (lam == n - 1) Pc[ph] = N;
@@ -135,7 +135,7 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
     __syncthreads();
 
     // ---- V phase: o = sum_j p_j v_j over this CTA's rows
-    v_phase<T, D, G, U>(Vc, lo, hi, i_cyc, n - 1, v_new, sl, rows_cap, o_warp, o_part);
+    v_phase<T, D, G, U>(Vc, lo, hi, st, n - 1, v_new, sl, rows_cap, o_warp, o_part);
 
     cluster.sync();  // (B) partial outputs, the appended row and every S update of the unit are complete
 
@@ -145,20 +145,21 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
             for (int rr = 0; rr < nsplit; ++rr) r += cluster.map_shared_rank(o_part, rr)[t];
             out[((size_t)b * cv.Hq + kh * G) * D + t] = Elem<T>::from_float(r);
         }
-        // ---- Algorithm 1, "length > c" branch: scope {idx, idx+1} = physical rows (2i, 2i+1)
+        // ---- Algorithm 1, "length > c" branch: scope {idx, idx+1} = physical rows (a + i, a + i + 1), survivor to row a
         if (warp == 0) {
             const int N1 = N + 1;
             if (N1 > cv.c) {
-                const int l = 2 * i_cyc, r = l + 1;
+                const int l = st.a + i_cyc, r = l + 1;
                 int evict_right = 0;
                 if (lane == 0) {
                     bool near_tie = false;
-                    evict_right = pair_evicts_right(__ldcg(Sc + l), N1 - __ldcg(Pc + l), __ldcg(Sc + r), N1 - __ldcg(Pc + r),
-                                                    cv.rule, &near_tie) ? 1 : 0;
+                    const int w0 = cv.w0[unit];
+                    evict_right = pair_evicts_right(__ldcg(Sc + l), score_count(N1, __ldcg(Pc + l), w0), __ldcg(Sc + r),
+                                                    score_count(N1, __ldcg(Pc + r), w0), cv.rule, &near_tie) ? 1 : 0;
                     if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
                 }
                 evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
-                const int src = evict_right ? l : r, dst = i_cyc;
+                const int src = evict_right ? l : r, dst = st.a;
                 if (src != dst) {
                     for (int e = lane; e < CHUNKS; e += 32) {
                         const uint4 kk = __ldcg(reinterpret_cast<const uint4*>(Kc + (size_t)src * D) + e);
@@ -169,10 +170,43 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
                     if (lane == 0) { Sc[dst] = __ldcg(Sc + src); Pc[dst] = __ldcg(Pc + src); }
                 }
             }
-            if (lane == 0) cv.n_seen[unit] = N1;
         }
     }
-    cluster.sync();  // (C) keep shared memory alive until CTA 0 has read it
+    cluster.sync();  // (C) keep shared memory alive until CTA 0 has read it; the survivor's move is complete
+    // ---- end of a cycle with a protected recent window: the nr rows behind the last pair move down next to the
+    //      middle region (see common.cuh), in rounds of "read into registers / cluster barrier / write"
+    if (N + 1 > cv.c && cv.nr > 0 && i_cyc == cv.cm - 1) {
+        constexpr int PER = 4;
+        const int src0 = cv.ns + 2 * cv.cm, dst0 = cv.ns + cv.cm, nmove = cv.nr;
+        const int gw = rank * kDecodeWarps + warp, nw_all = nsplit * kDecodeWarps;
+        for (int r0 = 0; r0 < nmove; r0 += nw_all * PER) {
+            uint4 kr[PER], vr[PER];
+            float sr[PER];
+            int32_t pr[PER];
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int it = r0 + u * nw_all + gw;
+                if (it >= nmove) continue;
+                if (lane < CHUNKS) {
+                    kr[u] = __ldcg(reinterpret_cast<const uint4*>(Kc + (size_t)(src0 + it) * D) + lane);
+                    vr[u] = __ldcg(reinterpret_cast<const uint4*>(Vc + (size_t)(src0 + it) * D) + lane);
+                }
+                if (lane == 0) { sr[u] = __ldcg(Sc + src0 + it); pr[u] = __ldcg(Pc + src0 + it); }
+            }
+            cluster.sync();
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int it = r0 + u * nw_all + gw;
+                if (it >= nmove) continue;
+                if (lane < CHUNKS) {
+                    reinterpret_cast<uint4*>(Kc + (size_t)(dst0 + it) * D)[lane] = kr[u];
+                    reinterpret_cast<uint4*>(Vc + (size_t)(dst0 + it) * D)[lane] = vr[u];
+                }
+                if (lane == 0) { Sc[dst0 + it] = sr[u]; Pc[dst0 + it] = pr[u]; }
+            }
+        }
+    }
+    if (rank == 0 && tid == 0) cv.n_seen[unit] = N + 1;
 }
 
 size_t decode_smem_bytes(int G, int D, int c, int split) {

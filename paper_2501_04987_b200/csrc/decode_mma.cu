@@ -150,12 +150,12 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         int Ns;
         asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(Ns) : "l"(cv.n_seen + unit));
         if (Ns >= 0) {
-            const UnitState ss = unit_state(Ns, cv.c);
+            const UnitState ss = unit_state(Ns, cv);
             const int blk_all = (ss.L + 1 + kBlk - 1) / kBlk, per = (blk_all + nsplit - 1) / nsplit;
             const int lo_s = min(rank * per * kBlk, ss.L), hi_s = min(min(lo_s + per * kBlk, ss.L), lo_s + kPrefetchRows);
             const unsigned char* Kb = reinterpret_cast<const unsigned char*>(cv.K) + (size_t)unit * cv.R * ROWB;
             const unsigned char* Vb = reinterpret_cast<const unsigned char*>(cv.V) + (size_t)unit * cv.R * ROWB;
-            const int a1 = min(hi_s, max(lo_s, ss.i));  // live indices [lo_s, a1) sit at row = index, [a1, hi_s) at index + i
+            const int a1 = min(hi_s, max(lo_s, ss.a));  // live indices [lo_s, a1) sit at row = index, [a1, hi_s) at index + i
             if (a1 > lo_s) {
                 l2_prefetch(Kb + (size_t)lo_s * ROWB, (uint32_t)(a1 - lo_s) * ROWB);
                 l2_prefetch(Vb + (size_t)lo_s * ROWB, (uint32_t)(a1 - lo_s) * ROWB);
@@ -174,9 +174,11 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     if (nsplit > 1) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 
     const int N = cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
+    const UnitState st = unit_state(N, cv);
     const int n = st.L + 1;  // live rows including the token appended by this step
     const int i_cyc = st.i;
+    const int a_cyc = st.a;          // live indices below it sit at row = index, the others at index + i_cyc
+    const int row_l = a_cyc + i_cyc; // the scope {idx, idx+1} is physical rows (row_l, row_l + 1); the survivor moves to a_cyc
     // rows are dealt to the cluster in whole 16-key blocks
     const int nblk_all = (n + kBlk - 1) / kBlk;
     const int blk_per = (nblk_all + nsplit - 1) / nsplit;
@@ -207,9 +209,9 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
             const uint32_t kst = ring_w + stage * STAGE, vst = kst + kBlk * ROWB;
             const int lam0 = lo + blk * kBlk;
             // fast path: all 16 rows exist, none is the new token, and they are consecutive physical rows
-            const bool whole = (lam0 + kBlk <= hi) && (lam0 + kBlk <= n - 1) && (lam0 >= i_cyc || lam0 + kBlk <= i_cyc);
+            const bool whole = (lam0 + kBlk <= hi) && (lam0 + kBlk <= n - 1) && (lam0 >= a_cyc || lam0 + kBlk <= a_cyc);
             if (whole) {
-                const size_t r0 = (size_t)phys_row(lam0, i_cyc) + c_rsub * ITERS;
+                const size_t r0 = (size_t)phys_row(lam0, st) + c_rsub * ITERS;
                 const unsigned char* ks = reinterpret_cast<const unsigned char*>(Kc) + r0 * ROWB + c_cidx * 16;
                 const unsigned char* vs = reinterpret_cast<const unsigned char*>(Vc) + r0 * ROWB + c_cidx * 16;
 #pragma unroll
@@ -224,7 +226,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
                     const int row = c_rsub * ITERS + it;
                     const int lam = lam0 + row;
                     const bool valid = lam < hi && lam != n - 1;  // the new token is merged separately
-                    const size_t ro = valid ? (size_t)phys_row(lam, i_cyc) * ROWB : 0;
+                    const size_t ro = valid ? (size_t)phys_row(lam, st) * ROWB : 0;
                     const uint32_t off = c_lane_off + it * ROWB + ((c_cidx ^ (c_row7 + it)) << 4);
                     cp_async_16_stream(kst + off, reinterpret_cast<const unsigned char*>(Kc) + ro + c_cidx * 16, valid, stream_policy);
                     cp_async_16_stream(vst + off, reinterpret_cast<const unsigned char*>(Vc) + ro + c_cidx * 16, valid, stream_policy);
@@ -235,22 +237,23 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     };
     // ---- prefetch what the epilogue needs, so that after the streaming loop nothing waits on a global load:
     //      S of this CTA's rows (4-byte cp.async; they join the first commit group), and in CTA 0 the K/V rows of
-    //      the eviction scope (rows 2i and 2i+1; the new token's row comes from k_in / v_in)
+    //      the eviction scope (rows row_l and row_l + 1; the new token's row comes from k_in / v_in)
     const bool will_evict = (N + 1 > cv.c);
-    int pos_l = 0, pos_r = 0;  // stream positions of the scope's two tokens (used by lane 0 of warp 0 in CTA 0)
+    int pos_l = 0, pos_r = 0, w0 = 0;  // stream positions of the scope's two tokens (used by lane 0 of warp 0 in CTA 0)
     if (rank == 0 && will_evict && tid == 0) {
-        pos_l = Pc[2 * i_cyc];
-        pos_r = (2 * i_cyc + 1 == new_row) ? N : Pc[2 * i_cyc + 1];
+        pos_l = Pc[row_l];
+        pos_r = (row_l + 1 == new_row) ? N : Pc[row_l + 1];
+        w0 = cv.w0[unit];
     }
     for (int j = tid; j < nrows; j += NT) {
         const int lam = lo + j;
         if (lam != n - 1)
-            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(s_old + j)), "l"(Sc + phys_row(lam, i_cyc)) : "memory");
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(s_old + j)), "l"(Sc + phys_row(lam, st)) : "memory");
     }
     if (rank == 0 && will_evict && warp == NW - 1) {
         for (int e = lane; e < 4 * CPR; e += 32) {
             const int which = e / CPR, cidx = e % CPR;   // 0: K left, 1: K right, 2: V left, 3: V right
-            const int prow = 2 * i_cyc + (which & 1);
+            const int prow = row_l + (which & 1);
             if (prow == new_row) continue;  // the appended row is taken from the staged inputs below
             const T* srcrow = ((which < 2) ? Kc : Vc) + (size_t)prow * D;
             cp_async_16(smem_u32(pair_kv + which * ROWB + cidx * 16), reinterpret_cast<const unsigned char*>(srcrow) + cidx * 16, true);
@@ -273,7 +276,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
                 reinterpret_cast<uint4*>(Vc + (size_t)new_row * D)[e] = reinterpret_cast<const uint4*>(tv)[e];
             }
         }
-        if (rank == 0 && will_evict && new_row == 2 * i_cyc + 1) {  // the scope's right row is the appended one
+        if (rank == 0 && will_evict && new_row == row_l + 1) {  // the scope's right row is the appended one
             for (int e = lane; e < CHUNKS; e += 32) {
                 reinterpret_cast<uint4*>(pair_kv + 1 * ROWB)[e] = reinterpret_cast<const uint4*>(tk)[e];
                 reinterpret_cast<uint4*>(pair_kv + 3 * ROWB)[e] = reinterpret_cast<const uint4*>(tv)[e];
@@ -472,7 +475,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     };
     if (nsplit > 1) {
         if (will_evict && tid < 2) {
-            const int lam = i_cyc + tid;  // live indices of physical rows 2i and 2i+1
+            const int lam = a_cyc + tid;  // live indices of the scope's physical rows
             if (lam >= lo && lam < hi) cluster.map_shared_rank(pair_s, 0)[tid] = updated_score(lam - lo);
         }
         __syncwarp();
@@ -495,16 +498,16 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     //      rows of the scope are left to the eviction below, which writes the survivor's score to its new row.
 #pragma unroll 8
     for (int j = tid; j < ncached; j += NT) {
-        const int ph = phys_row(lo + j, i_cyc);
+        const int ph = phys_row(lo + j, st);
         const float s_new = updated_score(j);
-        if (!(will_evict && (ph >> 1) == i_cyc)) Sc[ph] = s_new;
-        else if (nsplit == 1) pair_s[ph & 1] = s_new;  // a single CTA takes the scope's scores from its own loop
+        if (!(will_evict && (unsigned)(ph - row_l) < 2u)) Sc[ph] = s_new;
+        else if (nsplit == 1) pair_s[ph - row_l] = s_new;  // a single CTA takes the scope's scores from its own loop
     }
     if (owns_new && tid == NT - 1) {
         Pc[new_row] = N;
         const float s_new = updated_score(ncached);
-        if (!(will_evict && (new_row >> 1) == i_cyc)) Sc[new_row] = s_new;
-        else if (nsplit == 1) pair_s[new_row & 1] = s_new;
+        if (!(will_evict && (unsigned)(new_row - row_l) < 2u)) Sc[new_row] = s_new;
+        else if (nsplit == 1) pair_s[new_row - row_l] = s_new;
     }
 
     // (B) the scope's scores have arrived in CTA 0
@@ -512,27 +515,63 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     else __syncthreads();
 
     if (rank == 0 && warp == 0 && will_evict) {
-        // ---- Algorithm 1, "length > c" branch: scope {idx, idx+1} = physical rows (2i, 2i+1)
+        // ---- Algorithm 1, "length > c" branch: scope {idx, idx+1} = physical rows (row_l, row_l + 1)
         const int N1 = N + 1;
-        const int l = 2 * i_cyc, r = l + 1;
+        const int l = row_l, r = l + 1;
         int evict_right = 0;
         if (lane == 0) {
             bool near_tie = false;
             const float S_l = pair_s[0], S_r = pair_s[1];
-            evict_right = pair_evicts_right(S_l, N1 - pos_l, S_r, N1 - pos_r, cv.rule, &near_tie) ? 1 : 0;
+            evict_right = pair_evicts_right(S_l, score_count(N1, pos_l, w0), S_r, score_count(N1, pos_r, w0), cv.rule, &near_tie) ? 1 : 0;
             if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
             const int src = evict_right ? l : r;
-            Sc[i_cyc] = evict_right ? S_l : S_r;  // also when the survivor stays in place: the score update skipped the scope
-            Pc[i_cyc] = evict_right ? pos_l : pos_r;
+            Sc[a_cyc] = evict_right ? S_l : S_r;  // also when the survivor stays in place: the score update skipped the scope
+            Pc[a_cyc] = evict_right ? pos_l : pos_r;
         }
         evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
-        const int src = evict_right ? l : r, dst = i_cyc;
+        const int src = evict_right ? l : r, dst = a_cyc;
         if (src != dst) {  // survivor's K and V rows were staged in shared memory at kernel start
             const unsigned char* ksrc = pair_kv + (evict_right ? 0 : 1) * ROWB;
             const unsigned char* vsrc = pair_kv + (evict_right ? 2 : 3) * ROWB;
             for (int e = lane; e < CHUNKS; e += 32) {
                 reinterpret_cast<uint4*>(Kc + (size_t)dst * D)[e] = reinterpret_cast<const uint4*>(ksrc)[e];
                 reinterpret_cast<uint4*>(Vc + (size_t)dst * D)[e] = reinterpret_cast<const uint4*>(vsrc)[e];
+            }
+        }
+    }
+    // ---- end of a cycle with a protected recent window: the nr rows behind the last pair move down next to the
+    //      middle region, so that the next cycle starts from a contiguous cache.  Once per c_mid steps.  The whole
+    //      cluster takes part, in rounds of "read into registers / cluster barrier / write": a destination row can
+    //      be a source row of the same round when the window is longer than the middle region, never of a later one.
+    if (will_evict && cv.nr > 0 && i_cyc == cv.cm - 1) {
+        if (nsplit > 1) cluster.sync(); else __syncthreads();  // every S, pos and appended row of the unit is visible
+        constexpr int PER = 4;                 // rows per warp and round
+        const int src0 = cv.ns + 2 * cv.cm, dst0 = cv.ns + cv.cm, nmove = cv.nr;
+        const int gw = rank * NW + warp, nw_all = nsplit * NW;
+        for (int r0 = 0; r0 < nmove; r0 += nw_all * PER) {
+            uint4 kr[PER], vr[PER];
+            float sr[PER];
+            int32_t pr[PER];
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int it = r0 + u * nw_all + gw;
+                if (it >= nmove) continue;
+                if (lane < CHUNKS) {
+                    kr[u] = __ldcg(reinterpret_cast<const uint4*>(Kc + (size_t)(src0 + it) * D) + lane);
+                    vr[u] = __ldcg(reinterpret_cast<const uint4*>(Vc + (size_t)(src0 + it) * D) + lane);
+                }
+                if (lane == 0) { sr[u] = __ldcg(Sc + src0 + it); pr[u] = __ldcg(Pc + src0 + it); }
+            }
+            if (nsplit > 1) cluster.sync(); else __syncthreads();
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                const int it = r0 + u * nw_all + gw;
+                if (it >= nmove) continue;
+                if (lane < CHUNKS) {
+                    reinterpret_cast<uint4*>(Kc + (size_t)(dst0 + it) * D)[lane] = kr[u];
+                    reinterpret_cast<uint4*>(Vc + (size_t)(dst0 + it) * D)[lane] = vr[u];
+                }
+                if (lane == 0) { Sc[dst0 + it] = sr[u]; Pc[dst0 + it] = pr[u]; }
             }
         }
     }

@@ -72,7 +72,7 @@ extern "C" treekv_status treekv_prefill_chunk_static_scratch(treekv_ctx* ctx, co
         lens.m[b] = (uint16_t)m;
         if (m > max_m) max_m = m;
         if (m > 0) {
-            const int ns = evict_segment(ctx->n_seen[b], m, ctx->cv.c, 0).nseg;
+            const int ns = evict_segment(ctx->n_seen[b], m, ctx->cv, 0).nseg;
             if (ns > max_seg) max_seg = ns;
         }
     }
@@ -83,10 +83,13 @@ extern "C" treekv_status treekv_prefill_chunk_static_scratch(treekv_ctx* ctx, co
     PrefillScratch ps;
     ps.QT = (max_m * ctx->G + kQTileRows - 1) / kQTileRows;
     ps.n_max = ctx->cv.c + max_m;
-    ps.max_chunk = max_m;
+    // rows in flight at once: the survivors of a segment, or after a wrap the rows behind the last pair (the
+    // protected recent tokens and what is still above budget), which can be more than the chunk itself
+    const int stage_rows = max_m + ctx->cv.nr;
+    ps.max_chunk = stage_rows;
     const size_t b_col = up256(units * ps.QT * ps.n_max * sizeof(float));
-    const size_t b_row = up256(units * max_m * ctx->cv.d * ctx->elem);
-    const size_t b_scalar = up256(units * max_m * 4);
+    const size_t b_row = up256(units * stage_rows * ctx->cv.d * ctx->elem);
+    const size_t b_scalar = up256(units * stage_rows * 4);
     if (b_col + 2 * b_row + 2 * b_scalar > kStaticScratchBytes) return TREEKV_ERR_UNSUPPORTED;  // beyond the 16 MiB limit
     if (prefill_simt_smem_bytes(ctx->G, ctx->cv.d, ps.n_max) > 227 * 1024) return TREEKV_ERR_UNSUPPORTED;
     void* base_v = nullptr;
@@ -118,7 +121,7 @@ extern "C" treekv_status treekv_prefill_chunk_static_scratch(treekv_ctx* ctx, co
         int max_items = 0;
         for (int b = 0; b < ctx->cv.B; ++b) {
             if (!lens.m[b]) continue;
-            const EvictSegment sg = evict_segment(ctx->n_seen[b], lens.m[b], ctx->cv.c, seg);
+            const EvictSegment sg = evict_segment(ctx->n_seen[b], lens.m[b], ctx->cv, seg);
             if (sg.E + sg.rebase > max_items) max_items = sg.E + sg.rebase;
         }
         e = launch_chunk_evict(ctx->cv, ctx->dt, ps, lens, seg, max_items, s);

@@ -22,7 +22,7 @@ prefill_simt_kernel(CacheView cv, PrefillScratch ps, const T* __restrict__ q, T*
     if (t0 >= m) return;
     const int t1 = min(t0 + TOK, m);
     const int N = cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
+    const UnitState st = unit_state(N, cv);
     const int n = st.L + m;
     const int rows_cap = ps.n_max;
 
@@ -53,7 +53,7 @@ prefill_simt_kernel(CacheView cv, PrefillScratch ps, const T* __restrict__ q, T*
             for (int e = 0; e < VEC; ++e) qr[h][e] *= scale;
         }
         float mx[G];
-        k_phase<T, D, G, U>(Kc, 0, n_vis, st.i, -1, nullptr, qr, sl, rows_cap, mx);
+        k_phase<T, D, G, U>(Kc, 0, n_vis, st, -1, nullptr, qr, sl, rows_cap, mx);
         block_reduce<G>(mx, red, true);
         float sum[G];
 #pragma unroll
@@ -78,7 +78,7 @@ prefill_simt_kernel(CacheView cv, PrefillScratch ps, const T* __restrict__ q, T*
             col[j] += psum;  // same thread owns column j for every token: fixed summation order
         }
         __syncthreads();
-        v_phase<T, D, G, U>(Vc, 0, n_vis, st.i, -1, nullptr, sl, rows_cap, o_warp, o_part);
+        v_phase<T, D, G, U>(Vc, 0, n_vis, st, -1, nullptr, sl, rows_cap, o_warp, o_part);
         __syncthreads();
         for (int e = tid; e < G * D; e += kDecodeThreads)
             out[(((size_t)b * chunk_stride + t) * cv.Hq + kh * G) * D + e] = Elem<T>::from_float(o_part[e]);

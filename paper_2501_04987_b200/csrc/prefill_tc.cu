@@ -53,11 +53,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (t0 >= m) return;
     const int t1 = min(t0 + TOK, m);
     const int N = cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
-    KeyTiles kt;
-    kt.i = st.i; kt.L = st.L; kt.nvis = st.L + t1;
-    kt.nA = (st.i + 127) / 128;
-    kt.NT = kt.nA + (kt.nvis - st.i + 127) / 128;
+    const UnitState st = unit_state(N, cv);
+    const KeyTiles kt = key_tiles(st, st.L + t1);
     const int NT = kt.NT;
     const int n = st.L + m;
 

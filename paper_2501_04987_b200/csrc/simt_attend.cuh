@@ -40,7 +40,7 @@ __device__ inline void block_reduce(float (&v)[N], float* scratch /*[kDecodeWarp
 // to sl[h * rows_cap + (lam - lo)]; per-thread running maxima in mx.  qr holds this lane's slice of q, already
 // scaled.  Live index `special` (or -1) is read from special_row with plain loads instead of from the slab.
 template <typename T, int D, int G, int U>
-__device__ inline void k_phase(const T* Kc, int lo, int hi, int i_cyc, int special, const T* special_row,
+__device__ inline void k_phase(const T* Kc, int lo, int hi, const UnitState& st, int special, const T* special_row,
                                const float (&qr)[G][Elem<T>::kVec], float* sl, int rows_cap, float (&mx)[G]) {
     constexpr int VEC = Elem<T>::kVec;
     constexpr int LPR = D / VEC;
@@ -57,7 +57,7 @@ __device__ inline void k_phase(const T* Kc, int lo, int hi, int i_cyc, int speci
             raw[u] = make_uint4(0, 0, 0, 0);
             if (lam < hi) {
                 if (lam == special) raw[u] = ld_plain(reinterpret_cast<const uint4*>(special_row) + sub);
-                else raw[u] = ld_stream(reinterpret_cast<const uint4*>(Kc + (size_t)phys_row(lam, i_cyc) * D) + sub);
+                else raw[u] = ld_stream(reinterpret_cast<const uint4*>(Kc + (size_t)phys_row(lam, st) * D) + sub);
             }
         }
 #pragma unroll
@@ -85,7 +85,7 @@ __device__ inline void k_phase(const T* Kc, int lo, int hi, int i_cyc, int speci
 // [kDecodeWarps][G][D] scratch.  Contains one barrier; o_part is complete for the threads that wrote it only
 // after the caller's next barrier.
 template <typename T, int D, int G, int U>
-__device__ inline void v_phase(const T* Vc, int lo, int hi, int i_cyc, int special, const T* special_row,
+__device__ inline void v_phase(const T* Vc, int lo, int hi, const UnitState& st, int special, const T* special_row,
                                const float* sl, int rows_cap, float* o_warp, float* o_part) {
     constexpr int VEC = Elem<T>::kVec;
     constexpr int LPR = D / VEC;
@@ -105,7 +105,7 @@ __device__ inline void v_phase(const T* Vc, int lo, int hi, int i_cyc, int speci
             raw[u] = make_uint4(0, 0, 0, 0);
             if (lam < hi) {
                 if (lam == special) raw[u] = ld_plain(reinterpret_cast<const uint4*>(special_row) + sub);
-                else raw[u] = ld_stream(reinterpret_cast<const uint4*>(Vc + (size_t)phys_row(lam, i_cyc) * D) + sub);
+                else raw[u] = ld_stream(reinterpret_cast<const uint4*>(Vc + (size_t)phys_row(lam, st) * D) + sub);
             }
         }
 #pragma unroll

@@ -10,7 +10,7 @@ namespace treekv {
 // ---------------------------------------------------------------------------------------------------------
 __global__ void init_state_kernel(CacheView cv) {
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t < cv.B * cv.Hkv) cv.n_seen[t] = 0;
+    if (t < cv.B * cv.Hkv) { cv.n_seen[t] = 0; cv.w0[t] = 0; }
     if (t == 0) { cv.stats->near_ties = 0ull; cv.stats->error = 0u; cv.stats->pad = 0u; }
 }
 cudaError_t launch_init_state(const CacheView& cv, cudaStream_t stream) {
@@ -24,10 +24,10 @@ cudaError_t launch_init_state(const CacheView& cv, cudaStream_t stream) {
 __global__ void retained_positions_kernel(CacheView cv, int32_t* pos_out, int32_t* count_out) {
     const int unit = blockIdx.x;
     const int N = cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
+    const UnitState st = unit_state(N, cv);
     const int32_t* Pc = cv.pos + (size_t)unit * cv.R;
     for (int lam = threadIdx.x; lam < cv.c; lam += blockDim.x)
-        pos_out[(size_t)unit * cv.c + lam] = lam < st.L ? Pc[phys_row(lam, st.i)] : -1;
+        pos_out[(size_t)unit * cv.c + lam] = lam < st.L ? Pc[phys_row(lam, st)] : -1;
     if (threadIdx.x == 0) count_out[unit] = st.L;
 }
 cudaError_t launch_retained_positions(const CacheView& cv, int32_t* pos_out, int32_t* count_out, cudaStream_t stream) {
@@ -38,14 +38,14 @@ cudaError_t launch_retained_positions(const CacheView& cv, int32_t* pos_out, int
 __global__ void scores_kernel(CacheView cv, float* sbar_out) {
     const int unit = blockIdx.x;
     const int N = cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
+    const UnitState st = unit_state(N, cv);
     const int32_t* Pc = cv.pos + (size_t)unit * cv.R;
     const float* Sc = cv.S + (size_t)unit * cv.R;
     for (int lam = threadIdx.x; lam < cv.c; lam += blockDim.x) {
         float r = 0.f;
         if (lam < st.L) {
-            const int ph = phys_row(lam, st.i);
-            r = __fdiv_rn(Sc[ph], (float)(N - Pc[ph]));  // Algorithm 1: S-bar = S / C with C = tokens seen - position
+            const int ph = phys_row(lam, st);
+            r = __fdiv_rn(Sc[ph], (float)score_count(N, Pc[ph], cv.w0[unit]));  // Algorithm 1: S-bar = S / C
         }
         sbar_out[(size_t)unit * cv.c + lam] = r;
     }
@@ -65,13 +65,13 @@ __global__ void state_image_kernel(CacheView cv, StateImage img) {
     const int lam = blockIdx.x * (blockDim.x >> 5) + warp;
     if (lam >= cv.c) return;
     const int N = kImport ? img.seen[b] : cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
+    const UnitState st = unit_state(N, cv);
     const int chunks = cv.d * (int)sizeof(T) / 16;
     const size_t slot = (size_t)unit * cv.c + lam;
     uint4* ki = reinterpret_cast<uint4*>(reinterpret_cast<T*>(img.K) + slot * cv.d);
     uint4* vi = reinterpret_cast<uint4*>(reinterpret_cast<T*>(img.V) + slot * cv.d);
     if (lam < st.L) {
-        const size_t row = (size_t)unit * cv.R + phys_row(lam, st.i);
+        const size_t row = (size_t)unit * cv.R + phys_row(lam, st);
         uint4* kc = reinterpret_cast<uint4*>(reinterpret_cast<T*>(cv.K) + row * cv.d);
         uint4* vc = reinterpret_cast<uint4*>(reinterpret_cast<T*>(cv.V) + row * cv.d);
         if (kImport) {
@@ -119,7 +119,7 @@ __global__ void chunk_append_kernel(CacheView cv, const T* __restrict__ k, const
     const int t = blockIdx.x * (blockDim.x >> 5) + warp;
     if (t >= m) return;
     const int N = cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
+    const UnitState st = unit_state(N, cv);
     const int row = st.L + st.i + t;
     const int chunks = cv.d * (int)sizeof(T) / 16;
     const uint4* ks = reinterpret_cast<const uint4*>(k + (((size_t)b * chunk_stride + t) * cv.Hkv + kh) * cv.d);
@@ -153,7 +153,7 @@ __global__ void chunk_scores_kernel(CacheView cv, PrefillScratch ps, ChunkLens l
     if (m == 0) return;
     const int G = cv.Hq / cv.Hkv;
     const int N = cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
+    const UnitState st = unit_state(N, cv);
     const int n = st.L + m;
     const int lam = blockIdx.x * blockDim.x + threadIdx.x;
     if (lam >= n) return;
@@ -161,7 +161,7 @@ __global__ void chunk_scores_kernel(CacheView cv, PrefillScratch ps, ChunkLens l
     const float* part = ps.colsum + (size_t)unit * ps.QT * ps.n_max + lam;
     float s = 0.f;
     for (int t = 0; t < qt; ++t) s += part[(size_t)t * ps.n_max];
-    float* Sp = cv.S + (size_t)unit * cv.R + phys_row(lam, st.i);
+    float* Sp = cv.S + (size_t)unit * cv.R + phys_row(lam, st);
     *Sp = *Sp + s * (1.0f / (float)G);  // chunk rows were zeroed by the append
 }
 cudaError_t launch_chunk_scores(const CacheView& cv, const PrefillScratch& ps, const ChunkLens& lens, int max_m,
@@ -175,7 +175,7 @@ cudaError_t launch_chunk_scores(const CacheView& cv, const PrefillScratch& ps, c
 // ---------------------------------------------------------------------------------------------------------
 // Chunk eviction, one segment (see EvictSegment).  Algorithm 1's "length > c" branch repeated with frozen
 // averaged scores: between two wraps of idx the scopes are disjoint, so all pairs of a segment are decided
-// at once.  The survivor of pair p must land on row i+p, which can be a source row of an earlier pair, so the
+// at once.  The survivor of pair p must land on row ns+i+p, which can be a source row of an earlier pair, so the
 // move goes through staging rows: gather (decide + copy out), then scatter (copy in) as a second launch.
 template <typename T>
 __global__ void chunk_evict_gather_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int seg) {
@@ -186,7 +186,7 @@ __global__ void chunk_evict_gather_kernel(CacheView cv, PrefillScratch ps, Chunk
     const int m = lens.m[b];
     if (m == 0) return;
     const int N = cv.n_seen[unit];
-    const EvictSegment sg = evict_segment(N, m, cv.c, seg);
+    const EvictSegment sg = evict_segment(N, m, cv, seg);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int item = blockIdx.x * (blockDim.x >> 5) + warp;
     if (item >= sg.E + sg.rebase) return;
@@ -197,17 +197,19 @@ __global__ void chunk_evict_gather_kernel(CacheView cv, PrefillScratch ps, Chunk
     const int32_t* Pc = cv.pos + (size_t)unit * cv.R;
     int src;
     if (item < sg.E) {
-        const int l = 2 * (sg.i + item), r = l + 1;
+        const int l = cv.ns + 2 * (sg.i + item), r = l + 1;
         int evict_right = 0;
         if (lane == 0) {
             bool near_tie = false;
-            evict_right = pair_evicts_right(Sc[l], N1 - Pc[l], Sc[r], N1 - Pc[r], cv.rule, &near_tie) ? 1 : 0;
+            const int w0 = cv.w0[unit];
+            evict_right = pair_evicts_right(Sc[l], score_count(N1, Pc[l], w0), Sc[r], score_count(N1, Pc[r], w0), cv.rule,
+                                            &near_tie) ? 1 : 0;
             if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
         }
         evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
         src = evict_right ? l : r;
     } else {
-        src = 2 * cv.c + (item - sg.E);
+        src = cv.ns + 2 * cv.cm + (item - sg.E);
     }
     const int chunks = cv.d * (int)sizeof(T) / 16;
     const size_t so = ((size_t)unit * ps.max_chunk + item);
@@ -228,11 +230,11 @@ __global__ void chunk_evict_scatter_kernel(CacheView cv, PrefillScratch ps, Chun
     const int m = lens.m[b];
     if (m == 0) return;
     const int N = cv.n_seen[unit];
-    const EvictSegment sg = evict_segment(N, m, cv.c, seg);
+    const EvictSegment sg = evict_segment(N, m, cv, seg);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int item = blockIdx.x * (blockDim.x >> 5) + warp;
     if (item >= sg.E + sg.rebase) return;
-    const int dst = item < sg.E ? sg.i + item : cv.c + (item - sg.E);
+    const int dst = cv.ns + (item < sg.E ? sg.i + item : cv.cm + (item - sg.E));
     const int chunks = cv.d * (int)sizeof(T) / 16;
     const size_t so = ((size_t)unit * ps.max_chunk + item);
     const uint4* ks = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(ps.stage_K) + so * cv.d);
@@ -288,9 +290,10 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
     const int rank = (int)cluster.block_rank();
     const int G = cv.Hq / cv.Hkv;
     const int N = cv.n_seen[unit];
-    const UnitState st = unit_state(N, cv.c);
+    const UnitState st = unit_state(N, cv);
     const int n = st.L + m;
     const int N1 = N + m;
+    const int w0 = cv.w0[unit];
     T* Kc = reinterpret_cast<T*>(cv.K) + (size_t)unit * cv.R * cv.d;
     T* Vc = reinterpret_cast<T*>(cv.V) + (size_t)unit * cv.R * cv.d;
     float* Sc = cv.S + (size_t)unit * cv.R;
@@ -305,7 +308,7 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
             const float* part = ps.colsum + (size_t)unit * ps.QT * ps.n_max + lam;
             float s = 0.f;
             for (int t = 0; t < qt; ++t) s += part[(size_t)t * ps.n_max];
-            float* Sp = Sc + phys_row(lam, st.i);
+            float* Sp = Sc + phys_row(lam, st);
             *Sp = *Sp + s * inv_g;  // chunk rows were zeroed by the append
         }
     }
@@ -318,9 +321,9 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
     constexpr int kWarps = kEvictCluster * kEvictThreads / 32;
     constexpr int kRound = kWarps * kEvictItemsPerWarp;
     const int chunks = cv.d * (int)sizeof(T) / 16;  // 16-byte pieces per row: at most 32
-    const int nseg = evict_segment(N, m, cv.c, 0).nseg;
+    const int nseg = evict_segment(N, m, cv, 0).nseg;
     for (int seg = 0; seg < nseg; ++seg) {
-        const EvictSegment sg = evict_segment(N, m, cv.c, seg);
+        const EvictSegment sg = evict_segment(N, m, cv, seg);
         const int items = sg.E + sg.rebase;
         for (int r0 = 0; r0 < items; r0 += kRound) {
             uint4 kr[kEvictItemsPerWarp], vr[kEvictItemsPerWarp];
@@ -332,17 +335,18 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
                 if (item >= items) continue;
                 int src;
                 if (item < sg.E) {
-                    const int l = 2 * (sg.i + item), r = l + 1;
+                    const int l = cv.ns + 2 * (sg.i + item), r = l + 1;
                     int evict_right = 0;
                     if (lane == 0) {
                         bool near_tie = false;
-                        evict_right = pair_evicts_right(Sc[l], N1 - Pc[l], Sc[r], N1 - Pc[r], cv.rule, &near_tie) ? 1 : 0;
+                        evict_right = pair_evicts_right(Sc[l], score_count(N1, Pc[l], w0), Sc[r], score_count(N1, Pc[r], w0),
+                                                        cv.rule, &near_tie) ? 1 : 0;
                         if (near_tie) atomicAdd(&cv.stats->near_ties, 1ull);
                     }
                     evict_right = __shfl_sync(0xffffffffu, evict_right, 0);
                     src = evict_right ? l : r;
                 } else {
-                    src = 2 * cv.c + (item - sg.E);
+                    src = cv.ns + 2 * cv.cm + (item - sg.E);
                 }
                 if (lane < chunks) {
                     kr[u] = reinterpret_cast<const uint4*>(Kc + (size_t)src * cv.d)[lane];
@@ -355,7 +359,7 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
             for (int u = 0; u < kEvictItemsPerWarp; ++u) {
                 const int item = r0 + u * kWarps + gwarp;
                 if (item >= items) continue;
-                const int dst = item < sg.E ? sg.i + item : cv.c + (item - sg.E);
+                const int dst = cv.ns + (item < sg.E ? sg.i + item : cv.cm + (item - sg.E));
                 if (lane < chunks) {
                     reinterpret_cast<uint4*>(Kc + (size_t)dst * cv.d)[lane] = kr[u];
                     reinterpret_cast<uint4*>(Vc + (size_t)dst * cv.d)[lane] = vr[u];

@@ -126,3 +126,32 @@ def step_prefill(kv, orc, q, k, v, dtype, rep, chunk_lens=None, check_scores=Tru
     rep.max_out_err = max(rep.max_out_err, err)
     assert err <= OUT_TOL[dtype], "attention output off by %.3g (tolerance %.3g)" % (err, OUT_TOL[dtype])
     compare_state(kv, orc, rep, check_scores)
+
+
+def _workloads():
+    import workloads
+
+    return workloads
+
+
+def run_decode(kv, orc, w, t0, steps, rep, score_every=1, starts=None):
+    blk = 256
+    done = 0
+    while done < steps:
+        n = min(blk, steps - done)
+        st = [t0 + done] * w.batch if starts is None else [s + done for s in starts]
+        q, k, v = _workloads().tokens_at(w, 0, st, n)
+        for i in range(n):
+            step_decode(kv, orc, q[i], k[i], v[i], w.dtype, rep, check_scores=((done + i) % score_every == 0))
+        done += n
+
+
+def run_prefill(kv, orc, w, rep, lens_total, chunk, method="prefill_chunk"):
+    """Feed sequence b its first lens_total[b] tokens in chunks of `chunk` (ragged at the end)."""
+    lens_total = np.asarray(lens_total)
+    n_calls = int((lens_total.max() + chunk - 1) // chunk)
+    for c in range(n_calls):
+        q, k, v = _workloads().tokens(w, 0, c * chunk, (c + 1) * chunk)
+        lens = np.clip(lens_total - c * chunk, 0, chunk)
+        step_prefill(kv, orc, q.transpose(1, 0, 2, 3), k.transpose(1, 0, 2, 3), v.transpose(1, 0, 2, 3), w.dtype, rep,
+                     chunk_lens=lens, method=method)

@@ -8,6 +8,7 @@ import pytest
 
 import workloads as W
 from lockstep import Report, compare_state, step_decode, step_prefill
+from lockstep import run_decode as _run_decode, run_prefill as _run_prefill
 
 pytestmark = pytest.mark.gpu
 
@@ -33,29 +34,6 @@ def _pair(binding, w, max_chunk=None):
     kv = binding.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, mc)
     orc = Oracle(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.batch)
     return kv, orc
-
-
-def _run_decode(kv, orc, w, t0, steps, rep, score_every=1, starts=None):
-    blk = 256
-    done = 0
-    while done < steps:
-        n = min(blk, steps - done)
-        st = [t0 + done] * w.batch if starts is None else [s + done for s in starts]
-        q, k, v = W.tokens_at(w, 0, st, n)
-        for i in range(n):
-            step_decode(kv, orc, q[i], k[i], v[i], w.dtype, rep, check_scores=((done + i) % score_every == 0))
-        done += n
-
-
-def _run_prefill(kv, orc, w, rep, lens_total, chunk):
-    """Feed sequence b its first lens_total[b] tokens in chunks of `chunk` (ragged at the end)."""
-    lens_total = np.asarray(lens_total)
-    n_calls = int((lens_total.max() + chunk - 1) // chunk)
-    for c in range(n_calls):
-        q, k, v = W.tokens(w, 0, c * chunk, (c + 1) * chunk)
-        lens = np.clip(lens_total - c * chunk, 0, chunk)
-        step_prefill(kv, orc, q.transpose(1, 0, 2, 3), k.transpose(1, 0, 2, 3), v.transpose(1, 0, 2, 3), w.dtype, rep,
-                     chunk_lens=lens)
 
 
 # ---------------------------------------------------------------------------------------------------------
