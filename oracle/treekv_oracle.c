@@ -39,7 +39,23 @@
  *     n_recent newest (it is then the last slot of the middle region, exactly where Algorithm 1 appends).  S and
  *     C of every cached token, protected or not, advance as in Algorithm 1 from the token's arrival.  With
  *     n_sink = n_recent = 0 this is Algorithm 1 unchanged.
- *   PARITY UNPINNED: the last three readings are not fixed by anything the paper
+ *   - one-shot, block-level prefill (Section 4.2): the prompt is cut into blocks of b tokens, "each block
+ *     representing one token" of Algorithm 1; the last block is the observation window whose b queries score the
+ *     whole prompt: Algorithm 1's S and C updates are applied for those b rows only, so a token older than the
+ *     window has C = b and window token u (0-based) has C = b - u; a block's score is the mean of its tokens'
+ *     S/C; Algorithm 1's branch then runs on blocks with a cache of c / b blocks, blocks arriving in order.  The
+ *     output is plain causal attention over the whole prompt.  Afterwards the token-level pointer is the first
+ *     token of the block the block pointer stands on, idx = (idx_blocks - 1) b + 1, which equals
+ *     (tokens evicted mod c) + 1.  The paper gives neither b nor the treatment of a ragged tail: the prompt
+ *     length and c must be multiples of b here.  S and C carry on into decoding as they are.
+ *   - in-cache positions (Section 4.1 "Position Encoding"): positional encodings are re-assigned after eviction,
+ *     i.e. the token in cache slot j (0-based) is encoded at position j and the query at its own slot.  With
+ *     this switched on, q and k arrive WITHOUT positional encoding, the cache keeps k as given, and attention
+ *     applies rotary embedding (rotate-half pairing (t, t + d/2)) from a cos / sin table indexed by slot.  The
+ *     numeric contract follows the paper's "bf16 precision" set-up: the rotated q and k are computed in fp32 as
+ *     x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin) and rounded to the cache's element type before
+ *     the fp64 dot product (no rounding for an fp32 cache).
+ *   PARITY UNPINNED: the last five readings are not fixed by anything the paper
  *   prints; the tests constrain them (m=1 equals a decode step, mass
  *   conservation, score-free rules give identical retained sets) but cannot
  *   pin them to the paper.
@@ -67,6 +83,11 @@ typedef struct {
 typedef struct {
     int c, Hq, Hkv, d, B, g;
     int n_sink, n_recent; /* protected tokens at both ends (Section 5.2); 0, 0 = Algorithm 1 as printed */
+    /* in-cache positions (Section 4.1 "Position Encoding"): rotary tables by slot, NULL = position-agnostic */
+    const float *rope_cos, *rope_sin; /* [rope_slots][d/2], owned by the caller */
+    int rope_slots, rope_round_bf16;
+    /* block-level eviction pending after tkvo_prefill_oneshot_attend */
+    int *pending_block; /* [B], 0 = none */
     int rule, idx_mode;
     int64_t *n_seen;    /* [B] */
     int64_t *n_evicted; /* [B] */
@@ -105,6 +126,7 @@ tkvo *tkvo_create(int budget, int n_heads, int n_kv_heads, int head_dim, int bat
     o->idx = (int *)malloc(sizeof(int) * (size_t)batch);
     for (int b = 0; b < batch; ++b) o->idx[b] = 1;
     o->u = (tkvo_unit *)calloc((size_t)batch * n_kv_heads, sizeof(tkvo_unit));
+    o->pending_block = (int *)calloc((size_t)batch, sizeof(int));
     o->last_min_gap = INFINITY;
     return o;
 }
@@ -114,7 +136,7 @@ void tkvo_destroy(tkvo *o) {
     for (int i = 0; i < o->B * o->Hkv; ++i) {
         free(o->u[i].K); free(o->u[i].V); free(o->u[i].S); free(o->u[i].C); free(o->u[i].pos);
     }
-    free(o->u); free(o->n_seen); free(o->n_evicted); free(o->idx); free(o);
+    free(o->u); free(o->n_seen); free(o->n_evicted); free(o->idx); free(o->pending_block); free(o);
 }
 
 void tkvo_set_rule(tkvo *o, int rule) { o->rule = rule; }
@@ -145,15 +167,51 @@ static void append_token(tkvo *o, int b, const double *k, const double *v) {
     o->n_seen[b] += 1;
 }
 
+/* Section 4.1 "Position Encoding": in-cache positions.  Tables by slot; cos/sin are single-precision inputs. */
+int tkvo_set_rope(tkvo *o, const float *cos_tab, const float *sin_tab, int slots, int round_bf16) {
+    if (o->d % 2 || o->d > 512) return -1;
+    o->rope_cos = cos_tab; o->rope_sin = sin_tab; o->rope_slots = cos_tab ? slots : 0; o->rope_round_bf16 = round_bf16;
+    return 0;
+}
+
+static float round_to_bf16(float x) { /* round to nearest even to 8 significand bits, kept in a float */
+    uint32_t u;
+    memcpy(&u, &x, 4);
+    if ((u & 0x7f800000u) == 0x7f800000u) return x;
+    u += 0x7fffu + ((u >> 16) & 1u);
+    u &= 0xffff0000u;
+    memcpy(&x, &u, 4);
+    return x;
+}
+
+/* x (an element-type value held in a double) rotated to slot `slot`: pairs (t, t + d/2), two single-precision
+ * operations per output, then rounded to the cache's element type. */
+static void rope_row(const tkvo *o, const double *x, int slot, double *y) {
+    const int half = o->d / 2;
+    const float *cs = o->rope_cos + (size_t)slot * half, *sn = o->rope_sin + (size_t)slot * half;
+    for (int t = 0; t < half; ++t) {
+        const float x1 = (float)x[t], x2 = (float)x[t + half];
+        volatile float p1 = x2 * sn[t], p2 = x1 * sn[t]; /* each product rounded to single precision */
+        float y1 = fmaf(x1, cs[t], -p1), y2 = fmaf(x2, cs[t], p2);
+        if (o->rope_round_bf16) { y1 = round_to_bf16(y1); y2 = round_to_bf16(y2); }
+        y[t] = (double)y1; y[t + half] = (double)y2;
+    }
+}
+
 /* One query row against one unit: a = SoftMax(q K^T / sqrt(d)) over the first
- * n_vis slots (Section 3.1), out = a V.  a is returned in prob[0..n_vis). */
-static void attend_row(const tkvo *o, const tkvo_unit *u, const double *q, int n_vis, double *prob, double *out) {
+ * n_vis slots (Section 3.1), out = a V.  a is returned in prob[0..n_vis).
+ * With in-cache positions the query is encoded at slot n_vis - 1 (its own) and key j at slot j. */
+static void attend_row(const tkvo *o, const tkvo_unit *u, const double *q_in, int n_vis, double *prob, double *out) {
     const int d = o->d;
     const double inv = 1.0 / sqrt((double)d);
     double mx = -INFINITY;
+    double qbuf[512], kbuf[512];
+    const double *q = q_in;
+    if (o->rope_cos) { rope_row(o, q_in, n_vis - 1, qbuf); q = qbuf; }
     for (int j = 0; j < n_vis; ++j) {
         double s = 0.0;
         const double *kj = u->K + (size_t)j * d;
+        if (o->rope_cos) { rope_row(o, kj, j, kbuf); kj = kbuf; }
         for (int t = 0; t < d; ++t) s += q[t] * kj[t];
         s *= inv;
         prob[j] = s;
@@ -254,6 +312,131 @@ static int in_sorted(const int32_t *a, int n, int64_t x) {
     int lo = 0, hi = n;
     while (lo < hi) { int mid = (lo + hi) / 2; if (a[mid] < x) lo = mid + 1; else hi = mid; }
     return lo < n && a[lo] == x;
+}
+
+/*
+ * One-shot prefill, first half (Section 4.2): the whole prompt of lens[b] tokens enters an empty cache, every
+ * row attends causally (the output is plain attention over the prompt), and the last `block` rows - the
+ * observation window - advance S and C of every token they see (Algorithm 1's two update lines, for those
+ * rows only).  lens[b] must be a multiple of `block`; sequences with lens[b] = 0 are skipped.
+ * Returns 0, or -1 on a bad argument / non-empty cache.
+ */
+int tkvo_prefill_oneshot_attend(tkvo *o, const double *q, const double *k, const double *v, double *out,
+                                const int32_t *lens, int stride, int block) {
+    const int d = o->d, g = o->g;
+    if (block < 1 || o->c % block || o->n_sink || o->n_recent) return -1;
+    for (int b = 0; b < o->B; ++b)
+        if (lens[b] < 0 || lens[b] > stride || lens[b] % block || (lens[b] && o->n_seen[b])) return -1;
+    for (int b = 0; b < o->B; ++b) {
+        for (int i = 0; i < lens[b]; ++i) {
+            const size_t row = (size_t)b * stride + i;
+            append_token(o, b, k + row * o->Hkv * d, v + row * o->Hkv * d);
+        }
+        if (lens[b]) o->pending_block[b] = block;
+    }
+#pragma omp parallel for schedule(dynamic)
+    for (int bu = 0; bu < o->B * o->Hkv; ++bu) {
+        const int b = bu / o->Hkv, kh = bu % o->Hkv;
+        const int T = lens[b];
+        if (T <= 0) continue;
+        tkvo_unit *u = &o->u[bu];
+        double *prob = (double *)malloc(sizeof(double) * (size_t)T);
+        double *acc = (double *)calloc((size_t)T, sizeof(double));
+        for (int i = 0; i < T; ++i) {
+            const int in_window = (i >= T - block);
+            for (int hh = 0; hh < g; ++hh) {
+                const int h = kh * g + hh;
+                const size_t qo = (((size_t)b * stride + i) * o->Hq + h) * d;
+                attend_row(o, u, q + qo, i + 1, prob, out + qo);
+                if (in_window) for (int j = 0; j <= i; ++j) acc[j] += prob[j];
+            }
+            if (in_window) for (int j = 0; j <= i; ++j) u->C[j] += 1; /* Alg. 1: C <- C + 1, window rows only */
+        }
+        for (int j = 0; j < T; ++j) u->S[j] += acc[j] / (double)g;    /* Alg. 1: S <- S + a, group mean */
+        free(prob); free(acc);
+    }
+    return 0;
+}
+
+/*
+ * One-shot prefill, second half (Section 4.2, "Block-level Eviction"): a block's score is the mean of its
+ * tokens' S / C; blocks enter a cache of c / block blocks in order and Algorithm 1's "length > c" branch plays
+ * on blocks.  Near-ties and hints as in tkvo_evict (a block is "in the hint" when its first token is).
+ */
+void tkvo_evict_blocks(tkvo *o, const int32_t *hint_pos, const int32_t *hint_cnt, double near_tie_tol) {
+    o->last_near_ties = 0; o->last_hint_flips = 0; o->last_min_gap = INFINITY;
+    const int c = o->c, d = o->d;
+    for (int b = 0; b < o->B; ++b) {
+        const int bs = o->pending_block[b];
+        if (!bs) continue;
+        o->pending_block[b] = 0;
+        const int T = o->u[b * o->Hkv].len, nb = T / bs, cb = c / bs;
+        int idx_end = 1;
+        for (int kh = 0; kh < o->Hkv; ++kh) {
+            tkvo_unit *u = &o->u[b * o->Hkv + kh];
+            double *score = (double *)malloc(sizeof(double) * (size_t)nb);
+            for (int kb = 0; kb < nb; ++kb) { /* averaged importance of the b tokens of the block */
+                double a = 0.0;
+                for (int t = 0; t < bs; ++t) a += u->S[kb * bs + t] / (double)u->C[kb * bs + t];
+                score[kb] = a / (double)bs;
+            }
+            int *cache = (int *)malloc(sizeof(int) * (size_t)(cb + 1)); /* block numbers, in order */
+            int len = 0, idx = 1;
+            for (int kb = 0; kb < nb; ++kb) {
+                cache[len++] = kb; /* the block arrives */
+                if (len > cb) {
+                    const int l = idx - 1, r = idx;
+                    int evict_right;
+                    if (o->rule == TKVO_RULE_KEEP_LEFT) evict_right = 1;
+                    else if (o->rule == TKVO_RULE_EVICT_LEFT) evict_right = 0;
+                    else {
+                        const double sl = score[cache[l]], sr = score[cache[r]];
+                        evict_right = (sl > sr); /* Alg. 1: strict > */
+                        const double mxabs = fmax(fabs(sl), fabs(sr));
+                        const double gap = mxabs > 0.0 ? fabs(sl - sr) / mxabs : 0.0;
+                        if (gap < o->last_min_gap) o->last_min_gap = gap;
+                        if (gap < near_tie_tol) {
+                            o->last_near_ties += 1;
+                            if (hint_pos) {
+                                const int32_t *hp = hint_pos + ((size_t)b * o->Hkv + kh) * c;
+                                const int hn = hint_cnt[b * o->Hkv + kh];
+                                const int lin = in_sorted(hp, hn, u->pos[cache[l] * bs]);
+                                const int rin = in_sorted(hp, hn, u->pos[cache[r] * bs]);
+                                if (lin != rin) {
+                                    const int want = lin ? 1 : 0;
+                                    if (want != evict_right) { evict_right = want; o->last_hint_flips += 1; }
+                                }
+                            }
+                        }
+                    }
+                    const int gone = evict_right ? r : l;
+                    memmove(cache + gone, cache + gone + 1, sizeof(int) * (size_t)(len - gone - 1));
+                    len -= 1;
+                    idx = (idx % cb) + 1;
+                }
+            }
+            /* keep the tokens of the surviving blocks, in order */
+            int w = 0;
+            for (int s = 0; s < len; ++s) {
+                for (int t = 0; t < bs; ++t, ++w) {
+                    const int src = cache[s] * bs + t;
+                    if (src == w) continue;
+                    memcpy(u->K + (size_t)w * d, u->K + (size_t)src * d, sizeof(double) * d);
+                    memcpy(u->V + (size_t)w * d, u->V + (size_t)src * d, sizeof(double) * d);
+                    u->S[w] = u->S[src]; u->C[w] = u->C[src]; u->pos[w] = u->pos[src];
+                }
+            }
+            u->len = w;
+            idx_end = idx;
+            free(score); free(cache);
+        }
+        if (T > c) {
+            o->n_evicted[b] += T - c;
+            o->idx[b] = (idx_end - 1) * bs + 1; /* the first token of the block the block pointer stands on */
+        }
+    }
+    o->total_near_ties += o->last_near_ties;
+    o->total_hint_flips += o->last_hint_flips;
 }
 
 /*

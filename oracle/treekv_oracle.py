@@ -28,7 +28,7 @@ def build_oracle(force: bool = False) -> str:
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + ".%d.tmp" % os.getpid()
         subprocess.check_call(
-            ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-o", tmp, _SRC, "-lm"]
+            ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fPIC", "-shared", "-fopenmp", "-o", tmp, _SRC, "-lm"]
         )
         os.replace(tmp, _LIB)
     return _LIB
@@ -56,6 +56,12 @@ def _load():
         getattr(lib, name).restype = None
     lib.tkvo_evict.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_double]
     lib.tkvo_evict.restype = None
+    lib.tkvo_evict_blocks.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_double]
+    lib.tkvo_evict_blocks.restype = None
+    lib.tkvo_prefill_oneshot_attend.argtypes = [vp, dp, dp, dp, dp, C.POINTER(C.c_int32), C.c_int, C.c_int]
+    lib.tkvo_prefill_oneshot_attend.restype = C.c_int
+    lib.tkvo_set_rope.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_int, C.c_int]
+    lib.tkvo_set_rope.restype = C.c_int
     lib.tkvo_len.argtypes = [vp, C.c_int, C.c_int]
     lib.tkvo_len.restype = C.c_int
     for name in ("tkvo_n_seen", "tkvo_n_evicted"):
@@ -146,6 +152,57 @@ class Oracle:
             hc = hint_cnt.ctypes.data_as(C.POINTER(C.c_int32))
         self._lib.tkvo_evict(self._h, hp, hc, float(near_tie_tol))
         return self.last_near_ties, self.last_hint_flips
+
+    def _hints(self, hint_pos, hint_cnt):
+        hp = hc = None
+        if hint_pos is not None:
+            hint_pos = np.ascontiguousarray(hint_pos, dtype=np.int32)
+            hint_cnt = np.ascontiguousarray(hint_cnt, dtype=np.int32)
+            assert hint_pos.shape == (self.B, self.Hkv, self.c) and hint_cnt.shape == (self.B, self.Hkv)
+            hp = hint_pos.ctypes.data_as(C.POINTER(C.c_int32))
+            hc = hint_cnt.ctypes.data_as(C.POINTER(C.c_int32))
+        return hp, hc, hint_pos, hint_cnt
+
+    # ---- Section 4.2: one-shot, block-level prefill of an empty cache
+    def prefill_oneshot_attend(self, q, k, v, block, lens=None):
+        q = np.ascontiguousarray(q, dtype=np.float64)
+        stride = q.shape[1]
+        q = _f64(q, (self.B, stride, self.Hq, self.d))
+        k = _f64(k, (self.B, stride, self.Hkv, self.d))
+        v = _f64(v, (self.B, stride, self.Hkv, self.d))
+        if lens is None:
+            lens = [stride] * self.B
+        cl = np.ascontiguousarray(lens, dtype=np.int32)
+        out = np.zeros_like(q)
+        rc = self._lib.tkvo_prefill_oneshot_attend(self._h, _dp(q), _dp(k), _dp(v), _dp(out),
+                                                   cl.ctypes.data_as(C.POINTER(C.c_int32)), stride, int(block))
+        if rc != 0:
+            raise ValueError("one-shot prefill needs an empty, unprotected cache and lengths / budget that are multiples of the block")
+        return out
+
+    def evict_blocks(self, hint_pos=None, hint_cnt=None, near_tie_tol=1e-4):
+        hp, hc, _a, _b = self._hints(hint_pos, hint_cnt)
+        self._lib.tkvo_evict_blocks(self._h, hp, hc, float(near_tie_tol))
+        return self.last_near_ties, self.last_hint_flips
+
+    def prefill_oneshot(self, q, k, v, block, lens=None):
+        out = self.prefill_oneshot_attend(q, k, v, block, lens)
+        self.evict_blocks()
+        return out
+
+    # ---- Section 4.1 "Position Encoding": in-cache positions
+    def set_rope(self, cos, sin, round_bf16):
+        """cos, sin: float32 [slots, d/2] tables by cache slot (kept alive by this object); None switches it off."""
+        if cos is None:
+            self._rope = None
+            self._lib.tkvo_set_rope(self._h, None, None, 0, 0)
+            return
+        cos = np.ascontiguousarray(cos, dtype=np.float32); sin = np.ascontiguousarray(sin, dtype=np.float32)
+        assert cos.shape == sin.shape and cos.shape[1] == self.d // 2
+        self._rope = (cos, sin)
+        fp = C.POINTER(C.c_float)
+        assert self._lib.tkvo_set_rope(self._h, cos.ctypes.data_as(fp), sin.ctypes.data_as(fp), cos.shape[0],
+                                       1 if round_bf16 else 0) == 0
 
     def decode_step(self, q, k, v, active=None):
         out = self.decode_attend(q, k, v, active)
