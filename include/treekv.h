@@ -130,6 +130,24 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
                                    void* stream);
 
 /*
+ * One-shot, block-level prefill of an empty cache (Section 4.2): the whole prompt of host_lens[b] tokens is attended
+ * causally (dev_out = plain attention over the prompt), the last `block` tokens are the observation window whose
+ * queries alone score the prompt (Algorithm 1's S and C updates for those rows: a token older than the window gets
+ * C = block, window token u gets C = block - u), a block's importance is the mean of its tokens' S / C, and
+ * Algorithm 1's eviction branch runs on blocks of `block` tokens - each block standing for one token of Figure 3 - with
+ * a cache of budget / block blocks.  Afterwards the cache holds min(prompt, budget) tokens in whole blocks, and decode
+ * steps or chunks continue from there (the eviction pointer stands on the first token of the block the block pointer
+ * reached; S and C carry on).  The paper fixes neither `block` nor a ragged tail: prompt lengths and the budget must be
+ * multiples of `block` (TREEKV_ERR_INVALID_ARG otherwise).
+ *   dev_q, dev_out  [batch][stride][n_heads][head_dim]     dev_k, dev_v  [batch][stride][n_kv_heads][head_dim]
+ *   host_lens       [batch] int32 in 0..min(stride, max_chunk), 0 = sequence not in this call; NULL = all `stride`
+ * Sequences in the call must not have seen a token yet (TREEKV_ERR_BAD_STATE); with protected tokens set the call
+ * returns TREEKV_ERR_UNSUPPORTED.  Nothing is enqueued on an error.
+ */
+treekv_status treekv_prefill_oneshot(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v,
+                                     void* dev_out, const int32_t* host_lens, int stride, int block, void* stream);
+
+/*
  * The same two calls with HOST tensors (pageable or page-locked), all enqueued on `stream`: host_out is valid,
  * and the host inputs may be reused, once the stream has been synchronised.  Shapes as above.
  * treekv_decode_step_host: when all four tensors are page-locked memory the GPU can address (cudaHostAlloc /
@@ -195,11 +213,13 @@ treekv_status treekv_scores(treekv_ctx* ctx, float* dev_sbar, void* stream);
 /*
  * State image: everything Algorithm 1 carries from one step to the next, in cache order, so that a context of the
  * same shape can continue the stream elsewhere or later (the paper has no counterpart; idx and the counters C follow
- * from the tokens seen and the stored positions).  Layout of the image, each part starting on a 256-byte boundary:
+ * from the tokens seen, the stored positions and the scoring start).  Layout of the image, each part starting on a 256-byte boundary:
  *   K   [batch][n_kv_heads][budget][head_dim]  dtype     V    the same
  *   S   [batch][n_kv_heads][budget] float (sums, not averages)      pos  [batch][n_kv_heads][budget] int32
- *   tokens seen [batch] int32
- * Slots beyond a sequence's cache length are zero (pos: -1).
+ *   tokens seen [batch] int32                                       scoring start [batch] int32 (0 unless the
+ *                                                                   sequence was prefilled in one shot)
+ * Slots beyond a sequence's cache length are zero (pos: -1).  The protected-token setting is not part of the image:
+ * the importing context must have the same one.
  * treekv_export_state enqueues the copy and writes the host-side token counts to host_tokens_seen[batch] before
  * returning; treekv_import_state replaces the context's state by the image (enqueued on `stream`) and takes the
  * same counts back - they must be the ones exported with the image.

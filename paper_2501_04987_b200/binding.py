@@ -25,7 +25,7 @@ EXPORTS = [
     "treekv_get_stats", "treekv_tokens_seen", "treekv_set_rule", "treekv_set_option", "treekv_reset",
     "treekv_destroy", "treekv_status_string", "treekv_version",
     "treekv_state_bytes", "treekv_export_state", "treekv_import_state", "treekv_selftest_wait_giveup",
-    "treekv_set_protection",
+    "treekv_set_protection", "treekv_prefill_oneshot",
 ]
 
 
@@ -93,6 +93,8 @@ def _load():
     lib.treekv_export_state.argtypes = [vp, vp, C.POINTER(C.c_int64), vp]
     lib.treekv_import_state.restype = i32
     lib.treekv_import_state.argtypes = [vp, vp, C.POINTER(C.c_int64), vp]
+    lib.treekv_prefill_oneshot.restype = i32
+    lib.treekv_prefill_oneshot.argtypes = [vp, vp, vp, vp, vp, C.POINTER(C.c_int32), i32, i32, vp]
     lib.treekv_set_protection.restype = i32
     lib.treekv_set_protection.argtypes = [vp, i32, i32]
     lib.treekv_selftest_wait_giveup.restype = i32
@@ -147,6 +149,10 @@ def treekv_decode_step_host(ctx, q, k, v, out, active=None, stream=0) -> int:
 
 def treekv_prefill_chunk(ctx, q, k, v, out, chunk_lens, chunk_stride, stream=0) -> int:
     return lib.treekv_prefill_chunk(ctx, q, k, v, out, _i32(chunk_lens), chunk_stride, stream)
+
+
+def treekv_prefill_oneshot(ctx, q, k, v, out, lens, stride, block, stream=0) -> int:
+    return lib.treekv_prefill_oneshot(ctx, q, k, v, out, _i32(lens), stride, block, stream)
 
 
 def treekv_prefill_chunk_host(ctx, q, k, v, out, chunk_lens, chunk_stride, stream=0) -> int:
@@ -280,6 +286,17 @@ class TreeKV:
         self._chk(out, (B, stride, Hq, d))
         _check(treekv_prefill_chunk(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), chunk_lens,
                                     stride, self._stream()), "treekv_prefill_chunk")
+        return out
+
+    def prefill_oneshot(self, q, k, v, block, out=None, lens=None):
+        B, Hq, Hkv, d = self.batch, self.n_heads, self.n_kv_heads, self.head_dim
+        stride = q.shape[1]
+        self._chk(q, (B, stride, Hq, d)); self._chk(k, (B, stride, Hkv, d)); self._chk(v, (B, stride, Hkv, d))
+        if out is None:
+            out = self.torch.empty_like(q)
+        self._chk(out, (B, stride, Hq, d))
+        _check(treekv_prefill_oneshot(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lens, stride,
+                                      block, self._stream()), "treekv_prefill_oneshot")
         return out
 
     def prefill_chunk_static_scratch(self, q, k, v, out=None, chunk_lens=None):

@@ -149,7 +149,7 @@ treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_
     ctx->ps.colsum = reinterpret_cast<float*>(base + L.colsum);
     // (rows in flight during compaction stay in registers: the context has no staging rows; PrefillScratch's
     //  staging pointers are only used by the entry point that brings its own scratch)
-    ctx->ps.QT = L.QT; ctx->ps.n_max = L.n_max; ctx->ps.max_chunk = max_chunk;
+    ctx->ps.QT = L.QT; ctx->ps.n_max = L.n_max; ctx->ps.max_chunk = max_chunk; ctx->ps.window = 0;
     ctx->st_q = base + L.st_q; ctx->st_k = base + L.st_k; ctx->st_v = base + L.st_v; ctx->st_out = base + L.st_out;
     ctx->dt = dtype; ctx->max_chunk = max_chunk; ctx->G = n_heads / n_kv_heads;
     ctx->elem = dtype == TREEKV_F32 ? 4 : 2;
@@ -227,6 +227,29 @@ treekv_status decode_step_impl(treekv_ctx* ctx, const void* dev_q, const void* d
     return TREEKV_OK;
 }
 
+// Attention of a chunk over [cache | chunk] with the column sums of its probability matrix (all of the chunk's
+// rows, or the last ps.window tokens): tensor-core kernels for bf16 / head_dim 128, CUDA cores otherwise.
+treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, const void* dev_q, void* dev_out,
+                                     const ChunkLens& lens, int chunk_stride, int max_m, cudaStream_t s) {
+    cudaError_t e;
+    if (use_tc_prefill(ctx)) {
+        // q is [batch*chunk_stride tokens][n_heads][128]; a tile is 64 channels x G heads x 128/G tokens
+        CUtensorMap tmQ;
+        const uint64_t dims[3] = {128ull, (uint64_t)ctx->cv.Hq, (uint64_t)ctx->cv.B * (uint64_t)chunk_stride};
+        const uint64_t strides[2] = {256ull, (uint64_t)ctx->cv.Hq * 256ull};
+        const uint32_t box[3] = {64u, (uint32_t)ctx->G, (uint32_t)(128 / ctx->G)};
+        if (!make_tensor_map_bf16(&tmQ, dev_q, 3, dims, strides, box)) return TREEKV_ERR_CUDA;
+        // two query tiles per CTA once the one-tile grid would cover the machine at least twice (or on request)
+        const long tiles = (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + kQTileRows - 1) / kQTileRows);
+        const bool two = ctx->opt_prefill_path == 3 || (ctx->opt_prefill_path == 0 && tiles >= 2L * ctx->sm_count);
+        e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s)
+                : launch_prefill_tc(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s);
+    } else {
+        e = launch_prefill_simt(ctx->cv, ctx->dt, ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
+    }
+    return e == cudaSuccess ? TREEKV_OK : cuda_fail(ctx, e);
+}
+
 }  // namespace
 
 extern "C" {
@@ -256,22 +279,8 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, chunk_stride, max_m, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    if (use_tc_prefill(ctx)) {
-        // q is [batch*chunk_stride tokens][n_heads][128]; a tile is 64 channels x G heads x 128/G tokens
-        CUtensorMap tmQ;
-        const uint64_t dims[3] = {128ull, (uint64_t)ctx->cv.Hq, (uint64_t)ctx->cv.B * (uint64_t)chunk_stride};
-        const uint64_t strides[2] = {256ull, (uint64_t)ctx->cv.Hq * 256ull};
-        const uint32_t box[3] = {64u, (uint32_t)ctx->G, (uint32_t)(128 / ctx->G)};
-        if (!make_tensor_map_bf16(&tmQ, dev_q, 3, dims, strides, box)) return TREEKV_ERR_CUDA;
-        // two query tiles per CTA once the one-tile grid would cover the machine at least twice (or on request)
-        const long tiles = (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + kQTileRows - 1) / kQTileRows);
-        const bool two = ctx->opt_prefill_path == 3 || (ctx->opt_prefill_path == 0 && tiles >= 2L * ctx->sm_count);
-        e = two ? launch_prefill_tc2(ctx->cv, ctx->ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s)
-                : launch_prefill_tc(ctx->cv, ctx->ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s);
-    } else {
-        e = launch_prefill_simt(ctx->cv, ctx->dt, ctx->ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
-    }
-    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    const treekv_status ast = launch_chunk_attention(ctx, ctx->ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
+    if (ast != TREEKV_OK) return ast;
     // score update, all eviction segments and the token counters in one launch
     e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
@@ -282,6 +291,41 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
         const int64_t ev_before = before > ctx->cv.c ? before - ctx->cv.c : 0;
         const int64_t ev_after = ctx->n_seen[b] > ctx->cv.c ? ctx->n_seen[b] - ctx->cv.c : 0;
         ctx->evictions += (uint64_t)(ev_after - ev_before);
+    }
+    return TREEKV_OK;
+}
+
+treekv_status treekv_prefill_oneshot(treekv_ctx* ctx, const void* dev_q, const void* dev_k, const void* dev_v, void* dev_out,
+                                     const int32_t* host_lens, int stride, int block, void* stream) {
+    if (!ctx || !dev_q || !dev_k || !dev_v || !dev_out) return TREEKV_ERR_INVALID_ARG;
+    if (!aligned16(dev_q) || !aligned16(dev_k) || !aligned16(dev_v) || !aligned16(dev_out)) return TREEKV_ERR_INVALID_ARG;
+    if (ctx->max_chunk == 0) return TREEKV_ERR_BAD_STATE;  // decode-only context
+    if (stride < 1 || block < 1 || ctx->cv.c % block) return TREEKV_ERR_INVALID_ARG;
+    if (ctx->cv.ns || ctx->cv.nr) return TREEKV_ERR_UNSUPPORTED;  // block-level eviction with protected tokens is not defined
+    ChunkLens lens;
+    memset(&lens, 0, sizeof(lens));
+    int max_m = 0;
+    for (int b = 0; b < ctx->cv.B; ++b) {
+        const int m = host_lens ? host_lens[b] : stride;
+        if (m < 0 || m > stride || m > ctx->max_chunk || m % block) return TREEKV_ERR_INVALID_ARG;
+        if (m > 0 && ctx->n_seen[b] != 0) return TREEKV_ERR_BAD_STATE;  // the prompt enters an empty cache
+        lens.m[b] = (uint16_t)m;
+        if (m > max_m) max_m = m;
+    }
+    if (max_m == 0) return TREEKV_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, stride, max_m, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    PrefillScratch ps = ctx->ps;
+    ps.window = block;  // only the last block's queries score the prompt
+    const treekv_status ast = launch_chunk_attention(ctx, ps, dev_q, dev_out, lens, stride, max_m, s);
+    if (ast != TREEKV_OK) return ast;
+    e = launch_oneshot_update_evict(ctx->cv, ctx->dt, ps, lens, block, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 3;
+    for (int b = 0; b < ctx->cv.B; ++b) {
+        ctx->n_seen[b] += lens.m[b];
+        if (lens.m[b] > ctx->cv.c) ctx->evictions += (uint64_t)(lens.m[b] - ctx->cv.c);
     }
     return TREEKV_OK;
 }
@@ -355,11 +399,13 @@ static size_t state_image_layout(const treekv_ctx* ctx, void* base, StateImage* 
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
     const size_t oK = take(slots * ctx->cv.d * ctx->elem), oV = take(slots * ctx->cv.d * ctx->elem);
     const size_t oS = take(slots * 4), oP = take(slots * 4), oN = take((size_t)ctx->cv.B * 4);
+    const size_t oW = take((size_t)ctx->cv.B * 4);
     if (img) {
         char* p = static_cast<char*>(base);
         img->K = p + oK; img->V = p + oV;
         img->S = reinterpret_cast<float*>(p + oS); img->pos = reinterpret_cast<int32_t*>(p + oP);
         img->seen = reinterpret_cast<int32_t*>(p + oN);
+        img->w0 = reinterpret_cast<int32_t*>(p + oW);
     }
     return off;
 }

@@ -178,6 +178,8 @@ struct PrefillScratch {
     int QT;           // tiles per unit: ceil(G * max_chunk / 128)
     int n_max;        // c + max_chunk
     int max_chunk;
+    int window;       // 0: every query row of the chunk adds to the column sums (Algorithm 1 per row); > 0: only the
+                      // last `window` tokens of each sequence's chunk do (observation window of the one-shot prefill)
 };
 constexpr int kQTileRows = 128;  // query rows (token x head-in-group) per prefill tile
 
@@ -225,6 +227,7 @@ struct StateImage {
     float* S;
     int32_t* pos;
     int32_t* seen;  // [B]
+    int32_t* w0;    // [B] stream step at which scoring started (0 unless the sequence was prefilled in one shot)
 };
 cudaError_t launch_export_state(const CacheView& cv, treekv_dtype dt, const StateImage& img, cudaStream_t stream);
 cudaError_t launch_import_state(const CacheView& cv, treekv_dtype dt, const StateImage& img, cudaStream_t stream);
@@ -240,6 +243,10 @@ cudaError_t launch_chunk_finalize(const CacheView& cv, const ChunkLens& lens, cu
 // score update + every eviction segment + n_seen update of a chunk in one launch (a cluster per unit)
 cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
                                       cudaStream_t stream);
+
+// one-shot prefill of an empty cache: scores from the observation window, block means, Algorithm 1 on blocks
+cudaError_t launch_oneshot_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
+                                        int block, cudaStream_t stream);
 
 size_t prefill_simt_smem_bytes(int G, int D, int n_max);
 cudaError_t launch_prefill_simt(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const void* q, void* out,

@@ -87,6 +87,7 @@ extern "C" treekv_status treekv_prefill_chunk_static_scratch(treekv_ctx* ctx, co
     // protected recent tokens and what is still above budget), which can be more than the chunk itself
     const int stage_rows = max_m + ctx->cv.nr;
     ps.max_chunk = stage_rows;
+    ps.window = 0;
     const size_t b_col = up256(units * ps.QT * ps.n_max * sizeof(float));
     const size_t b_row = up256(units * stage_rows * ctx->cv.d * ctx->elem);
     const size_t b_scalar = up256(units * stage_rows * 4);

@@ -25,6 +25,7 @@ prefill_simt_kernel(CacheView cv, PrefillScratch ps, const T* __restrict__ q, T*
     const UnitState st = unit_state(N, cv);
     const int n = st.L + m;
     const int rows_cap = ps.n_max;
+    const int wstart = ps.window > 0 ? m - ps.window : 0;  // one-shot prefill: only the observation window scores
 
     const T* Kc = reinterpret_cast<const T*>(cv.K) + (size_t)unit * cv.R * D;
     const T* Vc = reinterpret_cast<const T*>(cv.V) + (size_t)unit * cv.R * D;
@@ -75,7 +76,7 @@ prefill_simt_kernel(CacheView cv, PrefillScratch ps, const T* __restrict__ q, T*
                 sl[h * rows_cap + j] = p;
                 psum += p;
             }
-            col[j] += psum;  // same thread owns column j for every token: fixed summation order
+            if (t >= wstart) col[j] += psum;  // same thread owns column j for every token: fixed summation order
         }
         __syncthreads();
         v_phase<T, D, G, U>(Vc, 0, n_vis, st, -1, nullptr, sl, rows_cap, o_warp, o_part);

@@ -270,6 +270,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         asm volatile("bar.sync 1, 512;" ::: "memory");  // nlse[] is complete
         // ---- pass B: probabilities, column sums, P^T for the tensor cores
         const int rmax = G * (t1 - t0);  // query columns [rmax, 128) are padding
+        // observation window (one-shot prefill): only the last ps.window tokens of the chunk add to the column sums
+        const int rwin = ps.window > 0 ? max(0, G * (m - ps.window - t0)) : 0;
         float* part = ps.colsum + ((size_t)unit * ps.QT + qt) * ps.n_max;
         int puse = 0;  // times this group's P^T buffer has been filled
         for (int j = grp; j < NT && ok; j += 2) {
@@ -283,7 +285,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const bool kvalid = row < valid;
             const int lam = lam0 + row;
             const int rmin = kvalid ? max(0, G * (lam - kt.L - t0)) : 128;  // first query column that sees this key
-            const bool full = __all_sync(0xffffffffu, rmin == 0) && rmax == 128;
+            const bool full = __all_sync(0xffffffffu, rmin == 0) && rmax == 128 && rwin == 0;
             float colsum = 0.f;
             unsigned char* prow = base_ptr + (1 + kRing) * kSlot + grp * kSlot + row * 128;
             auto probs32 = [&](auto full_tag, auto first_tag, const uint32_t (&v)[32], int cg) {
@@ -308,7 +310,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                             }
                         }
                     }
-                    colsum += ((p[0] + p[1]) + (p[2] + p[3])) + ((p[4] + p[5]) + (p[6] + p[7]));
+                    if constexpr (kFull) {
+                        colsum += ((p[0] + p[1]) + (p[2] + p[3])) + ((p[4] + p[5]) + (p[6] + p[7]));
+                    } else {
+                        const int r0 = cg * 32 + q4 * 8;  // columns below rwin belong to queries outside the window
+                        float w[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) w[e] = (r0 + e >= rwin) ? p[e] : 0.f;
+                        colsum += ((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]));
+                    }
                     __nv_bfloat162 t2;
                     t2 = __floats2bfloat162_rn(p[0], p[1]); pk[q4].x = *reinterpret_cast<uint32_t*>(&t2);
                     t2 = __floats2bfloat162_rn(p[2], p[3]); pk[q4].y = *reinterpret_cast<uint32_t*>(&t2);

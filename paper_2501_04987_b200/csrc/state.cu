@@ -86,8 +86,8 @@ __global__ void state_image_kernel(CacheView cv, StateImage img) {
         if (lane == 0) { img.S[slot] = 0.f; img.pos[slot] = -1; }
     }
     if (lam == 0 && lane == 0) {
-        if (kImport) cv.n_seen[unit] = N;
-        else if (unit % cv.Hkv == 0) img.seen[b] = N;
+        if (kImport) { cv.n_seen[unit] = N; cv.w0[unit] = img.w0[b]; }
+        else if (unit % cv.Hkv == 0) { img.seen[b] = N; img.w0[b] = cv.w0[unit]; }
     }
 }
 template <bool kImport>
@@ -379,6 +379,139 @@ cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, cons
     cfg.stream = stream;  // plain stream order behind the attention kernel; the kernel after it may be scheduled early
     if (dt == TREEKV_F32) return cudaLaunchKernelEx(&cfg, chunk_update_evict_kernel<float>, cv, ps, lens);
     return cudaLaunchKernelEx(&cfg, chunk_update_evict_kernel<__nv_bfloat16>, cv, ps, lens);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// One-shot, block-level prefill of an empty cache (Section 4.2 of the paper), the part after the attention: the
+// prompt's m tokens sit in rows [0, m); the attention kernel left the column sums of the observation window (the
+// last `bs` tokens) per query tile.  This kernel adds them to S (Algorithm 1's S update for the window's rows; the
+// counter C of a token is the number of window rows that see it, kept implicitly through w0 = m - bs), then plays
+// Algorithm 1's "length > c" branch on blocks of bs tokens - "each block representing one token": a block's score
+// is the mean of its tokens' S / C, the cache holds c / bs blocks, and the cycle-coordinate layout applies to
+// block rows (block r = token rows [r bs, (r+1) bs)), so that the final token rows are exactly the token-level
+// layout at cycle position ((m - c) mod c).  Per segment: one warp per pair decides (decisions go to the unit's
+// column-sum scratch, free by then), cluster barrier, then the rows move in rounds as in the kernel above.
+template <typename T>
+__global__ void __cluster_dims__(kEvictCluster, 1, 1) __launch_bounds__(kEvictThreads)
+oneshot_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int bs) {
+    pdl_trigger();
+    pdl_wait();
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int unit = blockIdx.y;
+    const int b = unit / cv.Hkv;
+    const int m = lens.m[b];
+    if (m == 0) return;  // the whole cluster shares the unit
+    const int rank = (int)cluster.block_rank();
+    const int G = cv.Hq / cv.Hkv;
+    const int wstart = m - bs;  // first token of the observation window; also the step at which scoring starts
+    T* Kc = reinterpret_cast<T*>(cv.K) + (size_t)unit * cv.R * cv.d;
+    T* Vc = reinterpret_cast<T*>(cv.V) + (size_t)unit * cv.R * cv.d;
+    float* Sc = cv.S + (size_t)unit * cv.R;
+    int32_t* Pc = cv.pos + (size_t)unit * cv.R;
+    float* scratch = ps.colsum + (size_t)unit * ps.QT * ps.n_max;
+
+    // ---- S of every prompt token = group mean of the window's column sums; only the query tiles that hold window
+    //      rows are added, in tile order
+    {
+        const int qt = (m * G + kQTileRows - 1) / kQTileRows;
+        const int tile0 = (wstart * G) / kQTileRows;
+        const float inv_g = 1.0f / (float)G;
+        for (int lam = rank * kEvictThreads + threadIdx.x; lam < m; lam += kEvictCluster * kEvictThreads) {
+            const float* part = scratch + lam;
+            float s = 0.f;
+            for (int t = tile0; t < qt; ++t) s += part[(size_t)t * ps.n_max];
+            Sc[lam] = Sc[lam] + s * inv_g;  // the append left S = 0
+        }
+    }
+    cluster.sync();  // every S of the unit is final, the column sums have been consumed
+    if (rank == 0 && threadIdx.x == 0) { cv.n_seen[unit] = m; cv.w0[unit] = wstart; }
+
+    // ---- Algorithm 1 on blocks
+    CacheView blk = cv;  // geometry in block units: a cache of c / bs blocks, nothing protected
+    blk.c = cv.c / bs; blk.cm = blk.c; blk.ns = 0; blk.nr = 0;
+    const int nb = m / bs, cb = blk.c;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gwarp = rank * (kEvictThreads / 32) + warp;
+    constexpr int kWarps = kEvictCluster * kEvictThreads / 32;
+    constexpr int kRound = kWarps * kEvictItemsPerWarp;
+    const int chunks = cv.d * (int)sizeof(T) / 16;
+    int* dec = reinterpret_cast<int*>(scratch);  // [pairs of the segment] 1 = the right block goes
+    const float inv_bs = 1.0f / (float)bs;
+    auto block_score = [&](int brow) {  // mean of S / C over the block's tokens, summed in a fixed order
+        float a = 0.f;
+        for (int t = lane; t < bs; t += 32) {
+            const int row = brow * bs + t;
+            a += __fdiv_rn(Sc[row], (float)score_count(m, Pc[row], wstart));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        return a * inv_bs;
+    };
+    const int nseg = evict_segment(0, nb, blk, 0).nseg;
+    for (int seg = 0; seg < nseg; ++seg) {
+        const EvictSegment sg = evict_segment(0, nb, blk, seg);
+        for (int p = gwarp; p < sg.E; p += kWarps) {
+            const int lb = 2 * (sg.i + p), rb = lb + 1;
+            const float sl = block_score(lb), sr = block_score(rb);
+            if (lane == 0) {
+                int evict_right;
+                if (cv.rule == TREEKV_RULE_KEEP_LEFT) evict_right = 1;
+                else if (cv.rule == TREEKV_RULE_EVICT_LEFT) evict_right = 0;
+                else {
+                    const float mx = fmaxf(fabsf(sl), fabsf(sr));
+                    if (!(fabsf(sl - sr) >= kNearTieRel * mx)) atomicAdd(&cv.stats->near_ties, 1ull);
+                    evict_right = sl > sr ? 1 : 0;  // strict: ties evict the left (older) block
+                }
+                dec[p] = evict_right;
+            }
+        }
+        cluster.sync();  // the segment's decisions are visible to the whole cluster
+        const int items = (sg.E + sg.rebase) * bs;  // token rows to move
+        for (int r0 = 0; r0 < items; r0 += kRound) {
+            uint4 kr[kEvictItemsPerWarp], vr[kEvictItemsPerWarp];
+            float sr[kEvictItemsPerWarp];
+            int32_t pr[kEvictItemsPerWarp];
+#pragma unroll
+            for (int u = 0; u < kEvictItemsPerWarp; ++u) {
+                const int item = r0 + u * kWarps + gwarp;
+                if (item >= items) continue;
+                const int ib = item / bs, t = item - ib * bs;
+                const int sb = ib < sg.E ? 2 * (sg.i + ib) + (dec[ib] ? 0 : 1) : 2 * cb + (ib - sg.E);
+                const int src = sb * bs + t;
+                if (lane < chunks) {
+                    kr[u] = reinterpret_cast<const uint4*>(Kc + (size_t)src * cv.d)[lane];
+                    vr[u] = reinterpret_cast<const uint4*>(Vc + (size_t)src * cv.d)[lane];
+                }
+                if (lane == 0) { sr[u] = Sc[src]; pr[u] = Pc[src]; }
+            }
+            cluster.sync();  // everything this round moves has been read
+#pragma unroll
+            for (int u = 0; u < kEvictItemsPerWarp; ++u) {
+                const int item = r0 + u * kWarps + gwarp;
+                if (item >= items) continue;
+                const int ib = item / bs, t = item - ib * bs;
+                const int db = ib < sg.E ? sg.i + ib : cb + (ib - sg.E);
+                const int dst = db * bs + t;
+                if (lane < chunks) {
+                    reinterpret_cast<uint4*>(Kc + (size_t)dst * cv.d)[lane] = kr[u];
+                    reinterpret_cast<uint4*>(Vc + (size_t)dst * cv.d)[lane] = vr[u];
+                }
+                if (lane == 0) { Sc[dst] = sr[u]; Pc[dst] = pr[u]; }
+            }
+        }
+        if (seg + 1 < nseg) cluster.sync();  // the next segment's pairs read rows (and overwrite decisions) of this one
+    }
+}
+
+cudaError_t launch_oneshot_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
+                                        int block, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kEvictCluster, cv.B * cv.Hkv);
+    cfg.blockDim = dim3(kEvictThreads);
+    cfg.stream = stream;
+    if (dt == TREEKV_F32) return cudaLaunchKernelEx(&cfg, oneshot_update_evict_kernel<float>, cv, ps, lens, block);
+    return cudaLaunchKernelEx(&cfg, oneshot_update_evict_kernel<__nv_bfloat16>, cv, ps, lens, block);
 }
 
 __global__ void chunk_finalize_kernel(CacheView cv, ChunkLens lens) {

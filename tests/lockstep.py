@@ -128,6 +128,33 @@ def step_prefill(kv, orc, q, k, v, dtype, rep, chunk_lens=None, check_scores=Tru
     compare_state(kv, orc, rep, check_scores)
 
 
+def step_oneshot(kv, orc, q, k, v, block, dtype, rep, lens=None, check_scores=True):
+    """One-shot block-level prefill of empty caches; q [B,T,Hq,d], k,v [B,T,Hkv,d] float32 numpy, dtype-rounded."""
+    import torch
+
+    B, T = q.shape[0], q.shape[1]
+    ls = [T] * B if lens is None else [int(x) for x in lens]
+    out_o = orc.prefill_oneshot_attend(q, k, v, block, ls)
+    out_g = kv.prefill_oneshot(_to_dev(torch, q, kv.tdtype), _to_dev(torch, k, kv.tdtype), _to_dev(torch, v, kv.tdtype),
+                               block, lens=ls)
+    pos_g, cnt_g = kv.retained_positions()
+    ev0 = evicted_total(orc)
+    nt, fl = orc.evict_blocks(pos_g.cpu().numpy(), cnt_g.cpu().numpy(), NEAR_TIE)
+    # decisions are taken per block pair: evicted tokens / block, per KV head
+    after = evicted_total(orc)
+    rep.decisions += (after - ev0) // block * orc.Hkv
+    rep.near_ties += nt; rep.flips += fl; rep.calls += 1
+    assert rep.flips <= rep.near_ties <= rep.decisions or rep.near_ties == 0, repr(rep)
+    og = out_g.float().cpu().numpy().astype(np.float64)
+    err = 0.0
+    for b in range(B):
+        if ls[b]:
+            err = max(err, float(np.abs(og[b, : ls[b]] - out_o[b, : ls[b]]).max()))
+    rep.max_out_err = max(rep.max_out_err, err)
+    assert err <= OUT_TOL[dtype], "attention output off by %.3g (tolerance %.3g)" % (err, OUT_TOL[dtype])
+    compare_state(kv, orc, rep, check_scores)
+
+
 def _workloads():
     import workloads
 
