@@ -21,8 +21,9 @@
  *     passed as void*, NULL = the default stream).
  *   - Tensors are contiguous, 16-byte aligned, element type = the context's
  *     dtype (fp32 or bf16).  q and k arrive with any position encoding already
- *     applied; the library is position-agnostic and records for every cached
- *     token its 0-based stream index.
+ *     applied; the library is position-agnostic (unless treekv_set_positions
+ *     switches in-cache positions on) and records for every cached token its
+ *     0-based stream index.
  *   - Grouped-query attention: query head h uses KV head h / (n_heads /
  *     n_kv_heads); the weight a cached token receives in a step is the mean
  *     over the query heads of its group (equal to Algorithm 1 when the group
@@ -260,6 +261,21 @@ treekv_status treekv_set_rule(treekv_ctx* ctx, treekv_rule rule);
  * (after creation or treekv_reset; else TREEKV_ERR_BAD_STATE).  Host-side only, nothing is enqueued.
  */
 treekv_status treekv_set_protection(treekv_ctx* ctx, int n_sink, int n_recent);
+/*
+ * In-cache positions (Section 4.1 "Position Encoding": positional encodings are re-assigned after eviction - a cache
+ * holding tokens {0,1,2,3,7,8,9} plus the new token is encoded at positions 0..7).  With tables set, q and k must
+ * arrive WITHOUT positional encoding; the cache keeps k as given, and every attention encodes the key in cache
+ * slot j (0-based, cache order) at position j and each query at its own slot (the last slot in a decode step, the
+ * row's slot in a chunk) with rotary embedding, rotate-half pairing (t, t + head_dim/2).
+ *   dev_cos, dev_sin  [slots][head_dim/2] float, device memory, 16-byte aligned, owned by the caller and read by
+ *                     every later call; slots >= budget + max(1, max_chunk).  Both NULL: back to position-agnostic.
+ * Numeric contract: x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin) in fp32, rounded to the context's dtype
+ * before the dot product (the paper's runs are bf16 throughout; an fp32 context does not round).
+ * Only on a context that has not seen a token (TREEKV_ERR_BAD_STATE otherwise).  Attention then runs on the CUDA-core
+ * kernels, which encode while they stream.  Host-side only, nothing is enqueued.
+ */
+treekv_status treekv_set_positions(treekv_ctx* ctx, const float* dev_cos, const float* dev_sin, int slots);
+
 treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value);
 
 /* Back to the empty cache (idx = 1, nothing seen).  Enqueued on `stream`. */

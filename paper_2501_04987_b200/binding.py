@@ -25,7 +25,7 @@ EXPORTS = [
     "treekv_get_stats", "treekv_tokens_seen", "treekv_set_rule", "treekv_set_option", "treekv_reset",
     "treekv_destroy", "treekv_status_string", "treekv_version",
     "treekv_state_bytes", "treekv_export_state", "treekv_import_state", "treekv_selftest_wait_giveup",
-    "treekv_set_protection", "treekv_prefill_oneshot",
+    "treekv_set_protection", "treekv_prefill_oneshot", "treekv_set_positions",
 ]
 
 
@@ -95,6 +95,8 @@ def _load():
     lib.treekv_import_state.argtypes = [vp, vp, C.POINTER(C.c_int64), vp]
     lib.treekv_prefill_oneshot.restype = i32
     lib.treekv_prefill_oneshot.argtypes = [vp, vp, vp, vp, vp, C.POINTER(C.c_int32), i32, i32, vp]
+    lib.treekv_set_positions.restype = i32
+    lib.treekv_set_positions.argtypes = [vp, vp, vp, i32]
     lib.treekv_set_protection.restype = i32
     lib.treekv_set_protection.argtypes = [vp, i32, i32]
     lib.treekv_selftest_wait_giveup.restype = i32
@@ -189,6 +191,10 @@ def treekv_set_rule(ctx, rule) -> int:
 
 def treekv_set_protection(ctx, n_sink, n_recent) -> int:
     return lib.treekv_set_protection(ctx, n_sink, n_recent)
+
+
+def treekv_set_positions(ctx, dev_cos, dev_sin, slots) -> int:
+    return lib.treekv_set_positions(ctx, dev_cos, dev_sin, slots)
 
 
 def treekv_set_option(ctx, opt, value) -> int:
@@ -354,6 +360,19 @@ class TreeKV:
 
     def set_protection(self, n_sink, n_recent):
         _check(treekv_set_protection(self._h, n_sink, n_recent), "treekv_set_protection")
+
+    def set_positions(self, cos, sin):
+        """cos, sin: float32 CUDA tensors [slots, head_dim/2] (kept alive by this object), or None, None."""
+        if cos is None:
+            _check(treekv_set_positions(self._h, None, None, 0), "treekv_set_positions")
+            self._rope = None
+            return
+        t = self.torch
+        if not (cos.is_cuda and cos.is_contiguous() and cos.dtype == t.float32 and sin.shape == cos.shape and sin.is_cuda
+                and sin.is_contiguous() and sin.dtype == t.float32 and cos.shape[1] == self.head_dim // 2):
+            raise ValueError("expected two contiguous float32 CUDA tensors of shape [slots, head_dim/2]")
+        _check(treekv_set_positions(self._h, cos.data_ptr(), sin.data_ptr(), cos.shape[0]), "treekv_set_positions")
+        self._rope = (cos, sin)
 
     def set_option(self, opt, value):
         _check(treekv_set_option(self._h, opt, value), "treekv_set_option")

@@ -71,12 +71,13 @@ treekv_status cuda_fail(treekv_ctx* ctx, cudaError_t e) {
     return TREEKV_ERR_CUDA;
 }
 
+// With in-cache positions the keys are encoded on the fly, which only the CUDA-core kernels do.
 bool use_tc_prefill(const treekv_ctx* ctx) {
-    return ctx->has_tma && ctx->opt_prefill_path != 1;
+    return ctx->has_tma && ctx->opt_prefill_path != 1 && !ctx->cv.rope_cos;
 }
 
 bool use_mma_decode(const treekv_ctx* ctx) {
-    if (ctx->dt != TREEKV_BF16) return false;
+    if (ctx->dt != TREEKV_BF16 || ctx->cv.rope_cos) return false;
     return ctx->opt_decode_path != 1;
 }
 
@@ -146,6 +147,7 @@ treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_
     ctx->cv.c = budget; ctx->cv.R = L.R; ctx->cv.Hq = n_heads; ctx->cv.Hkv = n_kv_heads; ctx->cv.B = batch;
     ctx->cv.d = head_dim; ctx->cv.rule = TREEKV_RULE_SCORES;
     ctx->cv.ns = 0; ctx->cv.nr = 0; ctx->cv.cm = budget;
+    ctx->cv.rope_cos = nullptr; ctx->cv.rope_sin = nullptr;
     ctx->ps.colsum = reinterpret_cast<float*>(base + L.colsum);
     // (rows in flight during compaction stay in registers: the context has no staging rows; PrefillScratch's
     //  staging pointers are only used by the entry point that brings its own scratch)
@@ -474,6 +476,19 @@ treekv_status treekv_set_protection(treekv_ctx* ctx, int n_sink, int n_recent) {
     for (int b = 0; b < ctx->cv.B; ++b)
         if (ctx->n_seen[b] != 0) return TREEKV_ERR_BAD_STATE;  // the layout of a cache in use cannot change
     ctx->cv.ns = n_sink; ctx->cv.nr = n_recent; ctx->cv.cm = ctx->cv.c - n_sink - n_recent;
+    return TREEKV_OK;
+}
+
+treekv_status treekv_set_positions(treekv_ctx* ctx, const float* dev_cos, const float* dev_sin, int slots) {
+    if (!ctx) return TREEKV_ERR_INVALID_ARG;
+    for (int b = 0; b < ctx->cv.B; ++b)
+        if (ctx->n_seen[b] != 0) return TREEKV_ERR_BAD_STATE;  // keys already cached were encoded by the caller
+    if (!dev_cos && !dev_sin) { ctx->cv.rope_cos = nullptr; ctx->cv.rope_sin = nullptr; return TREEKV_OK; }
+    if (!dev_cos || !dev_sin || !aligned16(dev_cos) || !aligned16(dev_sin)) return TREEKV_ERR_INVALID_ARG;
+    // slots in use: 0 .. budget during decode (the query sits in slot budget), 0 .. budget + chunk - 1 during prefill
+    const int need = ctx->cv.c + (ctx->max_chunk > 1 ? ctx->max_chunk : 1);
+    if (slots < need) return TREEKV_ERR_INVALID_ARG;
+    ctx->cv.rope_cos = dev_cos; ctx->cv.rope_sin = dev_sin;
     return TREEKV_OK;
 }
 

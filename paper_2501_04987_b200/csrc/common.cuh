@@ -58,6 +58,8 @@ struct CacheView {
     int ns;           // protected initial tokens (sinks)
     int nr;           // protected newest tokens (recent window)
     int cm;           // c - ns - nr: slots Algorithm 1 runs on = evictions per cycle
+    const float* rope_cos;  // in-cache positions (Section 4.1 "Position Encoding"): cos / sin by cache slot,
+    const float* rope_sin;  // [slots][d/2] fp32, caller-owned; nullptr = the library is position-agnostic
 };
 
 struct ActiveMask {
@@ -161,6 +163,28 @@ __device__ inline bool pair_evicts_right(float S_l, int C_l, float S_r, int C_r,
     *near_tie = !(fabsf(a - b) >= kNearTieRel * mx);
     return a > b;  // strict: ties and NaN evict the left (older) slot
 }
+
+// In-cache positions: x (this lane's slice of a row spread over LPR lanes, VEC elements each) encoded at `slot`.
+// Rotate-half pairing (t, t + d/2): the partner element sits LPR/2 lanes away.  Numeric contract: two fp32
+// operations per output, x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin), then rounding to the cache's
+// element type - as a model that keeps rotated keys in the cache dtype would produce them.  Every lane of the warp
+// must call this (shuffles); `slot` must be a valid table row for every lane.
+#ifdef __CUDACC__
+template <typename T, int D>
+__device__ inline void rope_apply(float (&f)[Elem<T>::kVec], int slot, int sub, const float* cos_tab, const float* sin_tab) {
+    constexpr int VEC = Elem<T>::kVec, LPR = D / VEC, HL = LPR / 2;
+    const bool lower = sub < HL;
+    const float* cs = cos_tab + (size_t)slot * (D / 2) + (sub % HL) * VEC;
+    const float* sn = sin_tab + (size_t)slot * (D / 2) + (sub % HL) * VEC;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+        const float partner = __shfl_xor_sync(0xffffffffu, f[e], HL);
+        const float ps = __fmul_rn(partner, __ldg(sn + e));
+        const float y = __fmaf_rn(f[e], __ldg(cs + e), lower ? -ps : ps);
+        f[e] = Elem<T>::to_float(Elem<T>::from_float(y));
+    }
+}
+#endif
 
 // chunk length of every sequence in a prefill call (0 = not in the call), passed by value
 struct ChunkLens {

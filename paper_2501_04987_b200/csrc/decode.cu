@@ -75,6 +75,7 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
         for (int h = 0; h < G; ++h) {
             const uint4 u = ld_plain(reinterpret_cast<const uint4*>(q + ((size_t)b * cv.Hq + kh * G + h) * D) + sub);
             Elem<T>::unpack(u, qr[h]);
+            if (cv.rope_cos) rope_apply<T, D>(qr[h], n - 1, sub, cv.rope_cos, cv.rope_sin);  // the query sits in the last slot
 #pragma unroll
             for (int e = 0; e < VEC; ++e) qr[h][e] *= scale;
         }
@@ -82,7 +83,7 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
 
     // ---- K phase: logits (in log2 units) of this CTA's rows
     float mx[G];
-    k_phase<T, D, G, U>(Kc, lo, hi, st, n - 1, k_new, qr, sl, rows_cap, mx);
+    k_phase<T, D, G, U>(Kc, lo, hi, st, n - 1, k_new, qr, sl, rows_cap, mx, cv.rope_cos, cv.rope_sin);
     block_reduce<G>(mx, red, true);  // includes the barrier that publishes sl
 
     // ---- e = 2^(s - max), local sum

@@ -50,11 +50,12 @@ prefill_simt_kernel(CacheView cv, PrefillScratch ps, const T* __restrict__ q, T*
             const uint4 u = ld_plain(reinterpret_cast<const uint4*>(
                                          q + (((size_t)b * chunk_stride + t) * cv.Hq + kh * G + h) * D) + sub);
             Elem<T>::unpack(u, qr[h]);
+            if (cv.rope_cos) rope_apply<T, D>(qr[h], n_vis - 1, sub, cv.rope_cos, cv.rope_sin);  // the row's own slot
 #pragma unroll
             for (int e = 0; e < VEC; ++e) qr[h][e] *= scale;
         }
         float mx[G];
-        k_phase<T, D, G, U>(Kc, 0, n_vis, st, -1, nullptr, qr, sl, rows_cap, mx);
+        k_phase<T, D, G, U>(Kc, 0, n_vis, st, -1, nullptr, qr, sl, rows_cap, mx, cv.rope_cos, cv.rope_sin);
         block_reduce<G>(mx, red, true);
         float sum[G];
 #pragma unroll

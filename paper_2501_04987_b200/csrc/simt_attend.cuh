@@ -41,7 +41,8 @@ __device__ inline void block_reduce(float (&v)[N], float* scratch /*[kDecodeWarp
 // scaled.  Live index `special` (or -1) is read from special_row with plain loads instead of from the slab.
 template <typename T, int D, int G, int U>
 __device__ inline void k_phase(const T* Kc, int lo, int hi, const UnitState& st, int special, const T* special_row,
-                               const float (&qr)[G][Elem<T>::kVec], float* sl, int rows_cap, float (&mx)[G]) {
+                               const float (&qr)[G][Elem<T>::kVec], float* sl, int rows_cap, float (&mx)[G],
+                               const float* rope_cos = nullptr, const float* rope_sin = nullptr) {
     constexpr int VEC = Elem<T>::kVec;
     constexpr int LPR = D / VEC;
     constexpr int RPW = 32 / LPR;
@@ -65,6 +66,8 @@ __device__ inline void k_phase(const T* Kc, int lo, int hi, const UnitState& st,
             const int lam = base + u * RPW + rsub;
             float f[VEC];
             Elem<T>::unpack(raw[u], f);
+            // in-cache positions: the key in cache slot lam is encoded at position lam
+            if (rope_cos) rope_apply<T, D>(f, min(lam, hi - 1), sub, rope_cos, rope_sin);
 #pragma unroll
             for (int h = 0; h < G; ++h) {
                 float a = 0.f;

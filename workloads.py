@@ -36,6 +36,7 @@ class Workload:
     key_scale: bool       # per-sequence key scale drawn in [0.5, 2]
     ragged: bool          # prefill lengths drawn in [prefill_len/2, prefill_len]
     seed: int
+    rotate: bool = True   # False: q, k are left without rotary embedding (for caches that assign positions themselves)
 
     @property
     def group(self) -> int:
@@ -125,6 +126,14 @@ def rope(x: np.ndarray, pos: np.ndarray, base: float) -> np.ndarray:
     return np.concatenate([x1 * cos - x2 * sin, x2 * cos + x1 * sin], axis=-1).astype(np.float32)
 
 
+def rope_tables(slots: int, d: int, base: float):
+    """cos, sin [slots, d/2] in single precision: the rotary cache a model hands to a library that assigns
+    positions by cache slot (angle = slot * base**(-2i/d))."""
+    inv_freq = base ** (-np.arange(d // 2, dtype=np.float64) * 2.0 / d)
+    ang = np.arange(slots, dtype=np.float64)[:, None] * inv_freq[None, :]
+    return np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)
+
+
 def seq_key_scales(w: Workload) -> np.ndarray:
     if not w.key_scale:
         return np.ones(w.batch, np.float32)
@@ -161,8 +170,8 @@ def tokens_at(w: Workload, layer: int, starts, T: int):
         if out_ch:
             kb[..., out_ch] *= 8.0
         kb *= scales[b]
-        q[:, b] = rope(qb, pos, w.rope_base)
-        k[:, b] = rope(kb, pos, w.rope_base)
+        q[:, b] = rope(qb, pos, w.rope_base) if w.rotate else qb
+        k[:, b] = rope(kb, pos, w.rope_base) if w.rotate else kb
         v[:, b] = vb
     return round_to(q, w.dtype), round_to(k, w.dtype), round_to(v, w.dtype)
 
