@@ -70,7 +70,11 @@ typedef enum {
     TREEKV_OPT_DECODE_SPLIT = 0, /* thread blocks per (sequence, KV head) in decode: 0 = automatic, else 1,2,4,8 */
     TREEKV_OPT_PREFILL_PATH = 1, /* 0 = automatic, 1 = CUDA-core kernel, 2 / 3 = tcgen05 tensor-core kernel with 128 / 256
                                     query rows per thread block (bf16, head_dim 128) */
-    TREEKV_OPT_DECODE_PATH = 2   /* 0 = automatic, 1 = CUDA-core kernel, 2 = cp.async + mma.sync kernel (bf16 only) */
+    TREEKV_OPT_DECODE_PATH = 2,  /* 0 = automatic, 1 = CUDA-core kernel, 2 = cp.async + mma.sync kernel (bf16 only) */
+    TREEKV_OPT_PREFILL_APPEND = 3 /* 0 = automatic: the tensor-core prefill kernels read the chunk's own keys and values
+                                    from dev_k / dev_v and append them to the cache themselves whenever every sequence's
+                                    chunk length is a multiple of 128 (no separate append kernel); 1 = always append with
+                                    a kernel of its own before the attention.  Same result either way. */
 } treekv_option;
 
 typedef struct {

@@ -231,10 +231,24 @@ treekv_status decode_step_impl(treekv_ctx* ctx, const void* dev_q, const void* d
 
 // Attention of a chunk over [cache | chunk] with the column sums of its probability matrix (all of the chunk's
 // rows, or the last ps.window tokens): tensor-core kernels for bf16 / head_dim 128, CUDA cores otherwise.
-treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, const void* dev_q, void* dev_out,
-                                     const ChunkLens& lens, int chunk_stride, int max_m, cudaStream_t s) {
+// `direct`: the tensor-core kernels take the chunk's key / value tiles from dev_k / dev_v and append the chunk to the
+// slabs themselves (see chunk_direct_ok); otherwise the chunk's rows must already be in the slabs.
+treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, const void* dev_q, const void* dev_k,
+                                     const void* dev_v, bool direct, void* dev_out, const ChunkLens& lens, int chunk_stride,
+                                     int max_m, cudaStream_t s) {
     cudaError_t e;
     if (use_tc_prefill(ctx)) {
+        ChunkTensors ct;
+        ct.k = nullptr; ct.v = nullptr;
+        if (direct) {
+            const uint64_t kdims[3] = {128ull, (uint64_t)ctx->cv.Hkv, (uint64_t)ctx->cv.B * (uint64_t)chunk_stride};
+            const uint64_t kstrides[2] = {256ull, (uint64_t)ctx->cv.Hkv * 256ull};
+            const uint32_t kbox[3] = {64u, 1u, 128u};
+            if (!make_tensor_map_bf16(&ct.tmK, dev_k, 3, kdims, kstrides, kbox) ||
+                !make_tensor_map_bf16(&ct.tmV, dev_v, 3, kdims, kstrides, kbox))
+                return TREEKV_ERR_CUDA;
+            ct.k = dev_k; ct.v = dev_v;
+        }
         // q is [batch*chunk_stride tokens][n_heads][128]; a tile is 64 channels x G heads x 128/G tokens
         CUtensorMap tmQ;
         const uint64_t dims[3] = {128ull, (uint64_t)ctx->cv.Hq, (uint64_t)ctx->cv.B * (uint64_t)chunk_stride};
@@ -244,12 +258,25 @@ treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, 
         // two query tiles per CTA once the one-tile grid would cover the machine at least twice (or on request)
         const long tiles = (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + kQTileRows - 1) / kQTileRows);
         const bool two = ctx->opt_prefill_path == 3 || (ctx->opt_prefill_path == 0 && tiles >= 2L * ctx->sm_count);
-        e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s)
-                : launch_prefill_tc(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, dev_out, lens, chunk_stride, max_m, s);
+        e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, s)
+                : launch_prefill_tc(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, s);
     } else {
         e = launch_prefill_simt(ctx->cv, ctx->dt, ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
     }
     return e == cudaSuccess ? TREEKV_OK : cuda_fail(ctx, e);
+}
+
+// The tensor-core kernels can read the chunk's keys and values from the caller's tensors - and append them - when
+// every chunk tile of 128 tokens holds tokens of the call only (rows past a sequence's length are the caller's
+// padding and may hold anything, which a value tile must not) and the cached tokens already cover the protected
+// initial tokens (so that the chunk's rows lie behind both cached segments).
+bool chunk_direct_ok(const treekv_ctx* ctx, const ChunkLens& lens) {
+    if (!use_tc_prefill(ctx) || ctx->opt_prefill_append == 1) return false;
+    for (int b = 0; b < ctx->cv.B; ++b) {
+        if (lens.m[b] == 0) continue;
+        if (lens.m[b] % 128 || ctx->n_seen[b] < ctx->cv.ns) return false;
+    }
+    return true;
 }
 
 }  // namespace
@@ -279,14 +306,19 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
     }
     if (max_m == 0) return TREEKV_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, chunk_stride, max_m, s);
-    if (e != cudaSuccess) return cuda_fail(ctx, e);
-    const treekv_status ast = launch_chunk_attention(ctx, ctx->ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
+    const bool direct = chunk_direct_ok(ctx, lens);
+    cudaError_t e = cudaSuccess;
+    if (!direct) {
+        e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, chunk_stride, max_m, s);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    const treekv_status ast =
+        launch_chunk_attention(ctx, ctx->ps, dev_q, dev_k, dev_v, direct, dev_out, lens, chunk_stride, max_m, s);
     if (ast != TREEKV_OK) return ast;
     // score update, all eviction segments and the token counters in one launch
     e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    ctx->launches += 3;  // append, attention, update + eviction
+    ctx->launches += direct ? 2 : 3;  // (append,) attention, update + eviction
     for (int b = 0; b < ctx->cv.B; ++b) {
         const int64_t before = ctx->n_seen[b];
         ctx->n_seen[b] += lens.m[b];
@@ -320,7 +352,7 @@ treekv_status treekv_prefill_oneshot(treekv_ctx* ctx, const void* dev_q, const v
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     PrefillScratch ps = ctx->ps;
     ps.window = block;  // only the last block's queries score the prompt
-    const treekv_status ast = launch_chunk_attention(ctx, ps, dev_q, dev_out, lens, stride, max_m, s);
+    const treekv_status ast = launch_chunk_attention(ctx, ps, dev_q, dev_k, dev_v, false, dev_out, lens, stride, max_m, s);
     if (ast != TREEKV_OK) return ast;
     e = launch_oneshot_update_evict(ctx->cv, ctx->dt, ps, lens, block, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
@@ -510,6 +542,10 @@ treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value) {
             if (value < 0 || value > 3) return TREEKV_ERR_INVALID_ARG;
             if (value >= 2 && !ctx->has_tma) return TREEKV_ERR_UNSUPPORTED;
             ctx->opt_prefill_path = value;
+            return TREEKV_OK;
+        case TREEKV_OPT_PREFILL_APPEND:
+            if (value < 0 || value > 1) return TREEKV_ERR_INVALID_ARG;
+            ctx->opt_prefill_append = value;
             return TREEKV_OK;
     }
     return TREEKV_ERR_INVALID_ARG;

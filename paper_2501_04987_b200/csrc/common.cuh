@@ -276,14 +276,22 @@ size_t prefill_simt_smem_bytes(int G, int D, int n_max);
 cudaError_t launch_prefill_simt(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const void* q, void* out,
                                 const ChunkLens& lens, int chunk_stride, int max_m, cudaStream_t stream);
 
+// The chunk's k and v tensors with tensor maps over them, when the tensor-core prefill kernels read their chunk tiles
+// from there and append the chunk themselves (k == nullptr: an append kernel put the rows into the slab first).
+struct ChunkTensors {
+    const void* k;
+    const void* v;
+    CUtensorMap tmK, tmV;  // channels x KV heads x tokens of the call, box 64 x 1 x 128
+};
+
 size_t prefill_tc2_smem_bytes();
 cudaError_t launch_prefill_tc2(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                               const CUtensorMap& tmV, void* out, const ChunkLens& lens, int chunk_stride, int max_m,
-                               cudaStream_t stream);  // 256 query rows per CTA, for large grids
+                               const CUtensorMap& tmV, const ChunkTensors& ct, void* out, const ChunkLens& lens,
+                               int chunk_stride, int max_m, cudaStream_t stream);  // 256 query rows per CTA, for large grids
 
 size_t prefill_tc_smem_bytes();
 cudaError_t launch_prefill_tc(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                              const CUtensorMap& tmV, void* out, const ChunkLens& lens, int chunk_stride, int max_m,
-                              cudaStream_t stream);
+                              const CUtensorMap& tmV, const ChunkTensors& ct, void* out, const ChunkLens& lens,
+                              int chunk_stride, int max_m, cudaStream_t stream);
 
 }  // namespace treekv

@@ -18,6 +18,7 @@ struct treekv_ctx {
     int opt_decode_split;
     int opt_prefill_path;
     int opt_decode_path;
+    int opt_prefill_append;
     int sm_count;
     int device;  // ordinal of the device that was current at creation: the workspace lives there
     // host-side record

@@ -33,7 +33,8 @@ enum Bar { Q_FULL = 0, RING_FULL = 1, RING_EMPTY = 4, S_FULL = 7, S_FREE = 11, P
 template <int G>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                   const __grid_constant__ CUtensorMap tmV, CacheView cv, PrefillScratch ps,
+                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKin,
+                   const __grid_constant__ CUtensorMap tmVin, ChunkDirect cd, CacheView cv, PrefillScratch ps,
                    __nv_bfloat16* __restrict__ out, ChunkLens lens, int chunk_stride) {
     constexpr int TOK = 128 / G;  // tokens per sub-tile
     const int unit = blockIdx.y, qt2 = blockIdx.x;
@@ -44,7 +45,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int t1c = min(t0c + 2 * TOK, m);
     const int N = cv.n_seen[unit];
     const UnitState st = unit_state(N, cv);
-    const KeyTiles kt = key_tiles(st, st.L + t1c);
+    const KeyTiles kt = key_tiles(st, st.L + t1c, cd.k != nullptr);
     const int NT = kt.NT;
     const int n = st.L + m;
 
@@ -87,24 +88,29 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tma_load_3d(sQ + s * kSlot + kHalf, &tmQ, 64, kh * G, b * chunk_stride + t0c + s * TOK, bar(Q_FULL));
             }
             int ld = 0;
-            auto load_tile = [&](const CUtensorMap* mp, int j) {
+            auto load_tile = [&](const CUtensorMap* mp, const CUtensorMap* mp_in, int j) {
                 int lam0, row0, valid;
-                tile_of(kt, j, lam0, row0, valid);
-                const int grow = unit * cv.R + row0;
+                const bool from_chunk = tile_of(kt, j, lam0, row0, valid);
                 const int slot = ld % kRing;
                 if (!mbar_wait(bar(RING_EMPTY + slot), ((ld / kRing) & 1) ^ 1)) { ok = false; return; }
                 const uint32_t dst = sRing + slot * kSlot;
                 mbar_arrive_expect_tx(bar(RING_FULL + slot), kSlot);
-                tma_load_2d(dst, mp, 0, grow, bar(RING_FULL + slot));
-                tma_load_2d(dst + kHalf, mp, 64, grow, bar(RING_FULL + slot));
+                if (from_chunk) {  // 128 tokens of the caller's tensor
+                    tma_load_3d(dst, mp_in, 0, kh, b * chunk_stride + row0, bar(RING_FULL + slot));
+                    tma_load_3d(dst + kHalf, mp_in, 64, kh, b * chunk_stride + row0, bar(RING_FULL + slot));
+                } else {
+                    const int grow = unit * cv.R + row0;
+                    tma_load_2d(dst, mp, 0, grow, bar(RING_FULL + slot));
+                    tma_load_2d(dst + kHalf, mp, 64, grow, bar(RING_FULL + slot));
+                }
                 ++ld;
             };
             // pass A: K tiles in order.  Pass B, in the order the MMA warp consumes them: K_0 | K_1 V_0 | K_2 V_1 | ...
-            for (int j = 0; j < NT && ok; ++j) load_tile(&tmK, j);
-            if (ok) load_tile(&tmK, 0);
+            for (int j = 0; j < NT && ok; ++j) load_tile(&tmK, &tmKin, j);
+            if (ok) load_tile(&tmK, &tmKin, 0);
             for (int j = 0; j < NT && ok; ++j) {
-                if (j + 1 < NT) load_tile(&tmK, j + 1);
-                if (ok) load_tile(&tmV, j);
+                if (j + 1 < NT) load_tile(&tmK, &tmKin, j + 1);
+                if (ok) load_tile(&tmV, &tmVin, j);
             }
             if (!ok) atomicOr(&cv.stats->error, 4u);
         }
@@ -213,6 +219,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         float* part_m = reinterpret_cast<float*>(p_area);
         float* part_l = part_m + 512;
         uint32_t va[32], vb[32];  // two chunks of 32 columns: the next one is in flight while this one is used
+        if (cd.k) append_own_tokens(cv, cd, unit, b, kh, chunk_stride, st, N, t0, t1, tid - 64 - sub * 256, 256);
         // ---- pass A: row statistics of the sub-tile over all key tiles
         {
             const int tq = max(t0c, min(t0 + row / G, t1 - 1));  // rows past the chunk repeat a real row: finite, unused
@@ -404,8 +411,8 @@ size_t prefill_tc2_smem_bytes() { return (size_t)(4 + kRing) * kSlot + 512 * siz
 
 template <int G>
 static cudaError_t launch_prefill_tc2_t(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ,
-                                        const CUtensorMap& tmK, const CUtensorMap& tmV, void* out, const ChunkLens& lens,
-                                        int chunk_stride, int max_m, cudaStream_t stream) {
+                                        const CUtensorMap& tmK, const CUtensorMap& tmV, const ChunkTensors& ct, void* out,
+                                        const ChunkLens& lens, int chunk_stride, int max_m, cudaStream_t stream) {
     auto kern = prefill_tc2_kernel<G>;
     const size_t smem = prefill_tc2_smem_bytes();
     static bool smem_set[64] = {};  // per device: the opt-in is needed once
@@ -418,19 +425,21 @@ static cudaError_t launch_prefill_tc2_t(const CacheView& cv, const PrefillScratc
         smem_set[dev] = true;
     }
     dim3 grid((max_m * G + 2 * kQTileRows - 1) / (2 * kQTileRows), cv.B * cv.Hkv);
-    kern<<<grid, kThreads, smem, stream>>>(tmQ, tmK, tmV, cv, ps, reinterpret_cast<__nv_bfloat16*>(out), lens, chunk_stride);
+    const ChunkDirect cd = {reinterpret_cast<const __nv_bfloat16*>(ct.k), reinterpret_cast<const __nv_bfloat16*>(ct.v)};
+    kern<<<grid, kThreads, smem, stream>>>(tmQ, tmK, tmV, ct.k ? ct.tmK : tmK, ct.k ? ct.tmV : tmV, cd, cv, ps,
+                                           reinterpret_cast<__nv_bfloat16*>(out), lens, chunk_stride);
     return cudaGetLastError();
 }
 
 cudaError_t launch_prefill_tc2(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                               const CUtensorMap& tmV, void* out, const ChunkLens& lens, int chunk_stride, int max_m,
-                               cudaStream_t stream) {
+                               const CUtensorMap& tmV, const ChunkTensors& ct, void* out, const ChunkLens& lens,
+                               int chunk_stride, int max_m, cudaStream_t stream) {
     if (cv.d != kD) return cudaErrorInvalidValue;
     switch (cv.Hq / cv.Hkv) {
-        case 1: return launch_prefill_tc2_t<1>(cv, ps, tmQ, tmK, tmV, out, lens, chunk_stride, max_m, stream);
-        case 2: return launch_prefill_tc2_t<2>(cv, ps, tmQ, tmK, tmV, out, lens, chunk_stride, max_m, stream);
-        case 4: return launch_prefill_tc2_t<4>(cv, ps, tmQ, tmK, tmV, out, lens, chunk_stride, max_m, stream);
-        case 8: return launch_prefill_tc2_t<8>(cv, ps, tmQ, tmK, tmV, out, lens, chunk_stride, max_m, stream);
+        case 1: return launch_prefill_tc2_t<1>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
+        case 2: return launch_prefill_tc2_t<2>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
+        case 4: return launch_prefill_tc2_t<4>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
+        case 8: return launch_prefill_tc2_t<8>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
     }
     return cudaErrorInvalidValue;
 }

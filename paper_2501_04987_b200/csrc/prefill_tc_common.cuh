@@ -14,25 +14,70 @@ constexpr uint32_t kTmemCols = 512;
 constexpr int kD = 128;
 constexpr int kThreads = 576;  // TMA warp, MMA warp, 2 groups x 8 softmax warps
 
+// Where a thread block's keys come from.  Cached tokens are two row segments of the unit's slab (live indices [0, a)
+// at row = index, [a, L) at row = index + i).  The chunk's own tokens are either rows of the slab behind them (an
+// append kernel ran first), or - "direct" - read from the caller's k / v tensors in tiles of 128 tokens, in which
+// case the attention kernel also appends its own tokens to the slab and no append kernel runs.
 struct KeyTiles {
-    int i;     // cycle position: live indices [0, a) sit at row = index, the others at row = index + i
+    int i;     // cycle position
     int a;     // split point (protected initial tokens + i)
     int L;     // cached rows before the chunk
     int nvis;  // live indices [0, nvis) are visible to at least one query of this thread block
     int nA;    // tiles over the first segment [0, a)
+    int nB;    // tiles over the second segment: [a, L) when direct, [a, nvis) otherwise
     int NT;    // all tiles
+    bool direct;
 };
-__device__ inline KeyTiles key_tiles(const UnitState& st, int nvis) {
+__device__ inline KeyTiles key_tiles(const UnitState& st, int nvis, bool direct) {
     KeyTiles kt;
-    kt.i = st.i; kt.a = st.a; kt.L = st.L; kt.nvis = nvis;
+    kt.i = st.i; kt.a = st.a; kt.L = st.L; kt.nvis = nvis; kt.direct = direct;
     kt.nA = (st.a + 127) / 128;
-    kt.NT = kt.nA + (nvis - st.a + 127) / 128;
+    kt.nB = ((direct ? st.L : nvis) - st.a + 127) / 128;
+    kt.NT = kt.nA + kt.nB + (direct ? (nvis - st.L + 127) / 128 : 0);
     return kt;
 }
-// key tile j: first live index, first physical row, rows that exist
-__device__ inline void tile_of(const KeyTiles& kt, int j, int& lam0, int& row0, int& valid) {
-    if (j < kt.nA) { lam0 = j * 128; row0 = lam0; valid = min(128, kt.a - lam0); }
-    else { lam0 = kt.a + (j - kt.nA) * 128; row0 = lam0 + kt.i; valid = min(128, kt.nvis - lam0); }
+// key tile j: first live index, first row (of the slab, or token of the chunk when the result is true), rows that exist
+__device__ inline bool tile_of(const KeyTiles& kt, int j, int& lam0, int& row0, int& valid) {
+    if (j < kt.nA) { lam0 = j * 128; row0 = lam0; valid = min(128, kt.a - lam0); return false; }
+    if (j < kt.nA + kt.nB) {
+        lam0 = kt.a + (j - kt.nA) * 128; row0 = lam0 + kt.i; valid = min(128, (kt.direct ? kt.L : kt.nvis) - lam0);
+        return false;
+    }
+    row0 = (j - kt.nA - kt.nB) * 128; lam0 = kt.L + row0; valid = min(128, kt.nvis - lam0);
+    return true;
+}
+
+// The chunk's k and v as the caller passed them ([batch][chunk_stride][n_kv_heads][128] bf16) when the kernel reads
+// its chunk tiles from there (tensor maps over the same memory: channels x heads x tokens, box 64 x 1 x 128);
+// k == nullptr: the chunk's rows are already in the slab.
+struct ChunkDirect {
+    const __nv_bfloat16* k;
+    const __nv_bfloat16* v;
+};
+
+// Direct mode: the thread block appends the tokens [t0, t1) of its own query rows to the unit's slab (Algorithm 1's
+// append: k, v, stream position, S = 0) - rows no thread block reads during this kernel.  `nthr` threads with
+// index `t` in [0, nthr) take part.
+__device__ inline void append_own_tokens(const CacheView& cv, const ChunkDirect& cd, int unit, int b, int kh, int chunk_stride,
+                                         const UnitState& st, int N, int t0, int t1, int t, int nthr) {
+    const int ntok = t1 - t0;
+    if (ntok <= 0) return;
+    const size_t rbase = (size_t)unit * cv.R + st.L + st.i + t0;
+    const size_t src0 = (((size_t)b * chunk_stride + t0) * cv.Hkv + kh) * (kD / 8);  // in 16-byte pieces
+    const size_t sstride = (size_t)cv.Hkv * (kD / 8);
+    const uint4* ks = reinterpret_cast<const uint4*>(cd.k);
+    const uint4* vs = reinterpret_cast<const uint4*>(cd.v);
+    uint4* kd = reinterpret_cast<uint4*>(cv.K) + rbase * (kD / 8);
+    uint4* vd = reinterpret_cast<uint4*>(cv.V) + rbase * (kD / 8);
+    for (int idx = t; idx < ntok * (kD / 8); idx += nthr) {
+        const int r = idx / (kD / 8), e = idx % (kD / 8);
+        kd[idx] = ks[src0 + r * sstride + e];
+        vd[idx] = vs[src0 + r * sstride + e];
+    }
+    for (int r = t; r < ntok; r += nthr) {
+        cv.pos[rbase + r] = N + t0 + r;
+        cv.S[rbase + r] = 0.f;
+    }
 }
 
 // 2^x on the special-function unit, one instruction (inputs here are <= ~0; results below 2^-126 flush to zero)

@@ -123,6 +123,37 @@ def test_two_tile_tensor_core_prefill_kernel(gpu, g, lens, chunk, budget):
     print("two-tile prefill g=%d" % g, rep)
 
 
+@pytest.mark.parametrize("path", [2, 3])
+@pytest.mark.parametrize("append", [0, 1])
+@pytest.mark.parametrize("g,budget,chunk,lens", [
+    (1, 300, 256, [5 * 256, 3 * 256]),        # budget not a multiple of the tile: both cached segments end in partial tiles
+    (4, 512, 128, [9 * 128, 9 * 128 + 64]),   # GQA; the second sequence ends in a ragged chunk (append kernel for that call)
+    (2, 200, 384, [4 * 384, 384]),            # chunks longer than the budget: several wraps per call
+])
+def test_fused_append_and_chunk_tiles_from_the_input_tensors(gpu, path, append, g, budget, chunk, lens):
+    """When every chunk length of a call is a multiple of 128 the tensor-core kernels read the chunk's own key / value
+    tiles from the caller's tensors and append the chunk themselves (two launches per call instead of three); forced
+    to the separate append kernel the same calls must give the same result.  Both are followed by the oracle."""
+    import torch
+
+    w = W.parity_slice(W.CONFIGS["cfg5"], layers=1, batch=2, n_heads=g * 2, n_kv_heads=2, budget=budget, chunk=chunk)
+    kv, orc = _pair(gpu, w)
+    kv.set_option(gpu.OPT_PREFILL_PATH, path)
+    kv.set_option(gpu.OPT_PREFILL_APPEND, append)
+    rep = Report()
+    _run_prefill(kv, orc, w, rep, lens, chunk)
+    assert [kv.tokens_seen(b) for b in range(2)] == lens
+    _run_decode(kv, orc, w, 0, 6, rep, starts=lens)
+    # one more full chunk for both sequences, without read-outs in between: the launch count shows which way it went
+    q, k, v = W.tokens_at(w, 0, [x + 6 for x in lens], chunk)
+    l0 = kv.stats()["kernel_launches"]
+    step_prefill(kv, orc, q.transpose(1, 0, 2, 3), k.transpose(1, 0, 2, 3), v.transpose(1, 0, 2, 3), w.dtype, rep)
+    torch.cuda.synchronize()
+    read_outs = 3  # retained positions (twice) and scores of the comparison
+    assert kv.stats()["kernel_launches"] - l0 - read_outs == (2 if append == 0 else 3)
+    assert kv.stats()["device_error"] == 0
+
+
 # ---------------------------------------------------------------------------------------------------------
 # edge cases
 # ---------------------------------------------------------------------------------------------------------
