@@ -383,6 +383,8 @@ def main():
     ap.add_argument("--prefill-legs", default="cfg5,cfg4,cfg3", help="prefill shapes to time, the first is `prefill` ('' = none)")
     ap.add_argument("--prefill-chunks", type=int, default=2, help="chunks per timed prefill block")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-eviction-stream", action="store_true",
+                    help="prefill legs: keep every kernel of a chunk on the caller's stream (TREEKV_OPT_EVICTION_STREAM off)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS)
     ap.add_argument("--decode-split", type=int, default=0, help="thread blocks per (sequence, KV head); 0 = automatic")
@@ -432,7 +434,8 @@ def main():
     # ------------------------------------------------------------------ prefill legs
     prefill_legs = []
     for name in [x for x in args.prefill_legs.split(",") if x]:
-        prefill_legs.append(run_prefill_leg(torch, binding, cfg(name), max(1, args.prefill_chunks), dev, rep, timer, peaks))
+        prefill_legs.append(run_prefill_leg(torch, binding, cfg(name), max(1, args.prefill_chunks), dev, rep, timer, peaks,
+                                            not args.no_eviction_stream))
     prefill = prefill_legs[0] if prefill_legs else None
     if sampler is not None:
         sampler.stop()
@@ -559,11 +562,14 @@ def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev
             "config": config_of(w)}
 
 
-def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks):
+def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks, eviction_stream=True):
     tdtype = torch.bfloat16 if pw.dtype == "bf16" else torch.float32
     world, rank = rep.world, rep.rank
     m, c = pw.chunk, pw.budget
     ctxs = [binding.TreeKV(c, pw.n_heads, pw.n_kv_heads, pw.head_dim, pw.dtype, pw.batch, m) for _ in range(pw.layers)]
+    if eviction_stream:
+        for x in ctxs:
+            x.set_option(binding.OPT_EVICTION_STREAM, 1)
     wr = W.parity_slice(pw, seed=pw.seed + 1000 * rank)
     ins = []
     for layer in range(pw.layers):   # the same chunk values every call: timing does not depend on them
@@ -604,7 +610,7 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks):
     return {"metric": "treekv_prefill_tokens_per_s", "value": tok_s, "unit": "tokens/s", "chunks_per_block": n_chunks,
             "blocks": t["blocks"], "region_ms": t["region_ms"], "ms_per_chunk_all_layers": ms / n_chunks,
             "gpu_launches": int(launches), "clocks": t["clocks"],
-            "config": config_of(pw, chunk=m,
+            "config": config_of(pw, chunk=m, eviction_stream=bool(eviction_stream),
                                 l2="no flush: a chunk reads %.0f MB of K/V per layer and a layer is revisited %d layers later (126 MB L2)"
                                    % (2 * pw.batch * pw.n_kv_heads * (c + m) * pw.head_dim * 2 / 1e6, pw.layers)),
             "roofline": {"bound": "tensor", "achieved": ach3, "peak": sus, "unit": "TFLOP/s", "frac": ach3 / sus,

@@ -71,10 +71,19 @@ typedef enum {
     TREEKV_OPT_PREFILL_PATH = 1, /* 0 = automatic, 1 = CUDA-core kernel, 2 / 3 = tcgen05 tensor-core kernel with 128 / 256
                                     query rows per thread block (bf16, head_dim 128) */
     TREEKV_OPT_DECODE_PATH = 2,  /* 0 = automatic, 1 = CUDA-core kernel, 2 = cp.async + mma.sync kernel (bf16 only) */
-    TREEKV_OPT_PREFILL_APPEND = 3 /* 0 = automatic: the tensor-core prefill kernels read the chunk's own keys and values
+    TREEKV_OPT_PREFILL_APPEND = 3, /* 0 = automatic: the tensor-core prefill kernels read the chunk's own keys and values
                                     from dev_k / dev_v and append them to the cache themselves whenever every sequence's
                                     chunk length is a multiple of 128 (no separate append kernel); 1 = always append with
                                     a kernel of its own before the attention.  Same result either way. */
+    TREEKV_OPT_EVICTION_STREAM = 4 /* 0 (default) = every kernel of a call runs on the caller's stream.  1 = the last
+                                    kernel of treekv_prefill_chunk (score update + eviction + compaction, which only
+                                    touches the workspace) runs on a stream the context owns, behind the chunk's
+                                    attention; whatever the caller enqueues next on its own stream - the rest of the
+                                    layer, the next layer's chunk - overlaps it, and every later call on this context
+                                    first orders its stream behind that kernel.  dev_out, dev_q, dev_k, dev_v are only
+                                    touched on the caller's stream.  Setting it creates (0: synchronises and destroys)
+                                    the stream and two events; treekv_destroy then waits for the stream; calls made
+                                    while the caller's stream is being captured into a graph are not supported. */
 } treekv_option;
 
 typedef struct {
@@ -285,7 +294,8 @@ treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value);
 /* Back to the empty cache (idx = 1, nothing seen).  Enqueued on `stream`. */
 treekv_status treekv_reset(treekv_ctx* ctx, void* stream);
 
-/* Frees the host-side context.  The workspace stays the caller's. */
+/* Frees the host-side context (with TREEKV_OPT_EVICTION_STREAM on, after waiting for the context's own stream).  The
+ * workspace stays the caller's. */
 void treekv_destroy(treekv_ctx* ctx);
 
 const char* treekv_status_string(treekv_status s);

@@ -184,7 +184,8 @@ treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_
 
 treekv_status treekv_reset(treekv_ctx* ctx, void* stream) {
     if (!ctx) return TREEKV_ERR_INVALID_ARG;
-    const cudaError_t e = launch_init_state(ctx->cv, static_cast<cudaStream_t>(stream));
+    cudaError_t e = join_eviction_stream(ctx, static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = launch_init_state(ctx->cv, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     memset(ctx->n_seen, 0, sizeof(ctx->n_seen));
     ctx->evictions = 0;
@@ -192,7 +193,16 @@ treekv_status treekv_reset(treekv_ctx* ctx, void* stream) {
     return TREEKV_OK;
 }
 
-void treekv_destroy(treekv_ctx* ctx) { delete ctx; }
+void treekv_destroy(treekv_ctx* ctx) {
+    if (!ctx) return;
+    if (ctx->side) {  // the workspace is the caller's to free after this call: nothing of ours may still run on it
+        cudaStreamSynchronize(ctx->side);
+        cudaEventDestroy(ctx->ev_attn);
+        cudaEventDestroy(ctx->ev_state);
+        cudaStreamDestroy(ctx->side);
+    }
+    delete ctx;
+}
 
 }  // extern "C"
 
@@ -212,6 +222,10 @@ treekv_status decode_step_impl(treekv_ctx* ctx, const void* dev_q, const void* d
         }
     }
     if (n_active == 0) return TREEKV_OK;
+    if (ctx->side_pending) {
+        const cudaError_t je = join_eviction_stream(ctx, static_cast<cudaStream_t>(stream));
+        if (je != cudaSuccess) return cuda_fail(ctx, je);
+    }
     const cudaError_t e =
         use_mma_decode(ctx)
             ? launch_decode_mma(ctx->cv, dev_q, dev_k, dev_v, dev_out, mask, pick_decode_split(ctx), inputs_final,
@@ -307,7 +321,9 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
     if (max_m == 0) return TREEKV_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool direct = chunk_direct_ok(ctx, lens);
-    cudaError_t e = cudaSuccess;
+    // the previous chunk's eviction must be over before this chunk's attention reads the cache and writes column sums
+    cudaError_t e = join_eviction_stream(ctx, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
     if (!direct) {
         e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, chunk_stride, max_m, s);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
@@ -315,8 +331,17 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
     const treekv_status ast =
         launch_chunk_attention(ctx, ctx->ps, dev_q, dev_k, dev_v, direct, dev_out, lens, chunk_stride, max_m, s);
     if (ast != TREEKV_OK) return ast;
-    // score update, all eviction segments and the token counters in one launch
-    e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, s);
+    // score update, all eviction segments and the token counters in one launch - on the eviction stream when there is
+    // one: nothing the caller does next with the chunk's output depends on it
+    if (ctx->side) {
+        e = cudaEventRecord(ctx->ev_attn, s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->side, ctx->ev_attn, 0);
+        if (e == cudaSuccess) e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, ctx->side);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_state, ctx->side);
+        ctx->side_pending = true;  // also after a failure half-way: a later call then still orders itself behind `side`
+    } else {
+        e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, s);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += direct ? 2 : 3;  // (append,) attention, update + eviction
     for (int b = 0; b < ctx->cv.B; ++b) {
@@ -348,7 +373,8 @@ treekv_status treekv_prefill_oneshot(treekv_ctx* ctx, const void* dev_q, const v
     }
     if (max_m == 0) return TREEKV_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, stride, max_m, s);
+    cudaError_t e = join_eviction_stream(ctx, s);
+    if (e == cudaSuccess) e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, stride, max_m, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     PrefillScratch ps = ctx->ps;
     ps.window = block;  // only the last block's queries score the prompt
@@ -413,7 +439,8 @@ treekv_status treekv_prefill_chunk_host(treekv_ctx* ctx, const void* host_q, con
 
 treekv_status treekv_retained_positions(treekv_ctx* ctx, int32_t* dev_pos, int32_t* dev_count, void* stream) {
     if (!ctx || !dev_pos || !dev_count) return TREEKV_ERR_INVALID_ARG;
-    const cudaError_t e = launch_retained_positions(ctx->cv, dev_pos, dev_count, static_cast<cudaStream_t>(stream));
+    cudaError_t e = join_eviction_stream(ctx, static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = launch_retained_positions(ctx->cv, dev_pos, dev_count, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return TREEKV_OK;
@@ -421,7 +448,8 @@ treekv_status treekv_retained_positions(treekv_ctx* ctx, int32_t* dev_pos, int32
 
 treekv_status treekv_scores(treekv_ctx* ctx, float* dev_sbar, void* stream) {
     if (!ctx || !dev_sbar) return TREEKV_ERR_INVALID_ARG;
-    const cudaError_t e = launch_scores(ctx->cv, dev_sbar, static_cast<cudaStream_t>(stream));
+    cudaError_t e = join_eviction_stream(ctx, static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = launch_scores(ctx->cv, dev_sbar, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return TREEKV_OK;
@@ -450,7 +478,8 @@ treekv_status treekv_export_state(treekv_ctx* ctx, void* dev_image, int64_t* hos
     if (!ctx || !dev_image || !host_tokens_seen || !aligned16(dev_image)) return TREEKV_ERR_INVALID_ARG;
     StateImage img;
     state_image_layout(ctx, dev_image, &img);
-    const cudaError_t e = launch_export_state(ctx->cv, ctx->dt, img, static_cast<cudaStream_t>(stream));
+    cudaError_t e = join_eviction_stream(ctx, static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = launch_export_state(ctx->cv, ctx->dt, img, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     for (int b = 0; b < ctx->cv.B; ++b) host_tokens_seen[b] = ctx->n_seen[b];
@@ -463,7 +492,8 @@ treekv_status treekv_import_state(treekv_ctx* ctx, const void* dev_image, const 
         if (host_tokens_seen[b] < 0 || host_tokens_seen[b] >= 0x7fffffff - 1) return TREEKV_ERR_INVALID_ARG;
     StateImage img;
     state_image_layout(ctx, const_cast<void*>(dev_image), &img);
-    const cudaError_t e = launch_import_state(ctx->cv, ctx->dt, img, static_cast<cudaStream_t>(stream));
+    cudaError_t e = join_eviction_stream(ctx, static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = launch_import_state(ctx->cv, ctx->dt, img, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     ctx->evictions = 0;
@@ -478,7 +508,8 @@ treekv_status treekv_get_stats(treekv_ctx* ctx, treekv_stats* host_out, void* st
     if (!ctx || !host_out) return TREEKV_ERR_INVALID_ARG;
     DevStats ds;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemcpyAsync(&ds, ctx->cv.stats, sizeof(ds), cudaMemcpyDeviceToHost, s);
+    cudaError_t e = join_eviction_stream(ctx, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&ds, ctx->cv.stats, sizeof(ds), cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     host_out->evictions = ctx->evictions;
@@ -543,6 +574,37 @@ treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value) {
             if (value >= 2 && !ctx->has_tma) return TREEKV_ERR_UNSUPPORTED;
             ctx->opt_prefill_path = value;
             return TREEKV_OK;
+        case TREEKV_OPT_EVICTION_STREAM: {
+            if (value < 0 || value > 1) return TREEKV_ERR_INVALID_ARG;
+            if (value == 1 && !ctx->side) {
+                // Lowest priority: an attention thread block fills an SM's shared memory, so an eviction block never shares
+                // an SM with one; the eviction kernel should take the SMs the attention kernel behind it leaves free (a
+                // grid smaller than the machine, or the tail of its last wave), not delay that kernel's blocks.
+                int lo = 0, hi = 0;
+                cudaError_t e = cudaDeviceGetStreamPriorityRange(&lo, &hi);
+                cudaStream_t st = nullptr;
+                cudaEvent_t ea = nullptr, es = nullptr;
+                if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&st, cudaStreamNonBlocking, lo);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ea, cudaEventDisableTiming);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&es, cudaEventDisableTiming);
+                if (e != cudaSuccess) {
+                    if (es) cudaEventDestroy(es);
+                    if (ea) cudaEventDestroy(ea);
+                    if (st) cudaStreamDestroy(st);
+                    return cuda_fail(ctx, e);
+                }
+                ctx->side = st; ctx->ev_attn = ea; ctx->ev_state = es;
+            } else if (value == 0 && ctx->side) {
+                // kernels already on the eviction stream stay ordered through side_pending; later chunks use the caller's
+                const cudaError_t e = cudaStreamSynchronize(ctx->side);
+                cudaEventDestroy(ctx->ev_attn);
+                cudaEventDestroy(ctx->ev_state);
+                cudaStreamDestroy(ctx->side);
+                ctx->side = nullptr; ctx->ev_attn = nullptr; ctx->ev_state = nullptr; ctx->side_pending = false;
+                if (e != cudaSuccess) return cuda_fail(ctx, e);
+            }
+            return TREEKV_OK;
+        }
         case TREEKV_OPT_PREFILL_APPEND:
             if (value < 0 || value > 1) return TREEKV_ERR_INVALID_ARG;
             ctx->opt_prefill_append = value;

@@ -19,6 +19,11 @@ struct treekv_ctx {
     int opt_prefill_path;
     int opt_decode_path;
     int opt_prefill_append;
+    // eviction stream (TREEKV_OPT_EVICTION_STREAM): the score update + eviction kernel of a chunk runs on `side`, after
+    // the chunk's attention (ev_attn), and everything enqueued later for this context waits for it (ev_state)
+    cudaStream_t side;
+    cudaEvent_t ev_attn, ev_state;
+    bool side_pending;  // a kernel on `side` may still be running that the caller's stream has not been told to wait for
     int sm_count;
     int device;  // ordinal of the device that was current at creation: the workspace lives there
     // host-side record
@@ -27,3 +32,14 @@ struct treekv_ctx {
     uint64_t launches;
     int last_cuda_error;
 };
+
+namespace treekv {
+// Orders `stream` behind the context's eviction stream, if a kernel there has not been waited for yet.  Every entry
+// point that enqueues work on the cache calls this first.
+inline cudaError_t join_eviction_stream(treekv_ctx* ctx, cudaStream_t stream) {
+    if (!ctx->side_pending) return cudaSuccess;
+    const cudaError_t e = cudaStreamWaitEvent(stream, ctx->ev_state, 0);
+    if (e == cudaSuccess) ctx->side_pending = false;
+    return e;
+}
+}  // namespace treekv

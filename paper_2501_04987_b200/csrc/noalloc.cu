@@ -111,6 +111,8 @@ extern "C" treekv_status treekv_prefill_chunk_static_scratch(treekv_ctx* ctx, co
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     auto fail = [&](cudaError_t err) { ctx->last_cuda_error = (int)err; return TREEKV_ERR_CUDA; };
+    e = join_eviction_stream(ctx, s);
+    if (e != cudaSuccess) return fail(e);
     e = launch_chunk_append(ctx->cv, ctx->dt, dev_k, dev_v, lens, chunk_stride, max_m, s);
     if (e != cudaSuccess) return fail(e);
     e = launch_prefill_simt(ctx->cv, ctx->dt, ps, dev_q, dev_out, lens, chunk_stride, max_m, s);

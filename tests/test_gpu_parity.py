@@ -347,6 +347,56 @@ def test_chained_launches_match_synchronised_launches(gpu, shape):
         assert torch.equal(x, y)
 
 
+def test_eviction_stream_gives_the_same_bits_and_follows_the_oracle(gpu):
+    """With the eviction stream on, a chunk's score update + eviction runs on a stream of the context's own while the
+    caller's stream goes on (here: with the next layer's chunk).  A stack of four contexts driven chunk after chunk and
+    then step after step without any synchronisation must end in exactly the state, and give exactly the outputs, of
+    the same stack with everything on one stream; and one context with the option on is followed by the oracle."""
+    import torch
+
+    w = W.parity_slice(W.CONFIGS["cfg3"], layers=4, batch=1, n_heads=4, n_kv_heads=4, budget=512, chunk=256)
+    n_chunks, steps = 6, 40
+    ins = []
+    for layer in range(w.layers):
+        qs, ks, vs = W.tokens(w, layer, 0, n_chunks * w.chunk + steps)
+        ins.append([torch.from_numpy(x).cuda().bfloat16() for x in (qs, ks, vs)])   # [T, B, H, d]
+    t0 = n_chunks * w.chunk
+    results = []
+    for side in (0, 1):
+        ctxs = [gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, w.chunk) for _ in range(w.layers)]
+        for kv in ctxs:
+            kv.set_option(gpu.OPT_EVICTION_STREAM, side)
+        outs_p = torch.empty((n_chunks, w.layers, w.batch, w.chunk, w.n_heads, w.head_dim), dtype=torch.bfloat16, device="cuda")
+        outs_d = torch.empty((steps, w.layers, w.batch, w.n_heads, w.head_dim), dtype=torch.bfloat16, device="cuda")
+        chunks = [[[x[c * w.chunk:(c + 1) * w.chunk].transpose(0, 1).contiguous() for x in ins[layer]]
+                   for layer in range(w.layers)] for c in range(n_chunks)]
+        torch.cuda.synchronize()
+        for c in range(n_chunks):
+            for layer, kv in enumerate(ctxs):
+                kv.prefill_chunk(*chunks[c][layer], out=outs_p[c, layer])
+        for s in range(steps):
+            for layer, kv in enumerate(ctxs):
+                kv.decode_step(ins[layer][0][t0 + s], ins[layer][1][t0 + s], ins[layer][2][t0 + s], out=outs_d[s, layer])
+        state = [(kv.scores().clone(), kv.retained_positions()[0].clone()) for kv in ctxs]
+        torch.cuda.synchronize()
+        assert all(kv.stats()["device_error"] == 0 for kv in ctxs)
+        results.append((outs_p.clone(), outs_d.clone(), state))
+        if side:
+            ctxs[0].set_option(gpu.OPT_EVICTION_STREAM, 0)   # switching it off again synchronises and frees the stream
+        del ctxs
+    assert torch.equal(results[0][0], results[1][0]) and torch.equal(results[0][1], results[1][1])
+    for (sa, pa), (sb, pb) in zip(results[0][2], results[1][2]):
+        assert torch.equal(sa, sb) and torch.equal(pa, pb)
+
+    w1 = W.parity_slice(W.CONFIGS["cfg5"], layers=1, batch=2, n_heads=8, n_kv_heads=2, budget=256, chunk=128)
+    kv, orc = _pair(gpu, w1)
+    kv.set_option(gpu.OPT_EVICTION_STREAM, 1)
+    rep = Report()
+    _run_prefill(kv, orc, w1, rep, [7 * 128 + 50, 5 * 128], 128)
+    _run_decode(kv, orc, w1, 0, 20, rep, starts=[7 * 128 + 50, 5 * 128])
+    assert kv.stats()["device_error"] == 0
+
+
 @pytest.mark.parametrize("pinned", [True, False])
 def test_host_entry_points_match_device_entry_points(gpu, pinned):
     """Page-locked host tensors are read by the decode kernel directly; pageable ones go through staging copies."""
