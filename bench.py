@@ -387,6 +387,8 @@ def main():
                     help="prefill legs: keep every kernel of a chunk on the caller's stream (TREEKV_OPT_EVICTION_STREAM off)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS)
+    ap.add_argument("--prefill-path", type=int, default=0, help="TREEKV_OPT_PREFILL_PATH for the prefill legs; 0 = automatic")
+    ap.add_argument("--prefill-key-split", type=int, default=0, help="TREEKV_OPT_PREFILL_KEY_SPLIT; 0 = automatic")
     ap.add_argument("--decode-split", type=int, default=0, help="thread blocks per (sequence, KV head); 0 = automatic")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling small cases)")
     args = ap.parse_args()
@@ -435,7 +437,7 @@ def main():
     prefill_legs = []
     for name in [x for x in args.prefill_legs.split(",") if x]:
         prefill_legs.append(run_prefill_leg(torch, binding, cfg(name), max(1, args.prefill_chunks), dev, rep, timer, peaks,
-                                            not args.no_eviction_stream))
+                                            not args.no_eviction_stream, args.prefill_path, args.prefill_key_split))
     prefill = prefill_legs[0] if prefill_legs else None
     if sampler is not None:
         sampler.stop()
@@ -562,14 +564,18 @@ def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev
             "config": config_of(w)}
 
 
-def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks, eviction_stream=True):
+def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks, eviction_stream=True, prefill_path=0, key_split=0):
     tdtype = torch.bfloat16 if pw.dtype == "bf16" else torch.float32
     world, rank = rep.world, rep.rank
     m, c = pw.chunk, pw.budget
     ctxs = [binding.TreeKV(c, pw.n_heads, pw.n_kv_heads, pw.head_dim, pw.dtype, pw.batch, m) for _ in range(pw.layers)]
-    if eviction_stream:
-        for x in ctxs:
+    for x in ctxs:
+        if eviction_stream:
             x.set_option(binding.OPT_EVICTION_STREAM, 1)
+        if prefill_path:
+            x.set_option(binding.OPT_PREFILL_PATH, prefill_path)
+        if key_split:
+            x.set_option(binding.OPT_PREFILL_KEY_SPLIT, key_split)
     wr = W.parity_slice(pw, seed=pw.seed + 1000 * rank)
     ins = []
     for layer in range(pw.layers):   # the same chunk values every call: timing does not depend on them

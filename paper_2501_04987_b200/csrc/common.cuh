@@ -287,7 +287,8 @@ struct ChunkTensors {
 size_t prefill_tc2_smem_bytes();
 cudaError_t launch_prefill_tc2(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                                const CUtensorMap& tmV, const ChunkTensors& ct, void* out, const ChunkLens& lens,
-                               int chunk_stride, int max_m, cudaStream_t stream);  // 256 query rows per CTA, for large grids
+                               int chunk_stride, int max_m, int key_split, cudaStream_t stream);  // 256 query rows per CTA;
+                               // key_split 2: pairs of CTAs that share the query rows and halve the key tiles
 
 size_t prefill_tc_smem_bytes();
 cudaError_t launch_prefill_tc(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,

@@ -19,6 +19,7 @@ struct treekv_ctx {
     int opt_prefill_path;
     int opt_decode_path;
     int opt_prefill_append;
+    int opt_prefill_key_split;
     // eviction stream (TREEKV_OPT_EVICTION_STREAM): the score update + eviction kernel of a chunk runs on `side`, after
     // the chunk's attention (ev_attn), and everything enqueued later for this context waits for it (ev_state)
     cudaStream_t side;

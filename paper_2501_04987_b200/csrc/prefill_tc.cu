@@ -226,7 +226,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
                         for (int e = 0; e < 32; e += 2) {
                             s0 += ex2(fmaf(__uint_as_float(v[e]), sc2, -mnew));
-                            s1 += ex2(fmaf(__uint_as_float(v[e + 1]), sc2, -mnew));
+                            const float x1 = fmaf(__uint_as_float(v[e + 1]), sc2, -mnew);
+                            s1 += ((e + 1) % kPolyEvery == kPolyEvery - 1) ? ex2_poly(x1) : ex2(x1);
                         }
                         lrun = lrun * ex2(mrun - mnew) + (s0 + s1);
                         mrun = mnew;

@@ -26,18 +26,20 @@ using namespace tc;
 
 constexpr int kRing = 3;       // K / V tiles in flight
 
-enum Bar { Q_FULL = 0, RING_FULL = 1, RING_EMPTY = 4, S_FULL = 7, S_FREE = 11, P_FULL = 15, P_FREE = 17, O_FULL = 19, N_BARS = 20 };
+enum Bar { Q_FULL = 0, RING_FULL = 1, RING_EMPTY = 4, S_FULL = 7, S_FREE = 11, P_FULL = 15, P_FREE = 17, O_FULL = 19,
+           X_STATS = 20, X_FREE = 21, X_RECV = 22, N_BARS = 23 };  // X_*: signalled by the other CTA of a key-split pair
 
 }  // namespace
 
-template <int G>
+template <int G, int KS>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKin,
                    const __grid_constant__ CUtensorMap tmVin, ChunkDirect cd, CacheView cv, PrefillScratch ps,
                    __nv_bfloat16* __restrict__ out, ChunkLens lens, int chunk_stride) {
     constexpr int TOK = 128 / G;  // tokens per sub-tile
-    const int unit = blockIdx.y, qt2 = blockIdx.x;
+    const int unit = blockIdx.y, qt2 = blockIdx.x / KS;
+    const int ks = KS > 1 ? (int)(blockIdx.x % KS) : 0;  // rank in the key-split cluster (cluster = KS consecutive blockIdx.x)
     const int b = unit / cv.Hkv, kh = unit % cv.Hkv;
     const int m = lens.m[b];
     const int t0c = qt2 * 2 * TOK;  // first token of the CTA
@@ -48,6 +50,9 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const KeyTiles kt = key_tiles(st, st.L + t1c, cd.k != nullptr);
     const int NT = kt.NT;
     const int n = st.L + m;
+    // this CTA's key tiles [jb, jb + nt): all of them, or its half (rank 0 the first, larger one: never empty)
+    const int jb = (KS > 1 && ks == 1) ? (NT + 1) / 2 : 0;
+    const int nt = KS > 1 ? (ks == 0 ? (NT + 1) / 2 : NT - (NT + 1) / 2) : NT;
 
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const uint32_t base = smem_addr_u32(smem_raw);
@@ -68,6 +73,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int s = 0; s < 4; ++s) { mbar_init(bar(S_FULL + s), 1); mbar_init(bar(S_FREE + s), 8); }
         for (int s = 0; s < 2; ++s) { mbar_init(bar(P_FULL + s), 8); mbar_init(bar(P_FREE + s), 1); }
         mbar_init(bar(O_FULL), 1);
+        mbar_init(bar(X_STATS), 8); mbar_init(bar(X_FREE), 1); mbar_init(bar(X_RECV), 16);
         mbar_fence_init();
         if (base & 1023u) atomicOr(&cv.stats->error, 32u);  // the tiles' swizzle needs a 1024-byte aligned base
     }
@@ -76,6 +82,8 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // both CTAs of a pair are running and their barriers are initialised before either signals the other
+    if constexpr (KS > 1) cluster_sync_all();
 
     bool ok = true;
     if (warp == 0) {
@@ -90,7 +98,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             int ld = 0;
             auto load_tile = [&](const CUtensorMap* mp, const CUtensorMap* mp_in, int j) {
                 int lam0, row0, valid;
-                const bool from_chunk = tile_of(kt, j, lam0, row0, valid);
+                const bool from_chunk = tile_of(kt, jb + j, lam0, row0, valid);
                 const int slot = ld % kRing;
                 if (!mbar_wait(bar(RING_EMPTY + slot), ((ld / kRing) & 1) ^ 1)) { ok = false; return; }
                 const uint32_t dst = sRing + slot * kSlot;
@@ -106,10 +114,10 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 ++ld;
             };
             // pass A: K tiles in order.  Pass B, in the order the MMA warp consumes them: K_0 | K_1 V_0 | K_2 V_1 | ...
-            for (int j = 0; j < NT && ok; ++j) load_tile(&tmK, &tmKin, j);
-            if (ok) load_tile(&tmK, &tmKin, 0);
-            for (int j = 0; j < NT && ok; ++j) {
-                if (j + 1 < NT) load_tile(&tmK, &tmKin, j + 1);
+            for (int j = 0; j < nt && ok; ++j) load_tile(&tmK, &tmKin, j);
+            if (ok && nt > 0) load_tile(&tmK, &tmKin, 0);
+            for (int j = 0; j < nt && ok; ++j) {
+                if (j + 1 < nt) load_tile(&tmK, &tmKin, j + 1);
                 if (ok) load_tile(&tmV, &tmVin, j);
             }
             if (!ok) atomicOr(&cv.stats->error, 4u);
@@ -135,7 +143,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 return r;
             };
             // ---- pass A: S_s = Q_s K_j^T into buffer 2 s + (j & 1)
-            for (int j = 0; j < NT && ok; ++j) {
+            for (int j = 0; j < nt && ok; ++j) {
                 int slot;
                 if (!(ok = ring_wait(slot))) break;
                 const uint32_t sK = sRing + slot * kSlot;
@@ -178,9 +186,9 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 umma_commit(bar(RING_EMPTY + slot));
                 (void)j;
             };
-            if (ok) issue_st(0);
-            for (int pj = 0; pj < NT && ok; ++pj) {
-                if (pj + 1 < NT) { issue_st(pj + 1); if (!ok) break; }
+            if (ok && nt > 0) issue_st(0);
+            for (int pj = 0; pj < nt && ok; ++pj) {
+                if (pj + 1 < nt) { issue_st(pj + 1); if (!ok) break; }
                 int slot;
                 if (!(ok = ring_wait(slot))) break;
                 const uint32_t sV = sRing + slot * kSlot;
@@ -224,13 +232,13 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         {
             const int tq = max(t0c, min(t0 + row / G, t1 - 1));  // rows past the chunk repeat a real row: finite, unused
             float mrun = -INFINITY, lrun = 0.f;
-            for (int j = 0; j < NT && ok; ++j) {
+            for (int j = 0; j < nt && ok; ++j) {
                 const int buf = 2 * sub + (j & 1);
                 const uint32_t tmSg = tmem + buf * 128 + lane_off;
                 if (!mbar_wait(bar(S_FULL + buf), (j >> 1) & 1)) { ok = false; break; }
                 tc_fence_after();
                 int lam0, row0, valid;
-                tile_of(kt, j, lam0, row0, valid);
+                tile_of(kt, jb + j, lam0, row0, valid);
                 const int limit = max(0, min(valid, kt.L + tq - lam0 + 1));  // columns [0, limit) are visible to this row
                 const bool full = __all_sync(0xffffffffu, limit >= 128);
                 auto stats32 = [&](const uint32_t (&v)[32], int cg) {
@@ -243,7 +251,8 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                         for (int e = 0; e < 32; e += 2) {
                             s0 += ex2(fmaf(__uint_as_float(v[e]), sc2, -mnew));
-                            s1 += ex2(fmaf(__uint_as_float(v[e + 1]), sc2, -mnew));
+                            const float x1 = fmaf(__uint_as_float(v[e + 1]), sc2, -mnew);
+                            s1 += ((e + 1) % kPolyEvery == kPolyEvery - 1) ? ex2_poly(x1) : ex2(x1);
                         }
                         lrun = lrun * ex2(mrun - mnew) + (s0 + s1);
                         mrun = mnew;
@@ -283,9 +292,25 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         asm volatile("bar.sync 1, 512;" ::: "memory");
         if (half == 0) {
             const float m0 = part_m[(sub * 2) * 128 + row], m1 = part_m[(sub * 2 + 1) * 128 + row];
-            const float M = fmaxf(m0, m1);
-            const float l = (m0 == -INFINITY ? 0.f : part_l[(sub * 2) * 128 + row] * ex2(m0 - M)) +
-                            (m1 == -INFINITY ? 0.f : part_l[(sub * 2 + 1) * 128 + row] * ex2(m1 - M));
+            float M = fmaxf(m0, m1);
+            float l = (m0 == -INFINITY ? 0.f : part_l[(sub * 2) * 128 + row] * ex2(m0 - M)) +
+                      (m1 == -INFINITY ? 0.f : part_l[(sub * 2 + 1) * 128 + row] * ex2(m1 - M));
+            if constexpr (KS > 1) {
+                // the other half of the keys: hand over this half's (max, sum), take the other's, combine - rank 0's
+                // term first on both sides, so the two CTAs normalise with the same log-sum-exp bit for bit
+                float* xstat = part_m + 1024;  // [2][128] x (max, sum), written by the other CTA
+                const uint32_t peer = (uint32_t)(ks ^ 1);
+                st_remote_v2(map_to_cta(smem_addr_u32(xstat + 2 * (sub * 128 + row)), peer), M, l);
+                fence_cluster();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(map_to_cta(bar(X_STATS), peer));
+                if (!mbar_wait_cluster(bar(X_STATS), 0)) ok = false;
+                const float2 o = *reinterpret_cast<const float2*>(xstat + 2 * (sub * 128 + row));
+                const float Mx = fmaxf(M, o.x);
+                const float la = M == -INFINITY ? 0.f : l * ex2(M - Mx), lb = o.x == -INFINITY ? 0.f : o.y * ex2(o.x - Mx);
+                l = ks == 0 ? la + lb : lb + la;
+                M = Mx;
+            }
             nlse[row] = -(M + log2f(l));
         }
         asm volatile("bar.sync 1, 512;" ::: "memory");  // lse[] is complete; the P^T area is free for pass B
@@ -294,14 +319,14 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         // observation window (one-shot prefill): only the last ps.window tokens of the chunk add to the column sums
         const int rwin = ps.window > 0 ? max(0, G * (m - ps.window - t0)) : 0;
         float* part = ps.colsum + ((size_t)unit * ps.QT + 2 * qt2 + sub) * ps.n_max;
-        const int fills_a = sub == 0 ? (NT + 1) / 2 : NT / 2;  // times pass A filled barrier pair `sub` (buffers 0 and 1)
+        const int fills_a = sub == 0 ? (nt + 1) / 2 : nt / 2;  // times pass A filled barrier pair `sub` (buffers 0 and 1)
         float* xrow = xch + sub * 128;
-        for (int j = 0; j < NT && ok; ++j) {
+        for (int j = 0; j < nt && ok; ++j) {
             const uint32_t tmSg = tmem + sub * 128 + lane_off;
             if (!mbar_wait(bar(S_FULL + sub), (fills_a + j) & 1)) { ok = false; break; }
             tc_fence_after();
             int lam0, row0, valid;
-            tile_of(kt, j, lam0, row0, valid);
+            tile_of(kt, jb + j, lam0, row0, valid);
             const bool kvalid = row < valid;
             const int lam = lam0 + row;
             const int rmin = kvalid ? max(0, G * (lam - kt.L - t0)) : 128;  // first query column that sees this key
@@ -381,22 +406,67 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             if (lane == 0) mbar_arrive(bar(P_FULL + sub));
         }
         // keys this CTA's queries cannot see contribute nothing
-        if (sub_live)
+        if (sub_live && ks == 0)
             for (int lam = kt.nvis + (tid - 64 - sub * 256); lam < n; lam += 256) part[lam] = 0.f;
-        // ---- epilogue: O_s^T (lane = channel, column = query row) -> out[token][head][channel]; 64 query columns per warp
+        // ---- epilogue: O_s^T (lane = channel, column = query row) -> out[token][head][channel]
         if (ok && mbar_wait(bar(O_FULL), 0)) {
             tc_fence_after();
+            if constexpr (KS == 1) {  // 64 query columns per warp
 #pragma unroll 1
-            for (int cg = 2 * half; cg < 2 * half + 2; ++cg) {
-                tmem_ld32(tmem + (2 + sub) * 128 + lane_off + cg * 32, va);
-                tmem_ld_wait_for(va);
+                for (int cg = 2 * half; cg < 2 * half + 2; ++cg) {
+                    tmem_ld32(tmem + (2 + sub) * 128 + lane_off + cg * 32, va);
+                    tmem_ld_wait_for(va);
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const int r = cg * 32 + e;
-                    if (r < rmax)
-                        out[(((size_t)b * chunk_stride + t0 + r / G) * cv.Hq + kh * G + (r % G)) * kD + row] =
-                            __float2bfloat16_rn(__uint_as_float(va[e]));
+                    for (int e = 0; e < 32; ++e) {
+                        const int r = cg * 32 + e;
+                        if (r < rmax)
+                            out[(((size_t)b * chunk_stride + t0 + r / G) * cv.Hq + kh * G + (r % G)) * kD + row] =
+                                __float2bfloat16_rn(__uint_as_float(va[e]));
+                    }
                 }
+            } else {
+                // Every MMA of this CTA has completed, so its ring is idle: tell the other CTA, which stages there the
+                // partial O^T of the sub-tile this CTA finishes.  A warp takes 32 query columns of its lane quarter:
+                // first of the other CTA's sub-tile (sent), then of its own (summed with what was received).
+                const uint32_t peer = (uint32_t)(ks ^ 1);
+                const int cg = sw >> 2;  // query columns [32 cg, 32 cg + 32)
+                const uint32_t stage = sRing + (uint32_t)((cg * 4 + quarter) * 32 * 32 * 4);  // [8 groups of 4 columns][32 lanes][4]
+                if (sw == 0 && lane == 0) mbar_arrive_remote(map_to_cta(bar(X_FREE), peer));
+                if (mbar_wait_cluster(bar(X_FREE), 0)) {
+                    tmem_ld32(tmem + (2 + (ks ^ 1)) * 128 + lane_off + cg * 32, va);
+                    tmem_ld_wait_for(va);
+                    const uint32_t dst = map_to_cta(stage, peer) + (uint32_t)lane * 16u;
+#pragma unroll
+                    for (int v4 = 0; v4 < 8; ++v4) {
+                        // a CTA without key tiles never wrote its accumulators: its partial is zero
+                        const float x0 = nt > 0 ? __uint_as_float(va[4 * v4]) : 0.f, x1 = nt > 0 ? __uint_as_float(va[4 * v4 + 1]) : 0.f;
+                        const float x2 = nt > 0 ? __uint_as_float(va[4 * v4 + 2]) : 0.f, x3 = nt > 0 ? __uint_as_float(va[4 * v4 + 3]) : 0.f;
+                        st_remote_v4(dst + (uint32_t)v4 * 512u, x0, x1, x2, x3);
+                    }
+                    fence_cluster();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_remote(map_to_cta(bar(X_RECV), peer));
+                } else {
+                    ok = false;
+                }
+                if (ok && mbar_wait_cluster(bar(X_RECV), 0)) {
+                    tmem_ld32(tmem + (2 + ks) * 128 + lane_off + cg * 32, va);
+                    tmem_ld_wait_for(va);
+                    const int t0o = t0c + ks * TOK;                     // this CTA finishes sub-tile ks
+                    const int rmaxo = t0o < m ? G * (min(t0o + TOK, m) - t0o) : 0;
+                    const float* rcv = reinterpret_cast<const float*>(smem_raw + (stage - base)) + lane * 4;
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const int r = cg * 32 + e;
+                        const float mine = nt > 0 ? __uint_as_float(va[e]) : 0.f, theirs = rcv[(e >> 2) * 128 + (e & 3)];
+                        if (r < rmaxo)
+                            out[(((size_t)b * chunk_stride + t0o + r / G) * cv.Hq + kh * G + (r % G)) * kD + row] =
+                                __float2bfloat16_rn(ks == 0 ? mine + theirs : theirs + mine);
+                    }
+                } else {
+                    ok = false;
+                }
+                if (!ok) atomicOr(&cv.stats->error, 16u);
             }
             tc_fence_before();
         } else {
@@ -404,16 +474,18 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
     }
     __syncthreads();
+    // neither CTA of a pair exits while the other may still write into its shared memory or signal its barriers
+    if constexpr (KS > 1) cluster_sync_all();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
 size_t prefill_tc2_smem_bytes() { return (size_t)(4 + kRing) * kSlot + 512 * sizeof(float) + N_BARS * 8 + 16; }
 
-template <int G>
+template <int G, int KS>
 static cudaError_t launch_prefill_tc2_t(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ,
                                         const CUtensorMap& tmK, const CUtensorMap& tmV, const ChunkTensors& ct, void* out,
                                         const ChunkLens& lens, int chunk_stride, int max_m, cudaStream_t stream) {
-    auto kern = prefill_tc2_kernel<G>;
+    auto kern = prefill_tc2_kernel<G, KS>;
     const size_t smem = prefill_tc2_smem_bytes();
     static bool smem_set[64] = {};  // per device: the opt-in is needed once
     int dev = 0;
@@ -424,23 +496,38 @@ static cudaError_t launch_prefill_tc2_t(const CacheView& cv, const PrefillScratc
         if (e != cudaSuccess) return e;
         smem_set[dev] = true;
     }
-    dim3 grid((max_m * G + 2 * kQTileRows - 1) / (2 * kQTileRows), cv.B * cv.Hkv);
     const ChunkDirect cd = {reinterpret_cast<const __nv_bfloat16*>(ct.k), reinterpret_cast<const __nv_bfloat16*>(ct.v)};
-    kern<<<grid, kThreads, smem, stream>>>(tmQ, tmK, tmV, ct.k ? ct.tmK : tmK, ct.k ? ct.tmV : tmV, cd, cv, ps,
-                                           reinterpret_cast<__nv_bfloat16*>(out), lens, chunk_stride);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(KS * ((max_m * G + 2 * kQTileRows - 1) / (2 * kQTileRows)), cv.B * cv.Hkv);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = KS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = KS > 1 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, tmQ, tmK, tmV, ct.k ? ct.tmK : tmK, ct.k ? ct.tmV : tmV, cd, cv, ps,
+                              reinterpret_cast<__nv_bfloat16*>(out), lens, chunk_stride);
 }
 
 cudaError_t launch_prefill_tc2(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                                const CUtensorMap& tmV, const ChunkTensors& ct, void* out, const ChunkLens& lens,
-                               int chunk_stride, int max_m, cudaStream_t stream) {
-    if (cv.d != kD) return cudaErrorInvalidValue;
+                               int chunk_stride, int max_m, int key_split, cudaStream_t stream) {
+    if (cv.d != kD || (key_split != 1 && key_split != 2)) return cudaErrorInvalidValue;
+#define TREEKV_TC2_CASE(g)                                                                                           \
+    case g:                                                                                                          \
+        return key_split == 2 ? launch_prefill_tc2_t<g, 2>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream) \
+                              : launch_prefill_tc2_t<g, 1>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
     switch (cv.Hq / cv.Hkv) {
-        case 1: return launch_prefill_tc2_t<1>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
-        case 2: return launch_prefill_tc2_t<2>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
-        case 4: return launch_prefill_tc2_t<4>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
-        case 8: return launch_prefill_tc2_t<8>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
+        TREEKV_TC2_CASE(1)
+        TREEKV_TC2_CASE(2)
+        TREEKV_TC2_CASE(4)
+        TREEKV_TC2_CASE(8)
     }
+#undef TREEKV_TC2_CASE
     return cudaErrorInvalidValue;
 }
 

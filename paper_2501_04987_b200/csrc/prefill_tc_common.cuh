@@ -87,5 +87,24 @@ __device__ inline float ex2(float x) {
     return y;
 }
 
+
+// 2^x for x <= 0 on the FMA and integer pipes (no special-function unit): x = n + f with n the nearest integer (taken
+// from the low mantissa bits of x + 1.5 * 2^23) and f in [-0.5, 0.5]; 2^f by a degree-4 polynomial (least-maximum
+// relative error fit, 2.9e-6 at most, mean 3e-7); 2^n by adding n to the exponent field.  Inputs below -125 give
+// 2^-125.  The special-function unit delivers 16 results per clock and SM, which is what bounds the statistics pass;
+// a share of its elements goes through here instead.
+__device__ inline float ex2_poly(float x) {
+    x = fmaxf(x, -125.0f);
+    const float t = __fadd_rn(x, 12582912.0f);
+    const float f = __fsub_rn(x, __fsub_rn(t, 12582912.0f));
+    float p = fmaf(0.00958283618092537f, f, 0.055906426161527634f);
+    p = fmaf(p, f, 0.24024099111557007f);
+    p = fmaf(p, f, 0.6931241750717163f);
+    p = fmaf(p, f, 1.0f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+// every kPolyEvery-th element of a row's 32-column chunk takes the polynomial in the statistics pass
+constexpr int kPolyEvery = 4;
+
 }  // namespace tc
 }  // namespace treekv

@@ -40,6 +40,47 @@ __device__ inline bool mbar_wait_limit(uint32_t bar, uint32_t parity, uint32_t l
     return false;
 }
 __device__ inline bool mbar_wait(uint32_t bar, uint32_t parity) { return mbar_wait_limit(bar, parity, kSpinLimit); }
+// ---- thread-block clusters: the same barriers and stores, aimed at another block of the cluster
+__device__ inline uint32_t cluster_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// cluster-wide address of `saddr` (a shared::cta address of this block's layout) in block `rank` of the cluster
+__device__ inline uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ inline void st_remote_v4(uint32_t caddr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(caddr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ inline void st_remote_v2(uint32_t caddr, float a, float b) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(caddr), "f"(a), "f"(b) : "memory");
+}
+__device__ inline void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+// one arrival on a barrier of another block; earlier stores of this thread (and, after a fence_cluster + __syncwarp,
+// of its warp) to that block's shared memory are visible to a thread that then passes mbar_wait_cluster
+__device__ inline void mbar_arrive_remote(uint32_t caddr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
+}
+__device__ inline bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {  // bounded; acquire at cluster scope
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+// every thread of every block of the cluster (all of them must call it, converged)
+__device__ inline void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // orders earlier generic-proxy accesses to shared memory before later async-proxy (TMA, tcgen05.mma) accesses
 __device__ inline void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 

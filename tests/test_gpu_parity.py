@@ -104,17 +104,21 @@ def test_cfg5_slice_ragged_gqa_prefill(gpu):
     print("cfg5 slice", rep)
 
 
+@pytest.mark.parametrize("key_split", [1, 2])
 @pytest.mark.parametrize("g,lens,chunk,budget", [
     (4, [2 * 1024 + 517, 2 * 1024 + 40], 512, 1024),   # GQA, ragged tails: a partial last tile and an empty second sub-tile
     (1, [5 * 384 + 200, 3 * 384], 384, 512),           # MHA, 1.5 pairs of tiles per chunk, chunks that wrap the idx cycle
     (8, [1300, 64], 256, 256),                         # eight heads per group: 16 tokens per sub-tile
+    (2, [3 * 64 + 9, 50], 64, 96),                     # a first chunk of one key tile: the second block of a key-split pair has none
 ])
-def test_two_tile_tensor_core_prefill_kernel(gpu, g, lens, chunk, budget):
+def test_two_tile_tensor_core_prefill_kernel(gpu, g, lens, chunk, budget, key_split):
     """The prefill kernel that gives a thread block two tiles of 128 query rows is only chosen for large grids;
-    here it is forced on small ragged cases and followed in lock-step like the one-tile kernel."""
+    here it is forced on small ragged cases and followed in lock-step like the one-tile kernel - one block per tile
+    pair, and pairs of blocks that split the key tiles and exchange row statistics and partial outputs."""
     w = W.parity_slice(W.CONFIGS["cfg5"], layers=1, batch=2, n_heads=g * 2, n_kv_heads=2, budget=budget, chunk=chunk)
     kv, orc = _pair(gpu, w)
     kv.set_option(gpu.OPT_PREFILL_PATH, 3)
+    kv.set_option(gpu.OPT_PREFILL_KEY_SPLIT, key_split)
     rep = Report()
     _run_prefill(kv, orc, w, rep, lens, chunk)
     assert [kv.tokens_seen(b) for b in range(2)] == lens
