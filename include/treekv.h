@@ -76,7 +76,8 @@ typedef enum {
                                     chunk length is a multiple of 128 (no separate append kernel); 1 = always append with
                                     a kernel of its own before the attention.  Same result either way. */
     TREEKV_OPT_PREFILL_KEY_SPLIT = 5, /* thread blocks that share the 256 query rows of a tile pair in the two-tile tensor-core
-                                    prefill kernel, each taking a share of the key tiles: 0 = automatic, 1, 2 */
+                                    prefill kernel, each taking a share of the key tiles: 0 (default) and 1 = one block, 2 = a pair of blocks
+                                    that halve the key tiles and exchange row statistics and partial outputs */
     TREEKV_OPT_EVICTION_STREAM = 4 /* 0 (default) = every kernel of a call runs on the caller's stream.  1 = the last
                                     kernel of treekv_prefill_chunk (score update + eviction + compaction, which only
                                     touches the workspace) runs on a stream the context owns, behind the chunk's

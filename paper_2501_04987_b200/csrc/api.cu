@@ -269,18 +269,13 @@ treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, 
         const uint64_t strides[2] = {256ull, (uint64_t)ctx->cv.Hq * 256ull};
         const uint32_t box[3] = {64u, (uint32_t)ctx->G, (uint32_t)(128 / ctx->G)};
         if (!make_tensor_map_bf16(&tmQ, dev_q, 3, dims, strides, box)) return TREEKV_ERR_CUDA;
-        // Which kernel: two query tiles per CTA (the more efficient shape: every K / V tile load feeds twice the tensor
-        // work) whenever its grid - if need be with the key tiles of a tile pair split over two CTAs - still covers
-        // most of the machine; one tile per CTA for smaller calls.  The key split is taken when it fills the last wave
-        // noticeably better (fewer CTAs than SMs, or a mostly empty last wave).
-        const long sms = ctx->sm_count;
-        const long pairs = (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + 2 * kQTileRows - 1) / (2 * kQTileRows));
-        const bool two = ctx->opt_prefill_path == 3 || (ctx->opt_prefill_path == 0 && 2 * pairs >= sms * 3 / 4);
-        int ks = ctx->opt_prefill_key_split;
-        if (two && ks == 0) {
-            auto fill = [&](long ctas) { return (double)ctas / (double)(((ctas + sms - 1) / sms) * sms); };
-            ks = fill(2 * pairs) > 1.04 * fill(pairs) ? 2 : 1;
-        }
+        // Which kernel: two query tiles per CTA (every K / V tile load feeds twice the tensor work) once the one-tile grid
+        // would cover the machine at least twice, one tile per CTA for smaller calls.  Splitting a tile pair's key tiles
+        // over two CTAs is on request only: measured, what the pair exchanges and sets up twice costs more than the
+        // fuller last wave gives back.
+        const long tiles = (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + kQTileRows - 1) / kQTileRows);
+        const bool two = ctx->opt_prefill_path == 3 || (ctx->opt_prefill_path == 0 && tiles >= 2L * ctx->sm_count);
+        const int ks = ctx->opt_prefill_key_split == 2 ? 2 : 1;
         e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, ks, s)
                 : launch_prefill_tc(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, s);
     } else {

@@ -226,8 +226,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
                         for (int e = 0; e < 32; e += 2) {
                             s0 += ex2(fmaf(__uint_as_float(v[e]), sc2, -mnew));
-                            const float x1 = fmaf(__uint_as_float(v[e + 1]), sc2, -mnew);
-                            s1 += ((e + 1) % kPolyEvery == kPolyEvery - 1) ? ex2_poly(x1) : ex2(x1);
+                            s1 += ex2(fmaf(__uint_as_float(v[e + 1]), sc2, -mnew));
                         }
                         lrun = lrun * ex2(mrun - mnew) + (s0 + s1);
                         mrun = mnew;
@@ -371,21 +370,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         // keys this tile's queries cannot see contribute nothing
         for (int lam = kt.nvis + (tid - 64); lam < n; lam += 512) part[lam] = 0.f;
-        // ---- epilogue: O^T (lane = channel, column = query row) -> out[token][head][channel]; 32 query columns per warp
+        // ---- epilogue: O^T (lane = channel, column = query row) -> out[token][head][channel], staged through the idle
+        //      P^T area so that whole rows are written; the four warps (lane quarters) that share 32 query columns
+        //      synchronise on a barrier of their own
         if (ok && mbar_wait(bar(O_FULL), 0)) {
             tc_fence_after();
-            {
-                const int cg = sw >> 2;  // one chunk of 32 query columns per warp
-                tmem_ld32(tmO + lane_off + cg * 32, va);
-                tmem_ld_wait_for(va);
+            const int cg = sw >> 2;  // one chunk of 32 query columns per warp
+            unsigned char* stage = base_ptr + (1 + kRing) * kSlot;
+            tmem_ld32(tmO + lane_off + cg * 32, va);
+            tmem_ld_wait_for(va);
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const int r = cg * 32 + e;
-                    if (r < rmax)
-                        out[(((size_t)b * chunk_stride + t0 + r / G) * cv.Hq + kh * G + (r % G)) * kD + row] =
-                            __float2bfloat16_rn(__uint_as_float(va[e]));
-                }
-            }
+            for (int e = 0; e < 32; ++e) stage_put(stage, cg * 32 + e, row, __uint_as_float(va[e]));
+            asm volatile("bar.sync %0, 128;" ::"r"(10 + cg) : "memory");
+            stage_flush<G>(stage, out, (size_t)b * chunk_stride + t0, cv.Hq, kh, cg * 32, 32, rmax, quarter * 32 + lane, 128);
             tc_fence_before();
         } else {
             atomicOr(&cv.stats->error, 16u);

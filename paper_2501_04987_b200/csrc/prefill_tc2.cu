@@ -251,8 +251,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                         for (int e = 0; e < 32; e += 2) {
                             s0 += ex2(fmaf(__uint_as_float(v[e]), sc2, -mnew));
-                            const float x1 = fmaf(__uint_as_float(v[e + 1]), sc2, -mnew);
-                            s1 += ((e + 1) % kPolyEvery == kPolyEvery - 1) ? ex2_poly(x1) : ex2(x1);
+                            s1 += ex2(fmaf(__uint_as_float(v[e + 1]), sc2, -mnew));
                         }
                         lrun = lrun * ex2(mrun - mnew) + (s0 + s1);
                         mrun = mnew;
@@ -411,19 +410,19 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         // ---- epilogue: O_s^T (lane = channel, column = query row) -> out[token][head][channel]
         if (ok && mbar_wait(bar(O_FULL), 0)) {
             tc_fence_after();
-            if constexpr (KS == 1) {  // 64 query columns per warp
+            if constexpr (KS == 1) {
+                // 64 query columns per warp, staged through the sub-tile's idle P^T buffer so that whole rows are
+                // written; the four warps (lane quarters) of a column half synchronise on a barrier of their own
+                unsigned char* stage = p_area + sub * kSlot;
 #pragma unroll 1
                 for (int cg = 2 * half; cg < 2 * half + 2; ++cg) {
                     tmem_ld32(tmem + (2 + sub) * 128 + lane_off + cg * 32, va);
                     tmem_ld_wait_for(va);
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const int r = cg * 32 + e;
-                        if (r < rmax)
-                            out[(((size_t)b * chunk_stride + t0 + r / G) * cv.Hq + kh * G + (r % G)) * kD + row] =
-                                __float2bfloat16_rn(__uint_as_float(va[e]));
-                    }
+                    for (int e = 0; e < 32; ++e) stage_put(stage, cg * 32 + e, row, __uint_as_float(va[e]));
                 }
+                asm volatile("bar.sync %0, 128;" ::"r"(10 + sub * 2 + half) : "memory");
+                stage_flush<G>(stage, out, (size_t)b * chunk_stride + t0, cv.Hq, kh, 64 * half, 64, rmax, quarter * 32 + lane, 128);
             } else {
                 // Every MMA of this CTA has completed, so its ring is idle: tell the other CTA, which stages there the
                 // partial O^T of the sub-tile this CTA finishes.  A warp takes 32 query columns of its lane quarter:
@@ -455,14 +454,14 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     const int t0o = t0c + ks * TOK;                     // this CTA finishes sub-tile ks
                     const int rmaxo = t0o < m ? G * (min(t0o + TOK, m) - t0o) : 0;
                     const float* rcv = reinterpret_cast<const float*>(smem_raw + (stage - base)) + lane * 4;
+                    unsigned char* ostage = p_area;  // rows are put together in the idle P^T area, see the one-CTA case
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
-                        const int r = cg * 32 + e;
                         const float mine = nt > 0 ? __uint_as_float(va[e]) : 0.f, theirs = rcv[(e >> 2) * 128 + (e & 3)];
-                        if (r < rmaxo)
-                            out[(((size_t)b * chunk_stride + t0o + r / G) * cv.Hq + kh * G + (r % G)) * kD + row] =
-                                __float2bfloat16_rn(ks == 0 ? mine + theirs : theirs + mine);
+                        stage_put(ostage, cg * 32 + e, row, ks == 0 ? mine + theirs : theirs + mine);
                     }
+                    asm volatile("bar.sync %0, 128;" ::"r"(10 + cg) : "memory");
+                    stage_flush<G>(ostage, out, (size_t)b * chunk_stride + t0o, cv.Hq, kh, cg * 32, 32, rmaxo, quarter * 32 + lane, 128);
                 } else {
                     ok = false;
                 }

@@ -88,23 +88,28 @@ __device__ inline float ex2(float x) {
 }
 
 
-// 2^x for x <= 0 on the FMA and integer pipes (no special-function unit): x = n + f with n the nearest integer (taken
-// from the low mantissa bits of x + 1.5 * 2^23) and f in [-0.5, 0.5]; 2^f by a degree-4 polynomial (least-maximum
-// relative error fit, 2.9e-6 at most, mean 3e-7); 2^n by adding n to the exponent field.  Inputs below -125 give
-// 2^-125.  The special-function unit delivers 16 results per clock and SM, which is what bounds the statistics pass;
-// a share of its elements goes through here instead.
-__device__ inline float ex2_poly(float x) {
-    x = fmaxf(x, -125.0f);
-    const float t = __fadd_rn(x, 12582912.0f);
-    const float f = __fsub_rn(x, __fsub_rn(t, 12582912.0f));
-    float p = fmaf(0.00958283618092537f, f, 0.055906426161527634f);
-    p = fmaf(p, f, 0.24024099111557007f);
-    p = fmaf(p, f, 0.6931241750717163f);
-    p = fmaf(p, f, 1.0f);
-    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+// Output staging.  O^T leaves tensor memory with a thread holding one channel of 32 query rows; written to `out` like
+// that, a warp store covers 64 bytes of one row.  Instead the rows are put together in shared memory - [128 query
+// rows][256 bytes], the 16-byte pieces of row r XOR-swizzled by (r & 15) so that both the 2-byte puts (a warp: 32
+// consecutive channels of one row) and the 16-byte gets (a quarter warp: 8 pieces of one row) are conflict-free -
+// and go out as whole 256-byte rows.
+__device__ inline void stage_put(unsigned char* stage, int r, int ch, float x) {
+    *reinterpret_cast<__nv_bfloat16*>(stage + r * 256 + ((((ch >> 3) ^ (r & 15)) << 4) | ((ch & 7) << 1))) =
+        __float2bfloat16_rn(x);
 }
-// every kPolyEvery-th element of a row's 32-column chunk takes the polynomial in the statistics pass
-constexpr int kPolyEvery = 4;
+// rows [r0, r0 + nrows) of the staged tile (those below rmax) -> out[token][head][channel]; row r is token r / G,
+// head r % G of the tile whose first token has index tok0 in the call's tensor; threads t of nthr take part
+template <int G>
+__device__ inline void stage_flush(const unsigned char* stage, __nv_bfloat16* __restrict__ out, size_t tok0, int Hq, int kh,
+                                   int r0, int nrows, int rmax, int t, int nthr) {
+    for (int idx = t; idx < nrows * 16; idx += nthr) {
+        const int r = r0 + (idx >> 4), c16 = idx & 15;
+        if (r < rmax) {
+            const uint4 v = *reinterpret_cast<const uint4*>(stage + r * 256 + ((c16 ^ (r & 15)) << 4));
+            *reinterpret_cast<uint4*>(out + ((tok0 + r / G) * Hq + kh * G + (r % G)) * kD + c16 * 8) = v;
+        }
+    }
+}
 
 }  // namespace tc
 }  // namespace treekv

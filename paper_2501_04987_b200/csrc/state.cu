@@ -266,14 +266,16 @@ cudaError_t launch_chunk_evict(const CacheView& cv, treekv_dtype dt, const Prefi
 
 // ---------------------------------------------------------------------------------------------------------
 // The three steps above in one launch: score update, every eviction segment of the chunk, n_seen += m.
-// A cluster of kEvictCluster thread blocks owns one unit.  Inside a segment the pairs are taken in rounds of
+// One thread block of kEvictThreads threads owns a unit (the code is written for a cluster of kEvictCluster blocks
+// per unit; one large block keeps the kernel's footprint to a few SMs, which matters when it runs beside the next
+// attention kernel on the eviction stream, and its barriers are block barriers).  Inside a segment the pairs are taken in rounds of
 // increasing pair index; a round first reads everything it moves into registers (decision, survivor's K and V
 // rows, its S and position), the cluster synchronises, then the round writes.  That is enough because the
 // destination row i+p of pair p can only be a source row of an earlier pair ((p-i)/2 < p) - read in this round
 // or a previous one - and never of a later pair; rows moved down after a wrap follow the same rule.  A new
 // segment starts after a further cluster barrier, since its pairs read rows the previous one wrote.
-constexpr int kEvictCluster = 4;
-constexpr int kEvictThreads = 512;
+constexpr int kEvictCluster = 1;
+constexpr int kEvictThreads = 1024;
 constexpr int kEvictItemsPerWarp = 4;
 
 template <typename T>
@@ -283,6 +285,7 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
     pdl_wait();
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+    auto unit_sync = [&]() { if (kEvictCluster == 1) __syncthreads(); else cluster.sync(); };
     const int unit = blockIdx.y;
     const int b = unit / cv.Hkv;
     const int m = lens.m[b];
@@ -312,7 +315,7 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
             *Sp = *Sp + s * inv_g;  // chunk rows were zeroed by the append
         }
     }
-    cluster.sync();  // every S of the unit is final; every block has read n_seen
+    unit_sync();  // every S of the unit is final; every block has read n_seen
     if (rank == 0 && threadIdx.x == 0) cv.n_seen[unit] = N1;
 
     // ---- eviction segments (Algorithm 1's "length > c" branch repeated with the scores frozen)
@@ -354,7 +357,7 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
                 }
                 if (lane == 0) { sr[u] = Sc[src]; pr[u] = Pc[src]; }
             }
-            cluster.sync();  // everything this round moves has been read
+            unit_sync();  // everything this round moves has been read
 #pragma unroll
             for (int u = 0; u < kEvictItemsPerWarp; ++u) {
                 const int item = r0 + u * kWarps + gwarp;
@@ -367,7 +370,7 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
                 if (lane == 0) { Sc[dst] = sr[u]; Pc[dst] = pr[u]; }
             }
         }
-        if (seg + 1 < nseg) cluster.sync();  // the next segment's pairs read rows this one wrote
+        if (seg + 1 < nseg) unit_sync();  // the next segment's pairs read rows this one wrote
     }
 }
 
@@ -398,6 +401,7 @@ oneshot_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int
     pdl_wait();
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+    auto unit_sync = [&]() { if (kEvictCluster == 1) __syncthreads(); else cluster.sync(); };
     const int unit = blockIdx.y;
     const int b = unit / cv.Hkv;
     const int m = lens.m[b];
@@ -424,7 +428,7 @@ oneshot_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int
             Sc[lam] = Sc[lam] + s * inv_g;  // the append left S = 0
         }
     }
-    cluster.sync();  // every S of the unit is final, the column sums have been consumed
+    unit_sync();  // every S of the unit is final, the column sums have been consumed
     if (rank == 0 && threadIdx.x == 0) { cv.n_seen[unit] = m; cv.w0[unit] = wstart; }
 
     // ---- Algorithm 1 on blocks
@@ -466,7 +470,7 @@ oneshot_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int
                 dec[p] = evict_right;
             }
         }
-        cluster.sync();  // the segment's decisions are visible to the whole cluster
+        unit_sync();  // the segment's decisions are visible to the whole cluster
         const int items = (sg.E + sg.rebase) * bs;  // token rows to move
         for (int r0 = 0; r0 < items; r0 += kRound) {
             uint4 kr[kEvictItemsPerWarp], vr[kEvictItemsPerWarp];
@@ -485,7 +489,7 @@ oneshot_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int
                 }
                 if (lane == 0) { sr[u] = Sc[src]; pr[u] = Pc[src]; }
             }
-            cluster.sync();  // everything this round moves has been read
+            unit_sync();  // everything this round moves has been read
 #pragma unroll
             for (int u = 0; u < kEvictItemsPerWarp; ++u) {
                 const int item = r0 + u * kWarps + gwarp;
@@ -500,7 +504,7 @@ oneshot_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int
                 if (lane == 0) { Sc[dst] = sr[u]; Pc[dst] = pr[u]; }
             }
         }
-        if (seg + 1 < nseg) cluster.sync();  // the next segment's pairs read rows (and overwrite decisions) of this one
+        if (seg + 1 < nseg) unit_sync();  // the next segment's pairs read rows (and overwrite decisions) of this one
     }
 }
 
