@@ -389,6 +389,9 @@ def main():
     ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS)
     ap.add_argument("--prefill-path", type=int, default=0, help="TREEKV_OPT_PREFILL_PATH for the prefill legs; 0 = automatic")
     ap.add_argument("--prefill-key-split", type=int, default=0, help="TREEKV_OPT_PREFILL_KEY_SPLIT; 0 = automatic")
+    ap.add_argument("--fill-by-image", action="store_true",
+                    help="decode legs: fill the caches through treekv_import_state (one launch per layer) instead of "
+                         "budget + 37 decode steps; for profiling runs")
     ap.add_argument("--decode-split", type=int, default=0, help="thread blocks per (sequence, KV head); 0 = automatic")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling small cases)")
     args = ap.parse_args()
@@ -427,11 +430,12 @@ def main():
     steps, warmup = max(1, args.steps), max(3, args.warmup)
 
     # ------------------------------------------------------------------ decode legs (the first is the headline, with e2e)
-    dec = run_decode_leg(torch, binding, w, steps, warmup, not args.no_e2e, args.decode_split, dev, rep, timer, peaks)
+    dec = run_decode_leg(torch, binding, w, steps, warmup, not args.no_e2e, args.decode_split, dev, rep, timer, peaks,
+                         args.fill_by_image)
     decode_legs = []
     for name in [x for x in args.decode_legs.split(",") if x and x != w.name]:
         decode_legs.append(run_decode_leg(torch, binding, cfg(name), steps, warmup, False, args.decode_split, dev, rep, timer,
-                                          peaks))
+                                          peaks, args.fill_by_image))
 
     # ------------------------------------------------------------------ prefill legs
     prefill_legs = []
@@ -471,7 +475,35 @@ def main():
     rep.close()
 
 
-def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev, rep, timer, peaks):
+def full_cache_image(torch, kv, w, n_seen, dev, seed):
+    """A state image (layout of treekv_export_state) of full caches after n_seen > budget tokens: seeded Gaussian K / V
+    with the recipe's outlier key channels, the newest `budget` stream positions, positive score sums."""
+    units, c, d = w.batch * w.n_kv_heads, w.budget, w.head_dim
+    e = 2 if w.dtype == "bf16" else 4
+    tdtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    up = lambda x: (x + 255) // 256 * 256
+    sizes = [units * c * d * e, units * c * d * e, units * c * 4, units * c * 4, w.batch * 4, w.batch * 4]
+    offs = [0]
+    for n in sizes:
+        offs.append(offs[-1] + up(n))
+    raw = torch.zeros(offs[-1] + 256, dtype=torch.uint8, device=dev)
+    img = raw[(-raw.data_ptr()) % 256:][:offs[-1]]
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed)
+    K = torch.randn((units, c, d), device=dev, generator=g)
+    K[..., W.outlier_channels(d, w.n_outliers)] *= 8.0
+    V = torch.randn((units, c, d), device=dev, generator=g)
+    pos = torch.arange(n_seen - c, n_seen, device=dev, dtype=torch.int32).repeat(units, 1)
+    S = torch.rand((units, c), device=dev, generator=g) * (n_seen - pos).float()
+    img[offs[0]:offs[0] + sizes[0]] = K.to(tdtype).contiguous().view(torch.uint8).reshape(-1)
+    img[offs[1]:offs[1] + sizes[1]] = V.to(tdtype).contiguous().view(torch.uint8).reshape(-1)
+    img[offs[2]:offs[2] + sizes[2]] = S.contiguous().view(torch.uint8).reshape(-1)
+    img[offs[3]:offs[3] + sizes[3]] = pos.contiguous().view(torch.uint8).reshape(-1)
+    img[offs[4]:offs[4] + sizes[4]] = torch.full((w.batch,), n_seen, dtype=torch.int32, device=dev).view(torch.uint8)
+    return img
+
+
+def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev, rep, timer, peaks, fill_by_image=False):
     """Decode steps/s of one configuration with every cache full; optionally the same through the host entry points."""
     e = 2 if w.dtype == "bf16" else 4
     tdtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
@@ -506,7 +538,15 @@ def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev
                 if st != 0:
                     raise RuntimeError("treekv_decode_step: " + binding.status_string(st))
 
-    decode_steps(w.budget + 37)   # fill every cache (untimed)
+    if fill_by_image:
+        # every cache full and 37 evictions into its cycle through the state image (one launch per layer) instead of
+        # budget + 37 decode steps: for profiling runs, where every launch before the captured one costs time
+        for layer, c in enumerate(ctxs):
+            c.import_state(full_cache_image(torch, c, w, w.budget + 37, dev, wr.seed + layer), [w.budget + 37] * w.batch)
+        for b in range(w.batch):
+            assert ctxs[0].tokens_seen(b) == w.budget + 37
+    else:
+        decode_steps(w.budget + 37)   # fill every cache (untimed)
     decode_steps(warmup)          # warm-up
     launches0 = sum(c.stats()["kernel_launches"] for c in ctxs)
     t = timer.measure(lambda i: decode_steps(steps))
