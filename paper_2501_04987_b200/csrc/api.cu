@@ -340,11 +340,11 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
     if (ctx->side) {
         e = cudaEventRecord(ctx->ev_attn, s);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->side, ctx->ev_attn, 0);
-        if (e == cudaSuccess) e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, ctx->side);
+        if (e == cudaSuccess) e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, true, ctx->side);
         if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_state, ctx->side);
         ctx->side_pending = true;  // also after a failure half-way: a later call then still orders itself behind `side`
     } else {
-        e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, s);
+        e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, false, s);
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += direct ? 2 : 3;  // (append,) attention, update + eviction

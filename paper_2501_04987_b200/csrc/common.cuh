@@ -264,9 +264,10 @@ cudaError_t launch_chunk_scores(const CacheView& cv, const PrefillScratch& ps, c
 cudaError_t launch_chunk_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
                                int seg, int max_items, cudaStream_t stream);  // gather + scatter: two launches
 cudaError_t launch_chunk_finalize(const CacheView& cv, const ChunkLens& lens, cudaStream_t stream);
-// score update + every eviction segment + n_seen update of a chunk in one launch (a cluster per unit)
+// score update + every eviction segment + n_seen update of a chunk in one launch; small_footprint: one large block
+// per unit instead of a cluster of four (for running beside another kernel)
 cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
-                                      cudaStream_t stream);
+                                      bool small_footprint, cudaStream_t stream);
 
 // one-shot prefill of an empty cache: scores from the observation window, block means, Algorithm 1 on blocks
 cudaError_t launch_oneshot_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,

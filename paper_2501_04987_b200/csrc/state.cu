@@ -266,21 +266,21 @@ cudaError_t launch_chunk_evict(const CacheView& cv, treekv_dtype dt, const Prefi
 
 // ---------------------------------------------------------------------------------------------------------
 // The three steps above in one launch: score update, every eviction segment of the chunk, n_seen += m.
-// One thread block of kEvictThreads threads owns a unit (the code is written for a cluster of kEvictCluster blocks
-// per unit; one large block keeps the kernel's footprint to a few SMs, which matters when it runs beside the next
-// attention kernel on the eviction stream, and its barriers are block barriers).  Inside a segment the pairs are taken in rounds of
+// A unit is owned by a cluster of CL thread blocks: four blocks of 512 threads when the kernel runs in the caller's
+// stream, where its latency counts (the barriers are cluster barriers), or one block of 1024 threads when it runs on
+// the context's eviction stream beside the next attention kernel, where a small footprint counts (block barriers).  Inside a segment the pairs are taken in rounds of
 // increasing pair index; a round first reads everything it moves into registers (decision, survivor's K and V
 // rows, its S and position), the cluster synchronises, then the round writes.  That is enough because the
 // destination row i+p of pair p can only be a source row of an earlier pair ((p-i)/2 < p) - read in this round
 // or a previous one - and never of a later pair; rows moved down after a wrap follow the same rule.  A new
 // segment starts after a further cluster barrier, since its pairs read rows the previous one wrote.
-constexpr int kEvictCluster = 1;
-constexpr int kEvictThreads = 1024;
+constexpr int evict_threads(int cl) { return cl == 1 ? 1024 : 512; }
 constexpr int kEvictItemsPerWarp = 4;
 
-template <typename T>
-__global__ void __cluster_dims__(kEvictCluster, 1, 1) __launch_bounds__(kEvictThreads)
+template <typename T, int kEvictCluster>
+__global__ void __launch_bounds__(evict_threads(kEvictCluster))
 chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
+    constexpr int kEvictThreads = evict_threads(kEvictCluster);
     pdl_trigger();
     pdl_wait();
     namespace cg = cooperative_groups;
@@ -374,14 +374,30 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
     }
 }
 
-cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
-                                      cudaStream_t stream) {
+template <typename T, int CL>
+static cudaError_t launch_chunk_update_evict_t(const CacheView& cv, const PrefillScratch& ps, const ChunkLens& lens,
+                                               cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kEvictCluster, cv.B * cv.Hkv);
-    cfg.blockDim = dim3(kEvictThreads);
+    cfg.gridDim = dim3(CL, cv.B * cv.Hkv);
+    cfg.blockDim = dim3(evict_threads(CL));
     cfg.stream = stream;  // plain stream order behind the attention kernel; the kernel after it may be scheduled early
-    if (dt == TREEKV_F32) return cudaLaunchKernelEx(&cfg, chunk_update_evict_kernel<float>, cv, ps, lens);
-    return cudaLaunchKernelEx(&cfg, chunk_update_evict_kernel<__nv_bfloat16>, cv, ps, lens);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CL;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = CL > 1 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, chunk_update_evict_kernel<T, CL>, cv, ps, lens);
+}
+
+cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
+                                      bool small_footprint, cudaStream_t stream) {
+    if (dt == TREEKV_F32)
+        return small_footprint ? launch_chunk_update_evict_t<float, 1>(cv, ps, lens, stream)
+                               : launch_chunk_update_evict_t<float, 4>(cv, ps, lens, stream);
+    return small_footprint ? launch_chunk_update_evict_t<__nv_bfloat16, 1>(cv, ps, lens, stream)
+                           : launch_chunk_update_evict_t<__nv_bfloat16, 4>(cv, ps, lens, stream);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -395,8 +411,9 @@ cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, cons
 // layout at cycle position ((m - c) mod c).  Per segment: one warp per pair decides (decisions go to the unit's
 // column-sum scratch, free by then), cluster barrier, then the rows move in rounds as in the kernel above.
 template <typename T>
-__global__ void __cluster_dims__(kEvictCluster, 1, 1) __launch_bounds__(kEvictThreads)
+__global__ void __cluster_dims__(4, 1, 1) __launch_bounds__(evict_threads(4))
 oneshot_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int bs) {
+    constexpr int kEvictCluster = 4, kEvictThreads = evict_threads(4);
     pdl_trigger();
     pdl_wait();
     namespace cg = cooperative_groups;
@@ -511,8 +528,8 @@ oneshot_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int
 cudaError_t launch_oneshot_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
                                         int block, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kEvictCluster, cv.B * cv.Hkv);
-    cfg.blockDim = dim3(kEvictThreads);
+    cfg.gridDim = dim3(4, cv.B * cv.Hkv);
+    cfg.blockDim = dim3(evict_threads(4));
     cfg.stream = stream;
     if (dt == TREEKV_F32) return cudaLaunchKernelEx(&cfg, oneshot_update_evict_kernel<float>, cv, ps, lens, block);
     return cudaLaunchKernelEx(&cfg, oneshot_update_evict_kernel<__nv_bfloat16>, cv, ps, lens, block);
