@@ -10,7 +10,8 @@ lasts at least a second, and the median block is reported (`blocks`, `region_ms`
 GPU and the output crosses it back inside the timed region, every layer of every step (the kernel reads and writes
 the host tensors itself; h2d / d2h bytes are counted from the tensors).
 `decode_legs`: the same measurement on the other decode shapes (configuration 2; the decode phases of
-configurations 5 and 3; configuration 1, which is launch-latency-bound).
+configurations 5 and 3; configuration 1, which is launch-latency-bound), and the headline configuration once more with
+in-cache positions (Section 4.1 "Position Encoding": keys rotated by cache slot inside the kernel).
 `prefill` / `prefill_legs`: chunked-prefill tokens/s (through all layers), steady state with full chunks, on
 configurations 5 (headline prefill), 4 and 3, each with a tensor roofline entry that gives the executed (three
 contractions) and the two-contraction fractions against the sustained, burst and nominal bf16 peaks.
@@ -401,6 +402,8 @@ def main():
     ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS)
     ap.add_argument("--prefill-path", type=int, default=0, help="TREEKV_OPT_PREFILL_PATH for the prefill legs; 0 = automatic")
     ap.add_argument("--prefill-key-split", type=int, default=0, help="TREEKV_OPT_PREFILL_KEY_SPLIT; 0 = automatic")
+    ap.add_argument("--no-positions-leg", action="store_true",
+                    help="skip the decode leg that repeats the headline configuration with in-cache positions")
     ap.add_argument("--fill-by-image", action="store_true",
                     help="decode legs: fill the caches through treekv_import_state (one launch per layer) instead of "
                          "budget + 37 decode steps; for profiling runs")
@@ -448,6 +451,10 @@ def main():
     for name in [x for x in args.decode_legs.split(",") if x and x != w.name]:
         decode_legs.append(run_decode_leg(torch, binding, cfg(name), steps, warmup, False, args.decode_split, dev, rep, timer,
                                           peaks, args.fill_by_image))
+
+    if not args.no_positions_leg:
+        decode_legs.append(run_decode_leg(torch, binding, w, steps, warmup, False, args.decode_split, dev, rep, timer, peaks,
+                                          args.fill_by_image, positions=True))
 
     # ------------------------------------------------------------------ prefill legs
     prefill_legs = []
@@ -515,7 +522,8 @@ def full_cache_image(torch, kv, w, n_seen, dev, seed):
     return img
 
 
-def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev, rep, timer, peaks, fill_by_image=False):
+def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev, rep, timer, peaks, fill_by_image=False,
+                   positions=False):
     """Decode steps/s of one configuration with every cache full; optionally the same through the host entry points."""
     e = 2 if w.dtype == "bf16" else 4
     tdtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
@@ -526,6 +534,12 @@ def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev
     if decode_split:
         for c in ctxs:
             c.set_option(binding.OPT_DECODE_SPLIT, decode_split)
+    if positions:
+        # in-cache positions (Section 4.1 "Position Encoding"): one cos / sin table by cache slot shared by every layer;
+        # q and k then arrive unrotated (the same seeded values, taken as such: timing does not depend on them)
+        cos, sin = (torch.from_numpy(x).to(dev) for x in W.rope_tables(w.budget + 1, w.head_dim, w.rope_base))
+        for c in ctxs:
+            c.set_positions(cos, sin)
     ring = 4
     ins = []
     for layer in range(w.layers):
@@ -613,7 +627,7 @@ def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev
             "ms_per_step": ms_per_step, "blocks": t["blocks"], "region_ms": t["region_ms"],
             "block_ms_min_max": [t["block_ms_min"], t["block_ms_max"]], "gpu_launches": int(launches),
             "clocks": t["clocks"], "roofline": roofline, "e2e": e2e, "tokens_per_s": steps_per_s * w.batch,
-            "config": config_of(w)}
+            "config": config_of(w, in_cache_positions=bool(positions))}
 
 
 def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks, eviction_stream=True, prefill_path=0, key_split=0):

@@ -71,13 +71,13 @@ treekv_status cuda_fail(treekv_ctx* ctx, cudaError_t e) {
     return TREEKV_ERR_CUDA;
 }
 
-// With in-cache positions the keys are encoded on the fly, which only the CUDA-core kernels do.
+// With in-cache positions the keys are encoded on the fly; of the prefill kernels only the CUDA-core one does that.
 bool use_tc_prefill(const treekv_ctx* ctx) {
     return ctx->has_tma && ctx->opt_prefill_path != 1 && !ctx->cv.rope_cos;
 }
 
 bool use_mma_decode(const treekv_ctx* ctx) {
-    if (ctx->dt != TREEKV_BF16 || ctx->cv.rope_cos) return false;
+    if (ctx->dt != TREEKV_BF16) return false;
     return ctx->opt_decode_path != 1;
 }
 

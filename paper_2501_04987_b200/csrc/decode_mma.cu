@@ -74,6 +74,28 @@ __device__ inline float ex2_fast(float x) {
 // 2^(a-b) with the convention 2^(-inf - anything) = 0, so empty partials (max = -inf) never produce NaN
 __device__ inline float exp2_diff(float a, float b) { return a == -INFINITY ? 0.f : ex2_fast(a - b); }
 
+// In-cache positions (Section 4.1 "Position Encoding"): 16-byte piece c (8 channels, c < D/16) of a row and its
+// rotate-half partner piece c + D/16, encoded at `slot`, with the numeric contract of rope_apply() in common.cuh:
+// x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin) in fp32, each rounded to bf16.
+__device__ inline void rope_piece_pair(uint4& lo, uint4& hi, const float* cos_row, const float* sin_row) {
+    float a[8], b[8];
+    Elem<__nv_bfloat16>::unpack(lo, a);
+    Elem<__nv_bfloat16>::unpack(hi, b);
+    float cs[8], sn[8];
+    *reinterpret_cast<float4*>(cs) = __ldg(reinterpret_cast<const float4*>(cos_row));
+    *reinterpret_cast<float4*>(cs + 4) = __ldg(reinterpret_cast<const float4*>(cos_row) + 1);
+    *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(sin_row));
+    *reinterpret_cast<float4*>(sn + 4) = __ldg(reinterpret_cast<const float4*>(sin_row) + 1);
+    float ya[8], yb[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        ya[e] = __fmaf_rn(a[e], cs[e], -__fmul_rn(b[e], sn[e]));
+        yb[e] = __fmaf_rn(b[e], cs[e], __fmul_rn(a[e], sn[e]));
+    }
+    lo = make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]), pack_bf16(ya[4], ya[5]), pack_bf16(ya[6], ya[7]));
+    hi = make_uint4(pack_bf16(yb[0], yb[1]), pack_bf16(yb[2], yb[3]), pack_bf16(yb[4], yb[5]), pack_bf16(yb[6], yb[7]));
+}
+
 constexpr int kBlk = 16;      // keys per pipeline stage
 constexpr int kPrefetchRows = 256;  // rows of K and of V a CTA asks L2 for before its stream-order wait (0 = none)
 constexpr int kMaxSplit = 8;  // largest cluster
@@ -267,6 +289,20 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     const T* tq = reinterpret_cast<const T*>(tok);
     const T* tk = reinterpret_cast<const T*>(tok + G * ROWB);
     const T* tv = reinterpret_cast<const T*>(tok + (G + 1) * ROWB);
+    // in-cache positions: the query sits in the last slot, n - 1; its staged rows are encoded in place.  Keys stay as
+    // given in the cache and are encoded at their slot in shared memory, tile by tile, below.
+    const bool rope = cv.rope_cos != nullptr;
+    if (rope) {
+        for (int e = tid; e < G * (CPR / 2); e += NT) {
+            const int r = e / (CPR / 2), cidx = e % (CPR / 2);
+            uint4* plo = reinterpret_cast<uint4*>(tok + r * ROWB) + cidx;
+            uint4* phi = plo + CPR / 2;
+            uint4 a = *plo, bq = *phi;
+            rope_piece_pair(a, bq, cv.rope_cos + (size_t)(n - 1) * (D / 2) + cidx * 8, cv.rope_sin + (size_t)(n - 1) * (D / 2) + cidx * 8);
+            *plo = a; *phi = bq;
+        }
+        __syncthreads();
+    }
 
     // ---- append (Algorithm 1: K <- K u {k}, V <- V u {v}); the step itself uses the staged copy of the new token
     if (warp == NW - 1) {
@@ -290,10 +326,26 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
 #pragma unroll
         for (int h = 0; h < G; ++h) sn[h] = -INFINITY;
         if (owns_new) {
+            // this lane's channels of the new key (lane, lane + 32, ...): with in-cache positions encoded at slot n - 1,
+            // channel e < D/2 pairing with e + D/2, which the same lane holds
+            float kn[D / 32];
+#pragma unroll
+            for (int u = 0; u < D / 32; ++u) kn[u] = __bfloat162float(tk[lane + 32 * u]);
+            if (rope) {
+#pragma unroll
+                for (int u = 0; u < D / 64; ++u) {
+                    const int e = lane + 32 * u;  // < D/2
+                    const float cs = __ldg(cv.rope_cos + (size_t)(n - 1) * (D / 2) + e), sv = __ldg(cv.rope_sin + (size_t)(n - 1) * (D / 2) + e);
+                    const float x1 = kn[u], x2 = kn[u + D / 64];
+                    kn[u] = __bfloat162float(__float2bfloat16_rn(__fmaf_rn(x1, cs, -__fmul_rn(x2, sv))));
+                    kn[u + D / 64] = __bfloat162float(__float2bfloat16_rn(__fmaf_rn(x2, cs, __fmul_rn(x1, sv))));
+                }
+            }
 #pragma unroll
             for (int h = 0; h < G; ++h) {
                 float a = 0.f;
-                for (int e = lane; e < D; e += 32) a += __bfloat162float(tq[h * D + e]) * __bfloat162float(tk[e]);
+#pragma unroll
+                for (int u = 0; u < D / 32; ++u) a += __bfloat162float(tq[h * D + lane + 32 * u]) * kn[u];
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
                 sn[h] = a * scale;
@@ -348,6 +400,22 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
         cp_async_wait<NS - 1>();
         __syncwarp();
         const uint32_t kst = ring_w + stage * STAGE, vst = kst + kBlk * ROWB;
+        if (rope) {
+            // encode the tile's keys at their cache slots, in place: row r of the tile is slot lo + 16 blk + r; a lane
+            // takes piece pairs (c, c + CPR/2) of rows, eight lanes per row (conflict-free 16-byte accesses)
+            unsigned char* kt = ring + (size_t)(warp * NS + stage) * STAGE;
+#pragma unroll
+            for (int i2 = 0; i2 < kBlk * (CPR / 2) / 32; ++i2) {
+                const int item = lane + 32 * i2, r = item / (CPR / 2), cidx = item % (CPR / 2);
+                const int slot = min(lo + blk * kBlk + r, n - 1);
+                uint4* plo = reinterpret_cast<uint4*>(kt + r * ROWB + ((cidx ^ (r & 7)) << 4));
+                uint4* phi = reinterpret_cast<uint4*>(kt + r * ROWB + (((cidx + CPR / 2) ^ (r & 7)) << 4));
+                uint4 a = *plo, bq = *phi;
+                rope_piece_pair(a, bq, cv.rope_cos + (size_t)slot * (D / 2) + cidx * 8, cv.rope_sin + (size_t)slot * (D / 2) + cidx * 8);
+                *plo = a; *phi = bq;
+            }
+            __syncwarp();
+        }
 
         // ---- logits of 16 keys x G heads
         float c[2][4];
