@@ -287,8 +287,9 @@ treekv_status treekv_set_protection(treekv_ctx* ctx, int n_sink, int n_recent);
  *                     every later call; slots >= budget + max(1, max_chunk).  Both NULL: back to position-agnostic.
  * Numeric contract: x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin) in fp32, rounded to the context's dtype
  * before the dot product (the paper's runs are bf16 throughout; an fp32 context does not round).
- * Only on a context that has not seen a token (TREEKV_ERR_BAD_STATE otherwise).  Attention then runs on the CUDA-core
- * kernels, which encode while they stream.  Host-side only, nothing is enqueued.
+ * Only on a context that has not seen a token (TREEKV_ERR_BAD_STATE otherwise).  Decode steps of a bf16
+ * context keep their fast kernel, which encodes each key tile in shared memory on its way to the tensor cores; prefill
+ * chunks and fp32 contexts run on the CUDA-core kernels, which encode while they stream.  Host-side only, nothing is enqueued.
  */
 treekv_status treekv_set_positions(treekv_ctx* ctx, const float* dev_cos, const float* dev_sin, int slots);
 
