@@ -249,7 +249,7 @@ treekv_status treekv_import_state(treekv_ctx* ctx, const void* dev_image, const 
 /* Counters and error words.  Synchronises `stream` to read the device-side counters.  *host_out is filled
  * whenever the read itself succeeded; the return value is TREEKV_ERR_TIMEOUT when device_error is non-zero, i.e.
  * when a kernel's bounded wait gave up (bits: 4 TMA producer, 8 MMA issuer, 16 softmax / epilogue warps of the
- * tensor-core prefill kernels, 32 misaligned shared memory, 64 the self-test below).  treekv_reset clears it. */
+ * tensor-core prefill kernels, 32 misaligned shared memory, 64 the self-test below, 128 the decode kernel's fetch of the step's q, k, v).  treekv_reset clears it. */
 treekv_status treekv_get_stats(treekv_ctx* ctx, treekv_stats* host_out, void* stream);
 
 /*

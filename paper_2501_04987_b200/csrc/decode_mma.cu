@@ -17,6 +17,7 @@
 #include <cooperative_groups.h>
 
 #include "common.cuh"
+#include "tma.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -154,14 +155,23 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     //      are fetched once, early, whether they live in HBM or in page-locked host memory.  When the caller
     //      guarantees that the inputs held their final values before the launch (host tensors filled by the CPU),
     //      the fetch starts before the stream-order wait and its latency hides behind the previous kernel's tail.
-    auto stage_inputs = [&]() {
-        const T* qrow = q + ((size_t)b * cv.Hq + kh * G) * D;
-        for (int e = lane; e < (G + 2) * CPR; e += 32) {
-            const int r = e / CPR, cidx = e % CPR;
-            const T* srow = r < G ? qrow + (size_t)r * D : (r == G ? k_new : v_new);
-            cp_async_16(smem_u32(tok + r * ROWB + cidx * 16), reinterpret_cast<const unsigned char*>(srow) + cidx * 16, true);
+    // They come as three bulk copies (the group's q rows are contiguous; one row each of k and v) that signal an
+    // mbarrier: across the bus a bulk copy travels as a few large read requests instead of one per 16-byte piece.
+    __shared__ __align__(8) uint64_t in_bar;
+    if (tid == 0) { mbar_init(smem_addr_u32(&in_bar), 1); mbar_fence_init(); }
+    __syncwarp();
+    auto stage_inputs = [&]() {  // warp 0
+        if (lane == 0) {
+            const T* qrow = q + ((size_t)b * cv.Hq + kh * G) * D;
+            const uint32_t bar = smem_addr_u32(&in_bar);
+            mbar_arrive_expect_tx(bar, (G + 2) * ROWB);
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_u32(tok)), "l"(qrow), "r"(G * ROWB), "r"(bar) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_u32(tok + G * ROWB)), "l"(k_new), "r"(ROWB), "r"(bar) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_u32(tok + (G + 1) * ROWB)), "l"(v_new), "r"(ROWB), "r"(bar) : "memory");
         }
-        cp_async_commit();
     };
     if (inputs_final && warp == 0 && active.test(b)) stage_inputs();
     // While the previous kernel of the stream drains, ask L2 for the first rows this CTA will stream.  This is a hint
@@ -284,7 +294,8 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
 #pragma unroll
     for (int s = 0; s < NS; ++s) issue(warp + s * NW, s);
 
-    if (warp == 0) cp_async_wait<NS>();  // the staged inputs have landed (the NS tile groups may still be in flight)
+    // the staged inputs have landed (bounded wait; a give-up is recorded and the step's result is then meaningless)
+    if (warp == 0 && !mbar_wait(smem_addr_u32(&in_bar), 0) && lane == 0) atomicOr(&cv.stats->error, 128u);
     __syncthreads();
     const T* tq = reinterpret_cast<const T*>(tok);
     const T* tk = reinterpret_cast<const T*>(tok + G * ROWB);
