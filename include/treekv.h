@@ -75,9 +75,11 @@ typedef enum {
                                     from dev_k / dev_v and append them to the cache themselves whenever every sequence's
                                     chunk length is a multiple of 128 (no separate append kernel); 1 = always append with
                                     a kernel of its own before the attention.  Same result either way. */
-    TREEKV_OPT_PREFILL_KEY_SPLIT = 5, /* thread blocks that share the 256 query rows of a tile pair in the two-tile tensor-core
-                                    prefill kernel, each taking a share of the key tiles: 0 (default) and 1 = one block, 2 = a pair of blocks
-                                    that halve the key tiles and exchange row statistics and partial outputs */
+    TREEKV_OPT_PREFILL_KEY_SPLIT = 5, /* two-tile tensor-core prefill kernel: which tile pairs (256 query rows) are given to a pair
+                                    of thread blocks that halve the pair's key tiles and exchange row statistics and
+                                    partial outputs.  0 = automatic:
+                                    the pairs of a last, at most half-full wave; 1 = none; 2 = every pair; 3 = the
+                                    automatic rule for a machine of four SMs (for tests) */
     TREEKV_OPT_EVICTION_STREAM = 4 /* 0 (default) = every kernel of a call runs on the caller's stream.  1 = the last
                                     kernel of treekv_prefill_chunk (score update + eviction + compaction, which only
                                     touches the workspace) runs on a stream the context owns, behind the chunk's

@@ -270,13 +270,27 @@ treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, 
         const uint32_t box[3] = {64u, (uint32_t)ctx->G, (uint32_t)(128 / ctx->G)};
         if (!make_tensor_map_bf16(&tmQ, dev_q, 3, dims, strides, box)) return TREEKV_ERR_CUDA;
         // Which kernel: two query tiles per CTA (every K / V tile load feeds twice the tensor work) once the one-tile grid
-        // would cover the machine at least twice, one tile per CTA for smaller calls.  Splitting a tile pair's key tiles
-        // over two CTAs is on request only: measured, what the pair exchanges and sets up twice costs more than the
-        // fuller last wave gives back.
+        // would cover the machine at least twice, one tile per CTA for smaller calls.
         const long tiles = (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + kQTileRows - 1) / kQTileRows);
         const bool two = ctx->opt_prefill_path == 3 || (ctx->opt_prefill_path == 0 && tiles >= 2L * ctx->sm_count);
-        const int ks = ctx->opt_prefill_key_split == 2 ? 2 : 1;
-        e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, ks, s)
+        // Key split of the two-tile kernel.  A grid that is not a whole number of waves ends with a wave of few CTAs; when
+        // those last tile pairs are at most half a wave, each of them goes to a cluster of two CTAs that halve its key
+        // tiles, so the last wave is full and about half as long (the CTAs of the full waves are launched as clusters
+        // too, one whole tile pair each, exchanging nothing).  Splitting every pair costs more in exchanges than it
+        // gains, and is on request only.  Option value 3 applies the same rule for a machine of four SMs (small test grids).
+        int n_whole = -1;
+        if (two) {
+            const long pairs = (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + 2 * kQTileRows - 1) / (2 * kQTileRows));
+            const int opt = ctx->opt_prefill_key_split;
+            if (opt == 2) {
+                n_whole = 0;
+            } else if (opt == 0 || opt == 3) {
+                const long sms = opt == 3 ? 4 : (ctx->sm_count & ~1);
+                const long rem = pairs % sms;
+                if (rem > 0 && 2 * rem <= sms && pairs > rem) n_whole = (int)((pairs - rem) / 2);
+            }
+        }
+        e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, n_whole, s)
                 : launch_prefill_tc(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, s);
     } else {
         e = launch_prefill_simt(ctx->cv, ctx->dt, ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
@@ -610,7 +624,7 @@ treekv_status treekv_set_option(treekv_ctx* ctx, treekv_option opt, int value) {
             return TREEKV_OK;
         }
         case TREEKV_OPT_PREFILL_KEY_SPLIT:
-            if (!(value == 0 || value == 1 || value == 2)) return TREEKV_ERR_INVALID_ARG;
+            if (value < 0 || value > 3) return TREEKV_ERR_INVALID_ARG;
             ctx->opt_prefill_key_split = value;
             return TREEKV_OK;
         case TREEKV_OPT_PREFILL_APPEND:

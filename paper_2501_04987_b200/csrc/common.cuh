@@ -288,8 +288,9 @@ struct ChunkTensors {
 size_t prefill_tc2_smem_bytes();
 cudaError_t launch_prefill_tc2(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                                const CUtensorMap& tmV, const ChunkTensors& ct, void* out, const ChunkLens& lens,
-                               int chunk_stride, int max_m, int key_split, cudaStream_t stream);  // 256 query rows per CTA;
-                               // key_split 2: pairs of CTAs that share the query rows and halve the key tiles
+                               int chunk_stride, int max_m, int n_whole_clusters, cudaStream_t stream);
+// 256 query rows per CTA.  n_whole_clusters < 0: one CTA per tile pair; else two-CTA clusters, the first n_whole_clusters
+// with one tile pair per CTA, the others splitting a pair's key tiles
 
 size_t prefill_tc_smem_bytes();
 cudaError_t launch_prefill_tc(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,

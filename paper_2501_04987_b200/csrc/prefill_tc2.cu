@@ -14,6 +14,7 @@
 // buffers of 128 columns); pass B holds S_s^T in buffers 0, 1 and O_s^T in buffers 2, 3.  Shared memory: two Q
 // tiles, a ring of three K / V tiles, one P^T tile per sub-tile.  All waits are bounded mbarrier waits; a wait
 // that gives up sets an error word and the CTA drains to its exit, where tensor memory is released.
+#include <algorithm>
 #include <type_traits>
 
 #include "prefill_tc_common.cuh"
@@ -36,14 +37,29 @@ __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKin,
                    const __grid_constant__ CUtensorMap tmVin, ChunkDirect cd, CacheView cv, PrefillScratch ps,
-                   __nv_bfloat16* __restrict__ out, ChunkLens lens, int chunk_stride) {
+                   __nv_bfloat16* __restrict__ out, ChunkLens lens, int chunk_stride, int pairs_per_unit,
+                   int n_whole_clusters) {
     constexpr int TOK = 128 / G;  // tokens per sub-tile
-    const int unit = blockIdx.y, qt2 = blockIdx.x / KS;
-    const int ks = KS > 1 ? (int)(blockIdx.x % KS) : 0;  // rank in the key-split cluster (cluster = KS consecutive blockIdx.x)
+    // KS == 1: grid (tile pairs, units).  KS == 2: a 1-D grid of two-CTA clusters over the call's items (unit, tile
+    // pair) in order: the CTAs of the first n_whole_clusters clusters take one whole item each (they exchange nothing
+    // and never synchronise with each other), every later cluster splits one item's key tiles between its CTAs - the
+    // items of a last, partial wave, which then fills the machine and is about half as long.
+    int unit, qt2, ks = 0;
+    bool split = false;
+    if constexpr (KS == 1) {
+        unit = blockIdx.y; qt2 = blockIdx.x;
+    } else {
+        const int cid = (int)(blockIdx.x >> 1), rk = (int)(blockIdx.x & 1);
+        split = cid >= n_whole_clusters;
+        const int item = split ? 2 * n_whole_clusters + (cid - n_whole_clusters) : 2 * cid + rk;
+        unit = item / pairs_per_unit; qt2 = item % pairs_per_unit;
+        ks = split ? rk : 0;
+        if (unit >= cv.B * cv.Hkv) return;  // the odd CTA of the last whole-item cluster
+    }
     const int b = unit / cv.Hkv, kh = unit % cv.Hkv;
     const int m = lens.m[b];
     const int t0c = qt2 * 2 * TOK;  // first token of the CTA
-    if (t0c >= m) return;
+    if (t0c >= m) return;  // uniform over a splitting cluster
     const int t1c = min(t0c + 2 * TOK, m);
     const int N = cv.n_seen[unit];
     const UnitState st = unit_state(N, cv);
@@ -51,8 +67,8 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int NT = kt.NT;
     const int n = st.L + m;
     // this CTA's key tiles [jb, jb + nt): all of them, or its half (rank 0 the first, larger one: never empty)
-    const int jb = (KS > 1 && ks == 1) ? (NT + 1) / 2 : 0;
-    const int nt = KS > 1 ? (ks == 0 ? (NT + 1) / 2 : NT - (NT + 1) / 2) : NT;
+    const int jb = (split && ks == 1) ? (NT + 1) / 2 : 0;
+    const int nt = split ? (ks == 0 ? (NT + 1) / 2 : NT - (NT + 1) / 2) : NT;
 
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const uint32_t base = smem_addr_u32(smem_raw);
@@ -83,7 +99,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     // both CTAs of a pair are running and their barriers are initialised before either signals the other
-    if constexpr (KS > 1) cluster_sync_all();
+    if (KS > 1 && split) cluster_sync_all();
 
     bool ok = true;
     if (warp == 0) {
@@ -294,7 +310,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             float M = fmaxf(m0, m1);
             float l = (m0 == -INFINITY ? 0.f : part_l[(sub * 2) * 128 + row] * ex2(m0 - M)) +
                       (m1 == -INFINITY ? 0.f : part_l[(sub * 2 + 1) * 128 + row] * ex2(m1 - M));
-            if constexpr (KS > 1) {
+            if (KS > 1 && split) {
                 // the other half of the keys: hand over this half's (max, sum), take the other's, combine - rank 0's
                 // term first on both sides, so the two CTAs normalise with the same log-sum-exp bit for bit
                 float* xstat = part_m + 1024;  // [2][128] x (max, sum), written by the other CTA
@@ -410,7 +426,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         // ---- epilogue: O_s^T (lane = channel, column = query row) -> out[token][head][channel]
         if (ok && mbar_wait(bar(O_FULL), 0)) {
             tc_fence_after();
-            if constexpr (KS == 1) {
+            if (KS == 1 || !split) {
                 // 64 query columns per warp, staged through the sub-tile's idle P^T buffer so that whole rows are
                 // written; the four warps (lane quarters) of a column half synchronise on a barrier of their own
                 unsigned char* stage = p_area + sub * kSlot;
@@ -473,8 +489,8 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
     }
     __syncthreads();
-    // neither CTA of a pair exits while the other may still write into its shared memory or signal its barriers
-    if constexpr (KS > 1) cluster_sync_all();
+    // neither CTA of a splitting pair exits while the other may still write into its shared memory or signal its barriers
+    if (KS > 1 && split) cluster_sync_all();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
@@ -483,7 +499,8 @@ size_t prefill_tc2_smem_bytes() { return (size_t)(4 + kRing) * kSlot + 512 * siz
 template <int G, int KS>
 static cudaError_t launch_prefill_tc2_t(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ,
                                         const CUtensorMap& tmK, const CUtensorMap& tmV, const ChunkTensors& ct, void* out,
-                                        const ChunkLens& lens, int chunk_stride, int max_m, cudaStream_t stream) {
+                                        const ChunkLens& lens, int chunk_stride, int max_m, int n_whole_clusters,
+                                        cudaStream_t stream) {
     auto kern = prefill_tc2_kernel<G, KS>;
     const size_t smem = prefill_tc2_smem_bytes();
     static bool smem_set[64] = {};  // per device: the opt-in is needed once
@@ -496,8 +513,15 @@ static cudaError_t launch_prefill_tc2_t(const CacheView& cv, const PrefillScratc
         smem_set[dev] = true;
     }
     const ChunkDirect cd = {reinterpret_cast<const __nv_bfloat16*>(ct.k), reinterpret_cast<const __nv_bfloat16*>(ct.v)};
+    const int pairs = (max_m * G + 2 * kQTileRows - 1) / (2 * kQTileRows), units = cv.B * cv.Hkv;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(KS * ((max_m * G + 2 * kQTileRows - 1) / (2 * kQTileRows)), cv.B * cv.Hkv);
+    if (KS == 1) {
+        cfg.gridDim = dim3(pairs, units);
+    } else {  // whole-item clusters first (two items each, the last one possibly with an idle CTA), then one cluster per split item
+        const long items = (long)pairs * units;
+        const long whole_items = std::min<long>(2L * n_whole_clusters, items);
+        cfg.gridDim = dim3((unsigned)(2 * (n_whole_clusters + (items - whole_items))));
+    }
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
@@ -509,17 +533,20 @@ static cudaError_t launch_prefill_tc2_t(const CacheView& cv, const PrefillScratc
     cfg.attrs = attr;
     cfg.numAttrs = KS > 1 ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kern, tmQ, tmK, tmV, ct.k ? ct.tmK : tmK, ct.k ? ct.tmV : tmV, cd, cv, ps,
-                              reinterpret_cast<__nv_bfloat16*>(out), lens, chunk_stride);
+                              reinterpret_cast<__nv_bfloat16*>(out), lens, chunk_stride, pairs, n_whole_clusters);
 }
 
+// n_whole_clusters < 0: one CTA per tile pair.  Otherwise clusters of two CTAs: the first n_whole_clusters take two tile
+// pairs each (one per CTA), every remaining tile pair gets a cluster that splits its key tiles.
 cudaError_t launch_prefill_tc2(const CacheView& cv, const PrefillScratch& ps, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                                const CUtensorMap& tmV, const ChunkTensors& ct, void* out, const ChunkLens& lens,
-                               int chunk_stride, int max_m, int key_split, cudaStream_t stream) {
-    if (cv.d != kD || (key_split != 1 && key_split != 2)) return cudaErrorInvalidValue;
-#define TREEKV_TC2_CASE(g)                                                                                           \
-    case g:                                                                                                          \
-        return key_split == 2 ? launch_prefill_tc2_t<g, 2>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream) \
-                              : launch_prefill_tc2_t<g, 1>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, stream);
+                               int chunk_stride, int max_m, int n_whole_clusters, cudaStream_t stream) {
+    if (cv.d != kD) return cudaErrorInvalidValue;
+#define TREEKV_TC2_CASE(g)                                                                                                    \
+    case g:                                                                                                                   \
+        return n_whole_clusters >= 0                                                                                          \
+                   ? launch_prefill_tc2_t<g, 2>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, n_whole_clusters, stream) \
+                   : launch_prefill_tc2_t<g, 1>(cv, ps, tmQ, tmK, tmV, ct, out, lens, chunk_stride, max_m, 0, stream);
     switch (cv.Hq / cv.Hkv) {
         TREEKV_TC2_CASE(1)
         TREEKV_TC2_CASE(2)

@@ -127,6 +127,27 @@ def test_two_tile_tensor_core_prefill_kernel(gpu, g, lens, chunk, budget, key_sp
     print("two-tile prefill g=%d" % g, rep)
 
 
+@pytest.mark.parametrize("g,batch,hkv,budget,chunk,lens", [
+    (1, 3, 1, 512, 384, [4 * 384 + 100, 2 * 384, 3 * 384 + 300]),   # 6 tile pairs: 4 in whole clusters, 2 split; ragged ends
+    (4, 1, 1, 256, 320, [5 * 320 + 64]),                             # 5 tile pairs: 4 whole, 1 split; chunks wrap the cycle
+    (2, 1, 3, 300, 256, [6 * 256 + 31]),                             # 6 pairs over 3 units
+])
+def test_two_tile_kernel_with_the_last_wave_split(gpu, g, batch, hkv, budget, chunk, lens):
+    """The two-tile prefill kernel gives the tile pairs of a last, at most half-full wave to clusters of two thread blocks
+    that halve the key tiles; the pairs of the full waves run in clusters too, one whole pair per block, exchanging
+    nothing.  Option value 3 applies that rule for a machine of four SMs, so that small grids mix both kinds of cluster in
+    one launch (here also with sequences that end early, i.e. blocks with nothing to do beside a busy partner)."""
+    w = W.parity_slice(W.CONFIGS["cfg5"], layers=1, batch=batch, n_heads=g * hkv, n_kv_heads=hkv, budget=budget, chunk=chunk)
+    kv, orc = _pair(gpu, w)
+    kv.set_option(gpu.OPT_PREFILL_PATH, 3)
+    kv.set_option(gpu.OPT_PREFILL_KEY_SPLIT, 3)
+    rep = Report()
+    _run_prefill(kv, orc, w, rep, lens, chunk)
+    assert [kv.tokens_seen(b) for b in range(batch)] == lens
+    _run_decode(kv, orc, w, 0, 6, rep, starts=lens)
+    assert kv.stats()["device_error"] == 0
+
+
 @pytest.mark.parametrize("path", [2, 3])
 @pytest.mark.parametrize("append", [0, 1])
 @pytest.mark.parametrize("g,budget,chunk,lens", [
