@@ -17,7 +17,7 @@ constexpr size_t kSmemLimit = 227 * 1024;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, S, pos, n_seen, w0, stats, colsum, st_q, st_k, st_v, st_out, total;
+    size_t K, V, Krot, S, pos, n_seen, w0, stats, colsum, st_q, st_k, st_v, st_out, total;
     int R, QT, n_max;
 };
 
@@ -49,6 +49,8 @@ Layout make_layout(int budget, int n_heads, int n_kv_heads, int head_dim, treekv
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
     L.K = take(units * L.R * head_dim * e);
     L.V = take(units * L.R * head_dim * e);
+    // keys encoded at their cache slots, rebuilt per call for the tensor-core prefill when in-cache positions are on
+    L.Krot = (dt == TREEKV_BF16 && head_dim == 128 && max_chunk > 0) ? take(units * L.R * head_dim * e) : 0;
     L.S = take(units * L.R * 4);
     L.pos = take(units * L.R * 4);
     L.n_seen = take(units * 4);
@@ -71,10 +73,8 @@ treekv_status cuda_fail(treekv_ctx* ctx, cudaError_t e) {
     return TREEKV_ERR_CUDA;
 }
 
-// With in-cache positions the keys are encoded on the fly; of the prefill kernels only the CUDA-core one does that.
-bool use_tc_prefill(const treekv_ctx* ctx) {
-    return ctx->has_tma && ctx->opt_prefill_path != 1 && !ctx->cv.rope_cos;
-}
+// (With in-cache positions the tensor-core kernels run on keys and queries encoded by a kernel of their own first.)
+bool use_tc_prefill(const treekv_ctx* ctx) { return ctx->has_tma && ctx->opt_prefill_path != 1; }
 
 bool use_mma_decode(const treekv_ctx* ctx) {
     if (ctx->dt != TREEKV_BF16) return false;
@@ -169,8 +169,10 @@ treekv_status treekv_create(treekv_ctx** out, int budget, int n_heads, int n_kv_
         const uint64_t dims[2] = {(uint64_t)head_dim, rows};
         const uint64_t strides[1] = {(uint64_t)head_dim * 2};
         const uint32_t box[2] = {64u, 128u};
+        ctx->k_rot = base + L.Krot;
         ctx->has_tma = make_tensor_map_bf16(&ctx->tmK, ctx->cv.K, 2, dims, strides, box) &&
-                       make_tensor_map_bf16(&ctx->tmV, ctx->cv.V, 2, dims, strides, box);
+                       make_tensor_map_bf16(&ctx->tmV, ctx->cv.V, 2, dims, strides, box) &&
+                       make_tensor_map_bf16(&ctx->tmKrot, ctx->k_rot, 2, dims, strides, box);
     }
     // The workspace starts as zeros: the tensor-core prefill reads whole 128-row tiles, and rows that hold no token
     // yet must be finite (they are multiplied by a probability of exactly zero).
@@ -252,6 +254,16 @@ treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, 
                                      int max_m, cudaStream_t s) {
     cudaError_t e;
     if (use_tc_prefill(ctx)) {
+        const CUtensorMap* tmKeys = &ctx->tmK;
+        if (ctx->cv.rope_cos) {
+            // in-cache positions: every live key encoded at its slot into the rotated slab, the chunk's queries at their
+            // own slots into the staging buffer (in place when the caller's q already is that buffer)
+            e = launch_rope_chunk(ctx->cv, lens, chunk_stride, max_m, ctx->k_rot, dev_q, ctx->st_q, s);
+            if (e != cudaSuccess) return cuda_fail(ctx, e);
+            ctx->launches += 1;
+            dev_q = ctx->st_q;
+            tmKeys = &ctx->tmKrot;
+        }
         ChunkTensors ct;
         ct.k = nullptr; ct.v = nullptr;
         if (direct) {
@@ -290,8 +302,8 @@ treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, 
                 if (rem > 0 && 2 * rem <= sms && pairs > rem) n_whole = (int)((pairs - rem) / 2);
             }
         }
-        e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, n_whole, s)
-                : launch_prefill_tc(ctx->cv, ps, tmQ, ctx->tmK, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, s);
+        e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, *tmKeys, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, n_whole, s)
+                : launch_prefill_tc(ctx->cv, ps, tmQ, *tmKeys, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, s);
     } else {
         e = launch_prefill_simt(ctx->cv, ctx->dt, ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
     }
@@ -303,7 +315,7 @@ treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, 
 // padding and may hold anything, which a value tile must not) and the cached tokens already cover the protected
 // initial tokens (so that the chunk's rows lie behind both cached segments).
 bool chunk_direct_ok(const treekv_ctx* ctx, const ChunkLens& lens) {
-    if (!use_tc_prefill(ctx) || ctx->opt_prefill_append == 1) return false;
+    if (!use_tc_prefill(ctx) || ctx->opt_prefill_append == 1 || ctx->cv.rope_cos) return false;
     for (int b = 0; b < ctx->cv.B; ++b) {
         if (lens.m[b] == 0) continue;
         if (lens.m[b] % 128 || ctx->n_seen[b] < ctx->cv.ns) return false;
@@ -326,6 +338,8 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
     if (!aligned16(dev_q) || !aligned16(dev_k) || !aligned16(dev_v) || !aligned16(dev_out)) return TREEKV_ERR_INVALID_ARG;
     if (ctx->max_chunk == 0) return TREEKV_ERR_BAD_STATE;  // decode-only context
     if (chunk_stride < 1) return TREEKV_ERR_INVALID_ARG;
+    // with in-cache positions the tensor-core path keeps the encoded queries in a staging buffer sized for max_chunk
+    if (ctx->cv.rope_cos && use_tc_prefill(ctx) && chunk_stride > ctx->max_chunk) return TREEKV_ERR_UNSUPPORTED;
     ChunkLens lens;
     memset(&lens, 0, sizeof(lens));
     int max_m = 0;
@@ -378,6 +392,7 @@ treekv_status treekv_prefill_oneshot(treekv_ctx* ctx, const void* dev_q, const v
     if (!aligned16(dev_q) || !aligned16(dev_k) || !aligned16(dev_v) || !aligned16(dev_out)) return TREEKV_ERR_INVALID_ARG;
     if (ctx->max_chunk == 0) return TREEKV_ERR_BAD_STATE;  // decode-only context
     if (stride < 1 || block < 1 || ctx->cv.c % block) return TREEKV_ERR_INVALID_ARG;
+    if (ctx->cv.rope_cos && use_tc_prefill(ctx) && stride > ctx->max_chunk) return TREEKV_ERR_UNSUPPORTED;
     if (ctx->cv.ns || ctx->cv.nr) return TREEKV_ERR_UNSUPPORTED;  // block-level eviction with protected tokens is not defined
     ChunkLens lens;
     memset(&lens, 0, sizeof(lens));

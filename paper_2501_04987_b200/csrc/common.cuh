@@ -186,6 +186,34 @@ __device__ inline void rope_apply(float (&f)[Elem<T>::kVec], int slot, int sub, 
 }
 #endif
 
+#ifdef __CUDACC__
+__device__ inline uint32_t rope_pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// In-cache positions (Section 4.1 "Position Encoding"): 16-byte piece c (8 channels, c < D/16) of a row and its
+// rotate-half partner piece c + D/16, encoded at `slot`, with the numeric contract of rope_apply() in common.cuh:
+// x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin) in fp32, each rounded to bf16.
+__device__ inline void rope_piece_pair(uint4& lo, uint4& hi, const float* cos_row, const float* sin_row) {
+    float a[8], b[8];
+    Elem<__nv_bfloat16>::unpack(lo, a);
+    Elem<__nv_bfloat16>::unpack(hi, b);
+    float cs[8], sn[8];
+    *reinterpret_cast<float4*>(cs) = __ldg(reinterpret_cast<const float4*>(cos_row));
+    *reinterpret_cast<float4*>(cs + 4) = __ldg(reinterpret_cast<const float4*>(cos_row) + 1);
+    *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(sin_row));
+    *reinterpret_cast<float4*>(sn + 4) = __ldg(reinterpret_cast<const float4*>(sin_row) + 1);
+    float ya[8], yb[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        ya[e] = __fmaf_rn(a[e], cs[e], -__fmul_rn(b[e], sn[e]));
+        yb[e] = __fmaf_rn(b[e], cs[e], __fmul_rn(a[e], sn[e]));
+    }
+    lo = make_uint4(rope_pack_bf16(ya[0], ya[1]), rope_pack_bf16(ya[2], ya[3]), rope_pack_bf16(ya[4], ya[5]), rope_pack_bf16(ya[6], ya[7]));
+    hi = make_uint4(rope_pack_bf16(yb[0], yb[1]), rope_pack_bf16(yb[2], yb[3]), rope_pack_bf16(yb[4], yb[5]), rope_pack_bf16(yb[6], yb[7]));
+}
+#endif
+
 // chunk length of every sequence in a prefill call (0 = not in the call), passed by value
 struct ChunkLens {
     uint16_t m[kMaxBatch];
@@ -268,6 +296,12 @@ cudaError_t launch_chunk_finalize(const CacheView& cv, const ChunkLens& lens, cu
 // per unit instead of a cluster of four (for running beside another kernel)
 cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
                                       bool small_footprint, cudaStream_t stream);
+
+// In-cache positions for the tensor-core prefill: the unit's live rows (cache and appended chunk) encoded at their slots
+// into the rotated-key slab k_rot (same geometry as the K slab), and the chunk's queries, encoded at their own slots,
+// into q_rot (may be q itself)
+cudaError_t launch_rope_chunk(const CacheView& cv, const ChunkLens& lens, int chunk_stride, int max_m, void* k_rot,
+                              const void* q, void* q_rot, cudaStream_t stream);
 
 // one-shot prefill of an empty cache: scores from the observation window, block means, Algorithm 1 on blocks
 cudaError_t launch_oneshot_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,

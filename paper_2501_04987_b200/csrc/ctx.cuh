@@ -7,6 +7,8 @@ struct treekv_ctx {
     treekv::CacheView cv;
     treekv::PrefillScratch ps;
     CUtensorMap tmK, tmV;  // 2-D maps over the K and V slabs (rows x head_dim), box 128 rows x 64 channels (bf16, d=128)
+    CUtensorMap tmKrot;    // the same over k_rot, the slab of keys encoded at their cache slots (in-cache positions)
+    void* k_rot;
     bool has_tma;
     treekv_dtype dt;
     int max_chunk;

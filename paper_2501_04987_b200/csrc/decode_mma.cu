@@ -75,28 +75,6 @@ __device__ inline float ex2_fast(float x) {
 // 2^(a-b) with the convention 2^(-inf - anything) = 0, so empty partials (max = -inf) never produce NaN
 __device__ inline float exp2_diff(float a, float b) { return a == -INFINITY ? 0.f : ex2_fast(a - b); }
 
-// In-cache positions (Section 4.1 "Position Encoding"): 16-byte piece c (8 channels, c < D/16) of a row and its
-// rotate-half partner piece c + D/16, encoded at `slot`, with the numeric contract of rope_apply() in common.cuh:
-// x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin) in fp32, each rounded to bf16.
-__device__ inline void rope_piece_pair(uint4& lo, uint4& hi, const float* cos_row, const float* sin_row) {
-    float a[8], b[8];
-    Elem<__nv_bfloat16>::unpack(lo, a);
-    Elem<__nv_bfloat16>::unpack(hi, b);
-    float cs[8], sn[8];
-    *reinterpret_cast<float4*>(cs) = __ldg(reinterpret_cast<const float4*>(cos_row));
-    *reinterpret_cast<float4*>(cs + 4) = __ldg(reinterpret_cast<const float4*>(cos_row) + 1);
-    *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(sin_row));
-    *reinterpret_cast<float4*>(sn + 4) = __ldg(reinterpret_cast<const float4*>(sin_row) + 1);
-    float ya[8], yb[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        ya[e] = __fmaf_rn(a[e], cs[e], -__fmul_rn(b[e], sn[e]));
-        yb[e] = __fmaf_rn(b[e], cs[e], __fmul_rn(a[e], sn[e]));
-    }
-    lo = make_uint4(pack_bf16(ya[0], ya[1]), pack_bf16(ya[2], ya[3]), pack_bf16(ya[4], ya[5]), pack_bf16(ya[6], ya[7]));
-    hi = make_uint4(pack_bf16(yb[0], yb[1]), pack_bf16(yb[2], yb[3]), pack_bf16(yb[4], yb[5]), pack_bf16(yb[6], yb[7]));
-}
-
 constexpr int kBlk = 16;      // keys per pipeline stage
 constexpr int kPrefetchRows = 256;  // rows of K and of V a CTA asks L2 for before its stream-order wait (0 = none)
 constexpr int kMaxSplit = 8;  // largest cluster

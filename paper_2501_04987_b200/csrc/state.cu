@@ -143,6 +143,56 @@ cudaError_t launch_chunk_append(const CacheView& cv, treekv_dtype dt, const void
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// In-cache positions (Section 4.1 "Position Encoding") for the tensor-core prefill kernels, whose operands go from
+// memory to the tensor cores without passing through registers: after the chunk has been appended, every live row of
+// a unit - cache slot lam, physical row phys_row(lam) - is encoded at position lam into the rotated-key slab (same row),
+// and every query row of the chunk at its own slot L + t.  Same arithmetic as rope_apply() / the oracle.  The slab is
+// rebuilt on every call because evictions move tokens to other slots; it costs one read and one write of the unit's
+// keys against two passes of attention over them.  bf16, head_dim 128.  One half-warp per row.
+__global__ void rope_chunk_kernel(CacheView cv, ChunkLens lens, int chunk_stride, __nv_bfloat16* __restrict__ k_rot,
+                                  const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ q_rot) {
+    constexpr int D = 128, CPR = 16;
+    const int unit = blockIdx.y;
+    const int b = unit / cv.Hkv, kh = unit % cv.Hkv;
+    const int m = lens.m[b];
+    if (m == 0) return;
+    const int G = cv.Hq / cv.Hkv;
+    const int N = cv.n_seen[unit];
+    const UnitState st = unit_state(N, cv);
+    const int n = st.L + m;
+    const int hw = (blockIdx.x * blockDim.x + threadIdx.x) >> 4, cidx = threadIdx.x & 7;  // half-warp index; piece pair (cidx, cidx + 8)
+    const bool second = (threadIdx.x >> 3) & 1;  // the half-warp's upper eight lanes take the next row
+    const int item = 2 * hw + (second ? 1 : 0);
+    if (item < n) {  // a key row
+        const int lam = item;
+        const size_t row = (size_t)unit * cv.R + phys_row(lam, st);
+        const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(cv.K) + row * D);
+        uint4* dst = reinterpret_cast<uint4*>(k_rot + row * D);
+        uint4 a = src[cidx], c2 = src[cidx + CPR / 2];
+        rope_piece_pair(a, c2, cv.rope_cos + (size_t)lam * (D / 2) + cidx * 8, cv.rope_sin + (size_t)lam * (D / 2) + cidx * 8);
+        dst[cidx] = a; dst[cidx + CPR / 2] = c2;
+    } else if (item < n + m * G) {  // a query row of the chunk: token t, head h of the group
+        const int r = item - n, t = r / G, h = r % G;
+        const size_t qo = (((size_t)b * chunk_stride + t) * cv.Hq + kh * G + h) * D;
+        const uint4* src = reinterpret_cast<const uint4*>(q + qo);
+        uint4* dst = reinterpret_cast<uint4*>(q_rot + qo);
+        const int slot = st.L + t;
+        uint4 a = src[cidx], c2 = src[cidx + CPR / 2];
+        rope_piece_pair(a, c2, cv.rope_cos + (size_t)slot * (D / 2) + cidx * 8, cv.rope_sin + (size_t)slot * (D / 2) + cidx * 8);
+        dst[cidx] = a; dst[cidx + CPR / 2] = c2;
+    }
+}
+cudaError_t launch_rope_chunk(const CacheView& cv, const ChunkLens& lens, int chunk_stride, int max_m, void* k_rot,
+                              const void* q, void* q_rot, cudaStream_t stream) {
+    const int G = cv.Hq / cv.Hkv;
+    const int items = cv.c + max_m + max_m * G;      // key rows + query rows of a unit, at most
+    dim3 grid((items * 8 + 255) / 256, cv.B * cv.Hkv);  // eight lanes per item
+    rope_chunk_kernel<<<grid, 256, 0, stream>>>(cv, lens, chunk_stride, reinterpret_cast<__nv_bfloat16*>(k_rot),
+                                                reinterpret_cast<const __nv_bfloat16*>(q), reinterpret_cast<__nv_bfloat16*>(q_rot));
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Chunk score update: S[row(lam)] += (sum over query tiles of the partial column sums) / G, tiles added in
 // a fixed order so the result does not depend on scheduling.
 __global__ void chunk_scores_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {

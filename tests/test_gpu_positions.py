@@ -63,14 +63,30 @@ def test_decode_with_in_cache_positions(gpu, dtype, d, hq, hkv, split, budget, p
     assert kv.stats()["device_error"] == 0 and rep.decisions > 0
 
 
-@pytest.mark.parametrize("dtype,d,g", [("bf16", 128, 4), ("f32", 64, 1), ("bf16", 64, 2)])
-def test_chunked_prefill_then_decode_with_in_cache_positions(gpu, dtype, d, g):
+@pytest.mark.parametrize("dtype,d,g,path", [("bf16", 128, 4, 0), ("bf16", 128, 4, 1), ("bf16", 128, 4, 3), ("bf16", 128, 1, 2),
+                                            ("f32", 64, 1, 0), ("bf16", 64, 2, 0)])
+def test_chunked_prefill_then_decode_with_in_cache_positions(gpu, dtype, d, g, path):
+    """bf16 / head_dim 128 takes the tensor-core kernels (paths 0, 2, 3), which run on keys and queries that a kernel of
+    their own has encoded at their slots first; path 1, fp32 and head_dim 64 take the CUDA-core kernel, which encodes
+    while it streams."""
     w = W.parity_slice(W.CONFIGS["cfg4"], layers=1, batch=2, n_heads=2 * g, n_kv_heads=2, head_dim=d, dtype=dtype, budget=96,
                        chunk=64, rotate=False)
     kv, orc = _pair(gpu, w, 64)
+    if path:
+        kv.set_option(gpu.OPT_PREFILL_PATH, path)
     rep = Report()
     run_prefill(kv, orc, w, rep, [5 * 64 + 20, 3 * 64], 64)
     run_decode(kv, orc, w, 0, 110, rep, starts=[5 * 64 + 20, 3 * 64])
+    assert kv.stats()["device_error"] == 0
+
+
+def test_larger_chunked_prefill_with_in_cache_positions_on_the_tensor_cores(gpu):
+    """Several key tiles per thread block, chunks that wrap the eviction cycle, a ragged tail, protected tokens."""
+    w = W.parity_slice(W.CONFIGS["cfg3"], layers=1, batch=2, n_heads=2, n_kv_heads=2, budget=384, chunk=256, rotate=False)
+    kv, orc = _pair(gpu, w, 256, ns=4, nr=60)
+    rep = Report()
+    run_prefill(kv, orc, w, rep, [5 * 256 + 77, 4 * 256], 256)
+    run_decode(kv, orc, w, 0, 20, rep, starts=[5 * 256 + 77, 4 * 256])
     assert kv.stats()["device_error"] == 0
 
 
