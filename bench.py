@@ -403,7 +403,7 @@ def main():
     ap.add_argument("--prefill-path", type=int, default=0, help="TREEKV_OPT_PREFILL_PATH for the prefill legs; 0 = automatic")
     ap.add_argument("--prefill-key-split", type=int, default=0, help="TREEKV_OPT_PREFILL_KEY_SPLIT; 0 = automatic")
     ap.add_argument("--no-positions-leg", action="store_true",
-                    help="skip the decode leg that repeats the headline configuration with in-cache positions")
+                    help="skip the decode and prefill legs that repeat the first configuration with in-cache positions")
     ap.add_argument("--fill-by-image", action="store_true",
                     help="decode legs: fill the caches through treekv_import_state (one launch per layer) instead of "
                          "budget + 37 decode steps; for profiling runs")
@@ -462,6 +462,10 @@ def main():
         prefill_legs.append(run_prefill_leg(torch, binding, cfg(name), max(1, args.prefill_chunks), dev, rep, timer, peaks,
                                             not args.no_eviction_stream, args.prefill_path, args.prefill_key_split))
     prefill = prefill_legs[0] if prefill_legs else None
+    if prefill_legs and not args.no_positions_leg:  # the first prefill configuration once more with in-cache positions
+        prefill_legs.append(run_prefill_leg(torch, binding, cfg(prefill["config"]["workload"]), max(1, args.prefill_chunks), dev,
+                                            rep, timer, peaks, not args.no_eviction_stream, args.prefill_path,
+                                            args.prefill_key_split, positions=True))
     if sampler is not None:
         sampler.stop()
 
@@ -630,12 +634,17 @@ def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev
             "config": config_of(w, in_cache_positions=bool(positions))}
 
 
-def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks, eviction_stream=True, prefill_path=0, key_split=0):
+def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks, eviction_stream=True, prefill_path=0, key_split=0,
+                    positions=False):
     tdtype = torch.bfloat16 if pw.dtype == "bf16" else torch.float32
     world, rank = rep.world, rep.rank
     m, c = pw.chunk, pw.budget
     ctxs = [binding.TreeKV(c, pw.n_heads, pw.n_kv_heads, pw.head_dim, pw.dtype, pw.batch, m) for _ in range(pw.layers)]
+    if positions:  # in-cache positions (Section 4.1 "Position Encoding"): one table by cache slot for every layer
+        cos, sin = (torch.from_numpy(x).to(dev) for x in W.rope_tables(c + m, pw.head_dim, pw.rope_base))
     for x in ctxs:
+        if positions:
+            x.set_positions(cos, sin)
         if eviction_stream:
             x.set_option(binding.OPT_EVICTION_STREAM, 1)
         if prefill_path:
@@ -682,7 +691,7 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks, evicti
     return {"metric": "treekv_prefill_tokens_per_s", "value": tok_s, "unit": "tokens/s", "chunks_per_block": n_chunks,
             "blocks": t["blocks"], "region_ms": t["region_ms"], "ms_per_chunk_all_layers": ms / n_chunks,
             "gpu_launches": int(launches), "clocks": t["clocks"],
-            "config": config_of(pw, chunk=m, eviction_stream=bool(eviction_stream),
+            "config": config_of(pw, chunk=m, eviction_stream=bool(eviction_stream), in_cache_positions=bool(positions),
                                 l2="no flush: a chunk reads %.0f MB of K/V per layer and a layer is revisited %d layers later (126 MB L2)"
                                    % (2 * pw.batch * pw.n_kv_heads * (c + m) * pw.head_dim * 2 / 1e6, pw.layers)),
             "roofline": {"bound": "tensor", "achieved": ach3, "peak": sus, "unit": "TFLOP/s", "frac": ach3 / sus,
