@@ -41,16 +41,16 @@ def _pair(binding, w, max_chunk, ns=0, nr=0):
     return kv, orc
 
 
-@pytest.mark.parametrize("path", [0, 1])
-@pytest.mark.parametrize("dtype,d,hq,hkv,split,budget", [("bf16", 128, 8, 2, 0, 40), ("bf16", 64, 2, 2, 2, 40), ("f32", 64, 4, 4, 0, 40),
-                                                         ("f32", 128, 4, 1, 4, 40), ("bf16", 128, 2, 2, 8, 40),
-                                                         ("bf16", 128, 8, 2, 1, 300), ("bf16", 64, 4, 1, 4, 200)])
+_DECODE_CASES = [("bf16", 128, 8, 2, 0, 40), ("bf16", 64, 2, 2, 2, 40), ("f32", 64, 4, 4, 0, 40), ("f32", 128, 4, 1, 4, 40),
+                 ("bf16", 128, 2, 2, 8, 40), ("bf16", 128, 8, 2, 1, 300), ("bf16", 64, 4, 1, 4, 200)]
+
+
+@pytest.mark.parametrize("dtype,d,hq,hkv,split,budget,path",
+                         [c + (0,) for c in _DECODE_CASES] + [c + (1,) for c in _DECODE_CASES if c[0] == "bf16"])
 def test_decode_with_in_cache_positions(gpu, dtype, d, hq, hkv, split, budget, path):
     """Both decode kernels: the mma.sync kernel (bf16, automatic) encodes each key tile at its slots in shared memory,
     the CUDA-core kernel (path 1, and fp32) in registers; budgets of several tiles per warp put the segment boundary
     of the cycle layout and ragged tails inside tiles."""
-    if path == 1 and dtype == "f32":
-        pytest.skip("fp32 always runs the CUDA-core kernel")
     w = W.parity_slice(W.CONFIGS["cfg2"], layers=1, batch=2, n_heads=hq, n_kv_heads=hkv, head_dim=d, dtype=dtype, budget=budget,
                        chunk=0, rotate=False)
     kv, orc = _pair(gpu, w, 0)
