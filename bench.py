@@ -590,7 +590,7 @@ def run_decode_leg(torch, binding, w, steps, warmup, with_e2e, decode_split, dev
     achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
     kernel = "decode_mma_kernel" if w.dtype == "bf16" else "decode_kernel"
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": measured_traffic(kernel, w.name),
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None if positions else measured_traffic(kernel, w.name),
                 "peak_source": peaks["source"], "kernel": kernel, "bytes_per_launch": bytes_per_launch,
                 "launch_us": launch_ms * 1e3, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
     if bytes_per_launch < 20e6:
@@ -700,7 +700,7 @@ def run_prefill_leg(torch, binding, pw, n_chunks, dev, rep, timer, peaks, evicti
                          "two_contractions": {"achieved": ach2, "frac": ach2 / sus, "frac_of_burst": ach2 / burst,
                                               "frac_of_nominal_2250": ach2 / NOMINAL_BF16_TFLOPS,
                                               "counts": "QK^T once and PV: what attention with column sums needs at the least"},
-                         "traffic": measured_traffic(kernel, pw.name), "kernel": kernel,
+                         "traffic": None if positions else measured_traffic(kernel, pw.name), "kernel": kernel,
                          "peak_source": peaks["source"] + " (sustained; the timed region lasts a second or more)",
                          "flops_per_chunk_all_layers": flops3}}
 
