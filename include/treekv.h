@@ -103,7 +103,8 @@ typedef struct {
  * Bytes of device workspace a context of this shape needs (0 if the shape is unsupported).
  * The workspace holds, per (sequence, KV head): K and V slabs of 2*budget + max_chunk rows, the score sums
  * S and the stream positions of the cached tokens; plus per-call scratch for chunked prefill (partial
- * column sums) and staging buffers for the *_host entry points.
+ * column sums), for bf16 / head_dim 128 contexts with chunks a third slab for keys encoded at their cache slots
+ * (used when in-cache positions are on), and staging buffers for the *_host entry points.
  * max_chunk = 0 makes a decode-only context.
  */
 size_t treekv_workspace_bytes(int budget, int n_heads, int n_kv_heads, int head_dim, treekv_dtype dtype,
@@ -291,7 +292,10 @@ treekv_status treekv_set_protection(treekv_ctx* ctx, int n_sink, int n_recent);
  * before the dot product (the paper's runs are bf16 throughout; an fp32 context does not round).
  * Only on a context that has not seen a token (TREEKV_ERR_BAD_STATE otherwise).  Decode steps of a bf16
  * context keep their fast kernel, which encodes each key tile in shared memory on its way to the tensor cores; prefill
- * chunks and fp32 contexts run on the CUDA-core kernels, which encode while they stream.  Host-side only, nothing is enqueued.
+ * chunks of a bf16 / head_dim 128 context keep the tensor-core kernels, which then run on keys and queries that a
+ * kernel of the same call has encoded at their slots (into a second key slab of the workspace and the query staging
+ * buffer: for such a context chunk_stride must not exceed max_chunk, TREEKV_ERR_UNSUPPORTED otherwise); fp32 contexts
+ * and head_dim 64 run on the CUDA-core kernels, which encode while they stream.  Host-side only, nothing is enqueued.
  */
 treekv_status treekv_set_positions(treekv_ctx* ctx, const float* dev_cos, const float* dev_sin, int slots);
 
