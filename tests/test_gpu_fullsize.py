@@ -164,7 +164,7 @@ def _lockstep_sampled(orc, rep, sampled, q, k, v, out, lens, pos_g, cnt_g, sb_g,
     rep.max_score_rel = max(rep.max_score_rel, float(rel.max()))
 
 
-def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_chunk=None):
+def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_chunk=None, positions=False):
     import torch
     from oracle import Oracle
 
@@ -176,6 +176,10 @@ def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_c
     seq_scale = torch.from_numpy(W.seq_key_scales(w)).cuda() if w.key_scale else None
     sampled = sorted(set([(0, 0), (B - 1, Hkv - 1), (B // 2, Hkv // 2)]))
     orc = Oracle(c, g, 1, d, len(sampled))   # sequence s of the oracle follows sampled unit s (one KV head, g query heads)
+    if positions:  # in-cache positions: the same tables on both sides; the brute-force rows below assume none, so they are skipped
+        cos, sin = W.rope_tables(c + m, d, w.rope_base)
+        kv.set_positions(torch.from_numpy(cos).cuda(), torch.from_numpy(sin).cuda())
+        orc.set_rope(cos, sin, round_bf16=True)
     rep = Report()
     hist_k = {u: np.zeros((0, d)) for u in sampled}   # full key / value streams of the sampled units (fp64)
     hist_v = {u: np.zeros((0, d)) for u in sampled}
@@ -196,7 +200,7 @@ def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_c
         out = kv.prefill_chunk(q, k, v, chunk_lens=lens)
         for (b, kh) in sampled:
             mb = lens[b]
-            if mb == 0:
+            if mb == 0 or positions:
                 continue
             kc = k[b, :mb, kh].float().cpu().numpy().astype(np.float64)
             vc = v[b, :mb, kh].float().cpu().numpy().astype(np.float64)
@@ -224,7 +228,7 @@ def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_c
         pos_before, cnt_before = kv.retained_positions()
         pos_before = pos_before.cpu().numpy(); cnt_before = cnt_before.cpu().numpy()
         out = kv.decode_step(q, k, v)
-        for (b, kh) in sampled:
+        for (b, kh) in ([] if positions else sampled):
             hist_k[(b, kh)] = np.concatenate([hist_k[(b, kh)], k[b, kh].float().cpu().numpy().astype(np.float64)[None]])
             hist_v[(b, kh)] = np.concatenate([hist_v[(b, kh)], v[b, kh].float().cpu().numpy().astype(np.float64)[None]])
             vis = np.concatenate([pos_before[b, kh, : cnt_before[b, kh]], [seen[b]]])
@@ -259,6 +263,15 @@ def test_cfg5_full_layer_ragged_prefill(gpu):
     lens = [2 * 4096 + 1024 + 517, 2 * 4096 + 100, 10 * 1024, 2 * 4096 + 1]
     err = _prefill_fullsize(gpu, w, lens, decode_steps=24)
     print("cfg5 full layer: max sampled out err %.3g" % err)
+
+
+def test_cfg5_full_layer_prefill_with_in_cache_positions(gpu):
+    """The same shape with in-cache positions (Section 4.1 "Position Encoding"): the key / query encoding kernel in front
+    of the two-tile tensor-core kernel at its full grid, then the mma.sync decode kernel encoding its tiles, with
+    one-head oracles in lock-step (every output row of the sampled units, retained positions, scores)."""
+    w = W.CONFIGS["cfg5"]
+    lens = [4096 + 1024 + 300, 4096 + 1024, 5 * 1024, 4096 + 17]
+    _prefill_fullsize(gpu, w, lens, decode_steps=8, positions=True)
 
 
 @pytest.mark.parametrize("c,Hq,Hkv", [(16384, 8, 2), (65536, 1, 1)])
