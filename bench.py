@@ -79,6 +79,8 @@ NCU_TRAFFIC = {
         "sha1": "ea6ab7f13538c1adac37fc88f1b172d716eea00e", "profile": "profiles/decode_mma_cfg3_1layer.md"},
     ('prefill_tc2_kernel', 'cfg5'): {"bytes_per_launch": 165586176, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
         "sha1": "d1e43f5667bba313a3102b69a860ed6b1922756f", "profile": "profiles/prefill_tc2_cfg5_1layer.md"},
+    ('prefill_tc2_kernel', 'cfg4'): {"bytes_per_launch": 1166771456, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
+        "sha1": "d1e43f5667bba313a3102b69a860ed6b1922756f", "profile": "profiles/prefill_tc2_cfg4_1layer.md"},
     ('prefill_tc_kernel', 'cfg3'): {"bytes_per_launch": 46755328, "sources": ['prefill_tc.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
         "sha1": "0998349f7d1d6602ae45ca3e94ef7be0d7e5e2e4", "profile": "profiles/prefill_tc_cfg3_2layers.md"},
 }
