@@ -194,15 +194,24 @@ __device__ inline uint32_t rope_pack_bf16(float lo, float hi) {
 // In-cache positions (Section 4.1 "Position Encoding"): 16-byte piece c (8 channels, c < D/16) of a row and its
 // rotate-half partner piece c + D/16, encoded at `slot`, with the numeric contract of rope_apply() in common.cuh:
 // x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin) in fp32, each rounded to bf16.
-__device__ inline void rope_piece_pair(uint4& lo, uint4& hi, const float* cos_row, const float* sin_row) {
+// cos / sin of eight consecutive channels (two float4 each), as loaded from the tables
+struct RopeTab {
+    float4 c0, c1, s0, s1;
+};
+__device__ inline RopeTab rope_tab_load(const float* cos_row, const float* sin_row) {
+    RopeTab t;
+    t.c0 = __ldg(reinterpret_cast<const float4*>(cos_row));
+    t.c1 = __ldg(reinterpret_cast<const float4*>(cos_row) + 1);
+    t.s0 = __ldg(reinterpret_cast<const float4*>(sin_row));
+    t.s1 = __ldg(reinterpret_cast<const float4*>(sin_row) + 1);
+    return t;
+}
+__device__ inline void rope_piece_pair(uint4& lo, uint4& hi, const RopeTab& t) {
     float a[8], b[8];
     Elem<__nv_bfloat16>::unpack(lo, a);
     Elem<__nv_bfloat16>::unpack(hi, b);
-    float cs[8], sn[8];
-    *reinterpret_cast<float4*>(cs) = __ldg(reinterpret_cast<const float4*>(cos_row));
-    *reinterpret_cast<float4*>(cs + 4) = __ldg(reinterpret_cast<const float4*>(cos_row) + 1);
-    *reinterpret_cast<float4*>(sn) = __ldg(reinterpret_cast<const float4*>(sin_row));
-    *reinterpret_cast<float4*>(sn + 4) = __ldg(reinterpret_cast<const float4*>(sin_row) + 1);
+    const float cs[8] = {t.c0.x, t.c0.y, t.c0.z, t.c0.w, t.c1.x, t.c1.y, t.c1.z, t.c1.w};
+    const float sn[8] = {t.s0.x, t.s0.y, t.s0.z, t.s0.w, t.s1.x, t.s1.y, t.s1.z, t.s1.w};
     float ya[8], yb[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
@@ -211,6 +220,9 @@ __device__ inline void rope_piece_pair(uint4& lo, uint4& hi, const float* cos_ro
     }
     lo = make_uint4(rope_pack_bf16(ya[0], ya[1]), rope_pack_bf16(ya[2], ya[3]), rope_pack_bf16(ya[4], ya[5]), rope_pack_bf16(ya[6], ya[7]));
     hi = make_uint4(rope_pack_bf16(yb[0], yb[1]), rope_pack_bf16(yb[2], yb[3]), rope_pack_bf16(yb[4], yb[5]), rope_pack_bf16(yb[6], yb[7]));
+}
+__device__ inline void rope_piece_pair(uint4& lo, uint4& hi, const float* cos_row, const float* sin_row) {
+    rope_piece_pair(lo, hi, rope_tab_load(cos_row, sin_row));
 }
 #endif
 

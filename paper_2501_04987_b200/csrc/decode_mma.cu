@@ -88,7 +88,7 @@ int mma_rows_cap(int c, int split) {
 
 }  // namespace
 
-template <int D, int G, int NW, int NS>
+template <int D, int G, int NW, int NS, bool ROPE>
 __global__ void __launch_bounds__(NW * 32)
 decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_in,
                   const __nv_bfloat16* __restrict__ v_in, __nv_bfloat16* __restrict__ out, ActiveMask active,
@@ -280,7 +280,7 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
     const T* tv = reinterpret_cast<const T*>(tok + (G + 1) * ROWB);
     // in-cache positions: the query sits in the last slot, n - 1; its staged rows are encoded in place.  Keys stay as
     // given in the cache and are encoded at their slot in shared memory, tile by tile, below.
-    const bool rope = cv.rope_cos != nullptr;
+    constexpr bool rope = ROPE;  // in-cache positions: a kernel of its own (it keeps the next tile's cos / sin in registers)
     if (rope) {
         for (int e = tid; e < G * (CPR / 2); e += NT) {
             const int r = e / (CPR / 2), cidx = e % (CPR / 2);
@@ -382,6 +382,21 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[cc][e] = 0.f;
 
+    // In-cache positions: the cos / sin values a lane needs for a tile (piece pairs (c, c + CPR/2) of rows, eight lanes
+    // per row) are fetched into registers one tile ahead, right after the previous tile has been encoded, so their
+    // latency hides behind that tile's MMAs.
+    constexpr int kRopeItems = kBlk * (CPR / 2) / 32;
+    RopeTab tab[ROPE ? kRopeItems : 1];
+    auto load_tabs = [&](int blk) {
+#pragma unroll
+        for (int i2 = 0; i2 < (ROPE ? kRopeItems : 0); ++i2) {
+            const int item = lane + 32 * i2, r = item / (CPR / 2), cidx = item % (CPR / 2);
+            const int slot = min(lo + blk * kBlk + r, n - 1);
+            tab[i2] = rope_tab_load(cv.rope_cos + (size_t)slot * (D / 2) + cidx * 8, cv.rope_sin + (size_t)slot * (D / 2) + cidx * 8);
+        }
+    };
+    if (rope && warp < nblk) load_tabs(warp);
+
     for (int it = 0;; ++it) {
         const int blk = warp + it * NW;
         if (blk >= nblk) break;
@@ -394,15 +409,15 @@ decode_mma_kernel(CacheView cv, const __nv_bfloat16* __restrict__ q, const __nv_
             // takes piece pairs (c, c + CPR/2) of rows, eight lanes per row (conflict-free 16-byte accesses)
             unsigned char* kt = ring + (size_t)(warp * NS + stage) * STAGE;
 #pragma unroll
-            for (int i2 = 0; i2 < kBlk * (CPR / 2) / 32; ++i2) {
+            for (int i2 = 0; i2 < (ROPE ? kRopeItems : 0); ++i2) {
                 const int item = lane + 32 * i2, r = item / (CPR / 2), cidx = item % (CPR / 2);
-                const int slot = min(lo + blk * kBlk + r, n - 1);
                 uint4* plo = reinterpret_cast<uint4*>(kt + r * ROWB + ((cidx ^ (r & 7)) << 4));
                 uint4* phi = reinterpret_cast<uint4*>(kt + r * ROWB + (((cidx + CPR / 2) ^ (r & 7)) << 4));
                 uint4 a = *plo, bq = *phi;
-                rope_piece_pair(a, bq, cv.rope_cos + (size_t)slot * (D / 2) + cidx * 8, cv.rope_sin + (size_t)slot * (D / 2) + cidx * 8);
+                rope_piece_pair(a, bq, tab[i2]);
                 *plo = a; *phi = bq;
             }
+            if (blk + NW < nblk) load_tabs(blk + NW);
             __syncwarp();
         }
 
@@ -653,10 +668,10 @@ static int decode_sm_count() {
     return std::max(sm_count[dev], 1);
 }
 
-template <int D, int G, int NS>
-static cudaError_t launch_decode_mma_ns(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+template <int D, int G, int NS, bool ROPE>
+static cudaError_t launch_decode_mma_nsr(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
                                         const ActiveMask& active, int split, int inputs_final, cudaStream_t stream) {
-    auto kern = decode_mma_kernel<D, G, kMmaWarps, NS>;
+    auto kern = decode_mma_kernel<D, G, kMmaWarps, NS, ROPE>;
     const int rows_cap = mma_rows_cap(cv.c, split);
     size_t smem = decode_mma_smem_bytes_ns(G, D, cv.c, split, NS);
     static size_t smem_set[64] = {};  // per device: the opt-in limit only ever needs raising
@@ -696,6 +711,13 @@ static cudaError_t launch_decode_mma_ns(const CacheView& cv, const void* q, cons
     using T = __nv_bfloat16;
     return cudaLaunchKernelEx(&cfg, kern, cv, reinterpret_cast<const T*>(q), reinterpret_cast<const T*>(k),
                               reinterpret_cast<const T*>(v), reinterpret_cast<T*>(out), active, rows_cap, inputs_final);
+}
+
+template <int D, int G, int NS>
+static cudaError_t launch_decode_mma_ns(const CacheView& cv, const void* q, const void* k, const void* v, void* out,
+                                        const ActiveMask& active, int split, int inputs_final, cudaStream_t stream) {
+    return cv.rope_cos ? launch_decode_mma_nsr<D, G, NS, true>(cv, q, k, v, out, active, split, inputs_final, stream)
+                       : launch_decode_mma_nsr<D, G, NS, false>(cv, q, k, v, out, active, split, inputs_final, stream);
 }
 
 // A thread block that has an SM to itself keeps three tiles per warp in flight instead of two (when they fit): one
