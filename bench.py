@@ -69,20 +69,20 @@ def measured_peaks():
 # profiles/, valid for the named workload's per-layer shape and only while the kernel's sources are the ones that
 # were profiled: a changed source file makes the entry stale and the reported traffic null.
 NCU_TRAFFIC = {
-    ('decode_mma_kernel', 'cfg4'): {"bytes_per_launch": 277511936, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
-        "sha1": "ea6ab7f13538c1adac37fc88f1b172d716eea00e", "profile": "profiles/decode_mma_cfg4_1layer.md"},
-    ('decode_mma_kernel', 'cfg2'): {"bytes_per_launch": 141881344, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
-        "sha1": "ea6ab7f13538c1adac37fc88f1b172d716eea00e", "profile": "profiles/decode_mma_cfg2_1layer.md"},
-    ('decode_mma_kernel', 'cfg5'): {"bytes_per_launch": 69300480, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
-        "sha1": "ea6ab7f13538c1adac37fc88f1b172d716eea00e", "profile": "profiles/decode_mma_cfg5_1layer.md"},
-    ('decode_mma_kernel', 'cfg3'): {"bytes_per_launch": 33920512, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
-        "sha1": "ea6ab7f13538c1adac37fc88f1b172d716eea00e", "profile": "profiles/decode_mma_cfg3_1layer.md"},
-    ('prefill_tc2_kernel', 'cfg5'): {"bytes_per_launch": 165586176, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
-        "sha1": "d1e43f5667bba313a3102b69a860ed6b1922756f", "profile": "profiles/prefill_tc2_cfg5_1layer.md"},
-    ('prefill_tc2_kernel', 'cfg4'): {"bytes_per_launch": 1166771456, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
-        "sha1": "d1e43f5667bba313a3102b69a860ed6b1922756f", "profile": "profiles/prefill_tc2_cfg4_1layer.md"},
-    ('prefill_tc_kernel', 'cfg3'): {"bytes_per_launch": 46755328, "sources": ['prefill_tc.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
-        "sha1": "0998349f7d1d6602ae45ca3e94ef7be0d7e5e2e4", "profile": "profiles/prefill_tc_cfg3_2layers.md"},
+    ('decode_mma_kernel', 'cfg4'): {"bytes_per_launch": 278167552, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
+        "sha1": "68d62dd60bbcd00707594a51ac84df544e179320", "profile": "profiles/decode_mma_cfg4_1layer.md"},
+    ('decode_mma_kernel', 'cfg2'): {"bytes_per_launch": 141089792, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
+        "sha1": "68d62dd60bbcd00707594a51ac84df544e179320", "profile": "profiles/decode_mma_cfg2_1layer.md"},
+    ('decode_mma_kernel', 'cfg5'): {"bytes_per_launch": 69239808, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
+        "sha1": "68d62dd60bbcd00707594a51ac84df544e179320", "profile": "profiles/decode_mma_cfg5_1layer.md"},
+    ('decode_mma_kernel', 'cfg3'): {"bytes_per_launch": 33949696, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
+        "sha1": "68d62dd60bbcd00707594a51ac84df544e179320", "profile": "profiles/decode_mma_cfg3_1layer.md"},
+    ('prefill_tc2_kernel', 'cfg5'): {"bytes_per_launch": 165677568, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
+        "sha1": "caa9d345bc96b97cebbf7872a73829f91129dac1", "profile": "profiles/prefill_tc2_cfg5_1layer.md"},
+    ('prefill_tc2_kernel', 'cfg4'): {"bytes_per_launch": 1167068928, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
+        "sha1": "caa9d345bc96b97cebbf7872a73829f91129dac1", "profile": "profiles/prefill_tc2_cfg4_1layer.md"},
+    ('prefill_tc_kernel', 'cfg3'): {"bytes_per_launch": 46872064, "sources": ['prefill_tc.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
+        "sha1": "8d92180bea87292fdd37121f278e962a3d3ccdc4", "profile": "profiles/prefill_tc_cfg3_2layers.md"},
 }
 
 
