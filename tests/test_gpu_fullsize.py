@@ -11,8 +11,9 @@ follow every unit at these sizes, so:
     retained before the chunk | chunk tokens up to the row's own] from the raw input stream, and the cache
     invariants that hold at any size are checked after every call (length = min(seen, budget), strictly increasing
     positions, every averaged score in [0, 1]).
-Inputs are seeded Gaussians drawn with torch on the device (keys with the configuration's outlier channels or
-per-sequence scale; no rotary embedding here - the lock-step tests on slices use the full recipe).
+Inputs are seeded Gaussians drawn with torch on the device with the recipe's structure (keys with the configuration's
+outlier channels or per-sequence scale; q and k carry rotary embedding at their stream positions);
+the lock-step tests on slices use the recipe's own counter-based generator.
 """
 import math
 
@@ -39,12 +40,22 @@ def gpu():
     return binding
 
 
-def _draw(torch, gen, shape, scale_last=None, seq_scale=None):
+def _draw(torch, gen, shape, scale_last=None, seq_scale=None, pos=None, base=None):
+    """Seeded Gaussians on the device with the recipe's structure: outlier key channels or per-sequence key scale, and -
+    when `pos` (stream positions, broadcastable to shape[:-2]) is given - rotate-half rotary embedding at those
+    positions, then rounding to bf16."""
     x = torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32)
     if scale_last is not None:
         x[..., scale_last] *= 8.0
     if seq_scale is not None:
         x *= seq_scale.view(-1, *([1] * (x.dim() - 1)))
+    if pos is not None:
+        d = shape[-1]
+        inv_freq = base ** (-torch.arange(d // 2, device="cuda", dtype=torch.float64) * 2.0 / d)
+        ang = pos.to(torch.float64).unsqueeze(-1).unsqueeze(-1) * inv_freq            # [..., 1, d/2]
+        cos, sin = torch.cos(ang).float(), torch.sin(ang).float()
+        x1, x2 = x[..., : d // 2], x[..., d // 2:]
+        x = torch.cat([x1 * cos - x2 * sin, x2 * cos + x1 * sin], dim=-1)
     return x.to(torch.bfloat16)
 
 
@@ -87,8 +98,9 @@ def test_cfg2_full_layer_decode_sampled_units(gpu):
     reps = [Report() for _ in sampled]
     max_err = 0.0
     for t in range(steps):
-        q = _draw(torch, gen, (w.batch, w.n_heads, w.head_dim))
-        k = _draw(torch, gen, (w.batch, w.n_kv_heads, w.head_dim), scale_last=out_ch)
+        pos = torch.full((w.batch,), t, device="cuda")
+        q = _draw(torch, gen, (w.batch, w.n_heads, w.head_dim), pos=pos, base=w.rope_base)
+        k = _draw(torch, gen, (w.batch, w.n_kv_heads, w.head_dim), scale_last=out_ch, pos=pos, base=w.rope_base)
         v = _draw(torch, gen, (w.batch, w.n_kv_heads, w.head_dim))
         out = kv.decode_step(q, k, v)
         pos, cnt = kv.retained_positions()
@@ -192,8 +204,10 @@ def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_c
     max_err = 0.0
     for call in range(len(bounds) - 1):
         lens = [max(0, min(bounds[call + 1], L) - bounds[call]) for L in lens_total]
-        q = _draw(torch, gen, (B, m, Hq, d))
-        k = _draw(torch, gen, (B, m, Hkv, d), seq_scale=seq_scale)
+        # the recipe rotates q and k at their stream positions (with in-cache positions they stay unrotated)
+        pos = None if positions else (torch.tensor(seen, device="cuda").view(B, 1) + torch.arange(m, device="cuda").view(1, m))
+        q = _draw(torch, gen, (B, m, Hq, d), pos=pos, base=w.rope_base)
+        k = _draw(torch, gen, (B, m, Hkv, d), seq_scale=seq_scale, pos=pos, base=w.rope_base)
         v = _draw(torch, gen, (B, m, Hkv, d))
         pos_before, cnt_before = kv.retained_positions()
         pos_before = pos_before.cpu().numpy(); cnt_before = cnt_before.cpu().numpy()
@@ -222,8 +236,9 @@ def _prefill_fullsize(gpu, w, lens_total, decode_steps, n_sample_rows=6, first_c
     assert [kv.tokens_seen(b) for b in range(B)] == seen
     # batched decode steps at ragged stream positions: sampled rows against brute force over the retained set
     for step in range(decode_steps):
-        q = _draw(torch, gen, (B, Hq, d))
-        k = _draw(torch, gen, (B, Hkv, d), seq_scale=seq_scale)
+        pos = None if positions else torch.tensor(seen, device="cuda").view(B)
+        q = _draw(torch, gen, (B, Hq, d), pos=pos, base=w.rope_base)
+        k = _draw(torch, gen, (B, Hkv, d), seq_scale=seq_scale, pos=pos, base=w.rope_base)
         v = _draw(torch, gen, (B, Hkv, d))
         pos_before, cnt_before = kv.retained_positions()
         pos_before = pos_before.cpu().numpy(); cnt_before = cnt_before.cpu().numpy()
