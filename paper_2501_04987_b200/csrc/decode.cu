@@ -29,6 +29,11 @@ decode_kernel(CacheView cv, const T* __restrict__ q, const T* __restrict__ k_in,
     const int rank = (int)cluster.block_rank();
     const int nsplit = (int)cluster.num_blocks();
     const int kh = blockIdx.y, b = blockIdx.z;
+    // Programmatic dependent launch: the next kernel in the stream may be scheduled while this one runs, and nothing
+    // below the wait touches memory before the previous kernel's writes are complete and visible.  Every block waits,
+    // also one of an inactive sequence.
+    pdl_trigger();
+    pdl_wait();
     if (!active.test(b)) return;  // the whole cluster shares b
 
     const int unit = b * cv.Hkv + kh;
@@ -222,20 +227,29 @@ static cudaError_t launch_decode_t(const CacheView& cv, const void* q, const voi
     auto kern = decode_kernel<T, D, G, U>;
     const int rows_cap = (cv.c + 1 + split - 1) / split;
     const size_t smem = decode_smem_bytes(G, D, cv.c, split);
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    static size_t smem_set[64] = {};  // per device: the opt-in limit only ever needs raising
+    int dev = 0;
+    cudaGetDevice(&dev);
+    dev &= 63;
+    if (smem > smem_set[dev]) {
+        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        smem_set[dev] = smem;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(split, cv.Hkv, cv.B);
     cfg.blockDim = dim3(kDecodeThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = split;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the kernel orders itself with griddepcontrol.wait
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, cv, reinterpret_cast<const T*>(q), reinterpret_cast<const T*>(k),
                               reinterpret_cast<const T*>(v), reinterpret_cast<T*>(out), active, rows_cap);
 }
