@@ -413,6 +413,25 @@ def test_eviction_stream_gives_the_same_bits_and_follows_the_oracle(gpu):
     for (sa, pa), (sb, pb) in zip(results[0][2], results[1][2]):
         assert torch.equal(sa, sb) and torch.equal(pa, pb)
 
+    # calls of every other kind right behind a chunk, without synchronising: each orders itself behind the eviction
+    kv = gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, w.chunk)
+    ref = gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, w.chunk)
+    kv.set_option(gpu.OPT_EVICTION_STREAM, 1)
+    for c in range(4):
+        kv.prefill_chunk(*chunks[c][0]); ref.prefill_chunk(*chunks[c][0])
+    img, seen = kv.export_state()                       # export behind a pending eviction
+    img_r, seen_r = ref.export_state()
+    units = w.batch * w.n_kv_heads
+    main = 2 * units * w.budget * w.head_dim * 2 + 2 * units * w.budget * 4   # K, V, S, positions (the rest is padded counters)
+    assert seen == seen_r and torch.equal(img[:main], img_r[:main])
+    kv.prefill_chunk(*chunks[4][0])
+    kv.reset()                                          # reset behind a pending eviction, then the same stream again
+    kv.import_state(img, seen)
+    kv.prefill_chunk(*chunks[4][0]); ref.prefill_chunk(*chunks[4][0])
+    assert torch.equal(kv.scores(), ref.scores()) and torch.equal(kv.retained_positions()[0], ref.retained_positions()[0])
+    assert kv.stats()["device_error"] == 0
+    del kv, ref
+
     w1 = W.parity_slice(W.CONFIGS["cfg5"], layers=1, batch=2, n_heads=8, n_kv_heads=2, budget=256, chunk=128)
     kv, orc = _pair(gpu, w1)
     kv.set_option(gpu.OPT_EVICTION_STREAM, 1)

@@ -138,3 +138,14 @@ def test_argument_and_state_errors(gpu):
     x = torch.zeros((1, 2, 64), device="cuda")
     kv.decode_step(x, x, x)
     assert gpu.treekv_set_positions(kv._h, cos.data_ptr(), sin.data_ptr(), 24) == 2      # the cache is in use
+    # tensor-core prefill with positions keeps the encoded queries in a buffer sized for max_chunk: a larger stride of the
+    # caller's tensors is refused before anything is enqueued
+    kv2 = gpu.TreeKV(256, 2, 2, 128, "bf16", 1, 128)
+    cos2 = torch.zeros((384, 64), device="cuda"); sin2 = torch.zeros((384, 64), device="cuda")
+    kv2.set_positions(cos2, sin2)
+    y = torch.zeros((1, 256, 2, 128), device="cuda", dtype=torch.bfloat16)
+    with pytest.raises(gpu.TreeKVError) as ei:
+        kv2.prefill_chunk(y, y, y, chunk_lens=[128])
+    assert ei.value.status == 4 and kv2.tokens_seen(0) == 0
+    kv2.prefill_chunk(y[:, :128].contiguous(), y[:, :128].contiguous(), y[:, :128].contiguous())
+    assert kv2.tokens_seen(0) == 128 and kv2.stats()["device_error"] == 0
