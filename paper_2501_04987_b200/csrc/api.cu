@@ -512,6 +512,19 @@ treekv_status treekv_export_state(treekv_ctx* ctx, void* dev_image, int64_t* hos
     StateImage img;
     state_image_layout(ctx, dev_image, &img);
     cudaError_t e = join_eviction_stream(ctx, static_cast<cudaStream_t>(stream));
+    // every part starts on a 256-byte boundary: zero the padding behind each, so that two images of the same state are equal
+    // byte for byte (the kernel fills every byte of the parts themselves)
+    {
+        const size_t slots = (size_t)ctx->cv.B * ctx->cv.Hkv * ctx->cv.c;
+        const size_t sizes[6] = {slots * ctx->cv.d * ctx->elem, slots * ctx->cv.d * ctx->elem, slots * 4, slots * 4,
+                                 (size_t)ctx->cv.B * 4, (size_t)ctx->cv.B * 4};
+        size_t off = 0;
+        for (int part = 0; part < 6 && e == cudaSuccess; ++part) {
+            const size_t end = off + sizes[part], next = align_up(end);
+            if (next > end) e = cudaMemsetAsync(static_cast<char*>(dev_image) + end, 0, next - end, static_cast<cudaStream_t>(stream));
+            off = next;
+        }
+    }
     if (e == cudaSuccess) e = launch_export_state(ctx->cv, ctx->dt, img, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;

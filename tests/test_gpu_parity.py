@@ -421,9 +421,7 @@ def test_eviction_stream_gives_the_same_bits_and_follows_the_oracle(gpu):
         kv.prefill_chunk(*chunks[c][0]); ref.prefill_chunk(*chunks[c][0])
     img, seen = kv.export_state()                       # export behind a pending eviction
     img_r, seen_r = ref.export_state()
-    units = w.batch * w.n_kv_heads
-    main = 2 * units * w.budget * w.head_dim * 2 + 2 * units * w.budget * 4   # K, V, S, positions (the rest is padded counters)
-    assert seen == seen_r and torch.equal(img[:main], img_r[:main])
+    assert seen == seen_r and torch.equal(img, img_r)
     kv.prefill_chunk(*chunks[4][0])
     kv.reset()                                          # reset behind a pending eviction, then the same stream again
     kv.import_state(img, seen)
