@@ -86,6 +86,13 @@ def compare_state(kv, orc, rep, check_scores=True):
         rep.max_score_rel = max(rep.max_score_rel, float(rel.max()))
 
 
+def _f64(t):
+    """Device tensor -> float64 numpy.  Rows the library does not write (beyond a sequence's length, inactive sequences)
+    hold whatever the allocation held, possibly signalling NaNs: they are never compared, only converted."""
+    with np.errstate(invalid="ignore"):
+        return t.float().cpu().numpy().astype(np.float64)
+
+
 def step_decode(kv, orc, q, k, v, dtype, rep, active=None, check_scores=True):
     """q [B,Hq,d], k,v [B,Hkv,d] float32 numpy holding dtype-rounded values."""
     import torch
@@ -97,7 +104,7 @@ def step_decode(kv, orc, q, k, v, dtype, rep, active=None, check_scores=True):
     ev0 = evicted_total(orc)
     nt, fl = orc.evict(pos_g.cpu().numpy(), cnt_g.cpu().numpy(), NEAR_TIE)
     rep.tally(orc, ev0, nt, fl)
-    og = out_g.float().cpu().numpy().astype(np.float64)
+    og = _f64(out_g)
     sel = slice(None) if active is None else np.asarray(active, bool)
     err = float(np.abs(og[sel] - out_o[sel]).max()) if np.size(og[sel]) else 0.0
     rep.max_out_err = max(rep.max_out_err, err)
@@ -118,7 +125,7 @@ def step_prefill(kv, orc, q, k, v, dtype, rep, chunk_lens=None, check_scores=Tru
     ev0 = evicted_total(orc)
     nt, fl = orc.evict(pos_g.cpu().numpy(), cnt_g.cpu().numpy(), NEAR_TIE)
     rep.tally(orc, ev0, nt, fl)
-    og = out_g.float().cpu().numpy().astype(np.float64)
+    og = _f64(out_g)
     err = 0.0
     for b in range(B):
         if lens[b]:
@@ -145,7 +152,7 @@ def step_oneshot(kv, orc, q, k, v, block, dtype, rep, lens=None, check_scores=Tr
     rep.decisions += (after - ev0) // block * orc.Hkv
     rep.near_ties += nt; rep.flips += fl; rep.calls += 1
     assert rep.flips <= rep.near_ties <= rep.decisions or rep.near_ties == 0, repr(rep)
-    og = out_g.float().cpu().numpy().astype(np.float64)
+    og = _f64(out_g)
     err = 0.0
     for b in range(B):
         if ls[b]:
