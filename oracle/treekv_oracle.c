@@ -55,7 +55,11 @@
  *     numeric contract follows the paper's "bf16 precision" set-up: the rotated q and k are computed in fp32 as
  *     x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin) and rounded to the cache's element type before
  *     the fp64 dot product (no rounding for an fp32 cache).
- *   PARITY UNPINNED: the last five readings are not fixed by anything the paper
+ *   - accumulated criterion (Section 4.1 "Importance Score": "accumulated and normalized attention weights" were
+ *     also tried; only the first has an evident definition): TKVO_RULE_ACCUMULATED compares S instead of
+ *     S-bar = S / C in Algorithm 1's branch, and block means of S in the one-shot prefill.  Pinned by a dictionary
+ *     restatement and by the closed form under uniform attention (older token = larger sum = keep-left ladder).
+ *   PARITY UNPINNED: the grouped-query, chunked-prefill, protected-token, one-shot and in-cache-position readings are not fixed by anything the paper
  *   prints; the tests constrain them (m=1 equals a decode step, mass
  *   conservation, score-free rules give identical retained sets) but cannot
  *   pin them to the paper.
@@ -68,6 +72,8 @@
 #define TKVO_RULE_SCORES 0     /* Algorithm 1 */
 #define TKVO_RULE_KEEP_LEFT 1  /* Section 5.4 ablation: always keep slot idx */
 #define TKVO_RULE_EVICT_LEFT 2 /* what an exact tie does: always evict slot idx */
+#define TKVO_RULE_ACCUMULATED 3 /* Section 4.1 "Importance Score" names accumulated attention weights as a criterion
+                                   the authors also tried: Algorithm 1 with S in place of S-bar = S / C */
 
 #define TKVO_IDX_CYCLE 0   /* idx <- (idx mod c) + 1   (prose of Section 4.1) */
 #define TKVO_IDX_LITERAL 1 /* idx <- (idx+1) mod c + 1 (Algorithm 1 as printed) */
@@ -377,7 +383,8 @@ void tkvo_evict_blocks(tkvo *o, const int32_t *hint_pos, const int32_t *hint_cnt
             double *score = (double *)malloc(sizeof(double) * (size_t)nb);
             for (int kb = 0; kb < nb; ++kb) { /* averaged importance of the b tokens of the block */
                 double a = 0.0;
-                for (int t = 0; t < bs; ++t) a += u->S[kb * bs + t] / (double)u->C[kb * bs + t];
+                for (int t = 0; t < bs; ++t)
+                    a += o->rule == TKVO_RULE_ACCUMULATED ? u->S[kb * bs + t] : u->S[kb * bs + t] / (double)u->C[kb * bs + t];
                 score[kb] = a / (double)bs;
             }
             int *cache = (int *)malloc(sizeof(int) * (size_t)(cb + 1)); /* block numbers, in order */
@@ -466,8 +473,9 @@ void tkvo_evict(tkvo *o, const int32_t *hint_pos, const int32_t *hint_cnt, doubl
                 if (o->rule == TKVO_RULE_KEEP_LEFT) evict_right = 1;
                 else if (o->rule == TKVO_RULE_EVICT_LEFT) evict_right = 0;
                 else {
-                    const double sl = u->S[l] / (double)u->C[l]; /* Alg. 1: S-bar = S / C */
-                    const double sr = u->S[r] / (double)u->C[r];
+                    const int acc = o->rule == TKVO_RULE_ACCUMULATED;
+                    const double sl = acc ? u->S[l] : u->S[l] / (double)u->C[l]; /* Alg. 1: S-bar = S / C */
+                    const double sr = acc ? u->S[r] : u->S[r] / (double)u->C[r];
                     evict_right = (sl > sr);                      /* Alg. 1: strict > */
                     const double mxabs = fmax(fabs(sl), fabs(sr));
                     const double gap = mxabs > 0.0 ? fabs(sl - sr) / mxabs : 0.0;

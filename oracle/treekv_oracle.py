@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "treekv_oracle.c")
 _LIB = os.path.join(_HERE, "libtreekv_oracle.so")
 
-RULE_SCORES, RULE_KEEP_LEFT, RULE_EVICT_LEFT = 0, 1, 2
+RULE_SCORES, RULE_KEEP_LEFT, RULE_EVICT_LEFT, RULE_ACCUMULATED = 0, 1, 2, 3
 IDX_CYCLE, IDX_LITERAL = 0, 1
 
 _lib = None

@@ -10,7 +10,7 @@ import math
 import numpy as np
 import pytest
 
-from oracle import RULE_EVICT_LEFT, RULE_KEEP_LEFT, Oracle
+from oracle import RULE_ACCUMULATED, RULE_EVICT_LEFT, RULE_KEEP_LEFT, Oracle
 
 
 def _prompt(seed, T, Hq, Hkv, d):
@@ -69,13 +69,15 @@ def _brute_force_blocks(sbar, b, cb, rule=None):
     return [x["first"] + t for x in cache for t in range(b)], idx
 
 
+@pytest.mark.parametrize("accumulated", [False, True])
 @pytest.mark.parametrize("c,b,T", [(12, 4, 36), (16, 2, 70), (8, 8, 40), (6, 1, 31), (12, 3, 12), (12, 3, 9)])
-def test_block_tournament_matches_brute_force(oracle_lib, c, b, T):
+def test_block_tournament_matches_brute_force(oracle_lib, c, b, T, accumulated):
+    """`accumulated`: block means of S instead of S / C (Section 4.1 "Importance Score", the criterion also tried)."""
     Hq, Hkv, d = 2, 1, 4
     q, k, v = _prompt(42, T, Hq, Hkv, d)
-    o = Oracle(c, Hq, Hkv, d, 1)
+    o = Oracle(c, Hq, Hkv, d, 1, rule=RULE_ACCUMULATED) if accumulated else Oracle(c, Hq, Hkv, d, 1)
     o.prefill_oneshot_attend(q, k, v, b)
-    sbar = o.unit(0, 0)[3].copy()
+    sbar = o.unit(0, 0)[1].copy() if accumulated else o.unit(0, 0)[3].copy()
     S_before = o.unit(0, 0)[1].copy()
     o.evict_blocks()
     want, idx_b = _brute_force_blocks(sbar, b, c // b)

@@ -10,7 +10,7 @@ import os
 import numpy as np
 import pytest
 
-from oracle import IDX_LITERAL, RULE_EVICT_LEFT, RULE_KEEP_LEFT, RULE_SCORES, Oracle
+from oracle import IDX_LITERAL, RULE_ACCUMULATED, RULE_EVICT_LEFT, RULE_KEEP_LEFT, RULE_SCORES, Oracle
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -107,11 +107,12 @@ def test_output_is_attention_over_retained_set(oracle_lib):
         assert len(retained) <= c
 
 
-def _brute_force_treekv(q, k, v, c):
+def _brute_force_treekv(q, k, v, c, accumulated=False):
     """Independent restatement for one head: dictionaries keyed by token, scores from their definition.
 
     Averaged attention weight of token j at step t (Section 4.1 "Importance Score"): the mean, over the
-    steps since j arrived, of the attention weight j received.
+    steps since j arrived, of the attention weight j received.  `accumulated`: the sum instead of the mean
+    (the accumulated attention weight the same paragraph names as a criterion that was also tried).
     """
     T, d = q.shape
     received = {}          # token -> list of weights received, one per step present
@@ -126,8 +127,8 @@ def _brute_force_treekv(q, k, v, c):
             received[j].append(w)
         if len(cache) > c:
             a, b = cache[idx - 1], cache[idx]
-            sa = sum(received[a]) / len(received[a])
-            sb = sum(received[b]) / len(received[b])
+            sa = sum(received[a]) / (1 if accumulated else len(received[a]))
+            sb = sum(received[b]) / (1 if accumulated else len(received[b]))
             cache.remove(b if sa > sb else a)
             idx = idx % c + 1
         history.append(list(cache))
@@ -143,6 +144,39 @@ def test_matches_brute_force_on_tiny_inputs(oracle_lib):
         for t in range(T):
             o.decode_step(q[t], k[t], v[t])
             assert list(o.positions(0, 0)) == hist[t], (seed, c, t)
+
+
+def test_accumulated_criterion_matches_brute_force_and_differs_from_the_average(oracle_lib):
+    """Section 4.1 "Importance Score": accumulated attention weights as the criterion, S in place of S / C."""
+    differs = False
+    for seed, c in [(11, 4), (12, 5), (13, 8)]:
+        T, d = 37, 4
+        q, k, v = _stream(seed, T, 1, 1, d, peaked=True)
+        hist = _brute_force_treekv(q[:, 0, 0], k[:, 0, 0], v[:, 0, 0], c, accumulated=True)
+        hist_avg = _brute_force_treekv(q[:, 0, 0], k[:, 0, 0], v[:, 0, 0], c)
+        o = Oracle(c, 1, 1, d, 1, rule=RULE_ACCUMULATED)
+        for t in range(T):
+            o.decode_step(q[t], k[t], v[t])
+            assert list(o.positions(0, 0)) == hist[t], (seed, c, t)
+        differs |= hist[-1] != hist_avg[-1]
+    assert differs   # the inputs tell the two criteria apart
+
+
+def test_accumulated_criterion_under_uniform_attention_is_the_keep_left_ladder(oracle_lib):
+    """With q = 0 every cached token receives 1 / len in every step, so of two tokens the older one has the strictly
+    larger accumulated weight and the left member of every scope survives: the retained set is the closed form of the
+    keep-left ablation (c = 8, 64 tokens: 1, 41, 49, 53, 57, 59, 61, 63).  The averaged criterion sees exact ties for
+    tokens that arrived after the fill instead and ends elsewhere."""
+    c, T, d = 8, 64, 2
+    _, k, v = _stream(10, T, 1, 1, d)
+    q = np.zeros((T, 1, 1, d))
+    o = Oracle(c, 1, 1, d, 1, rule=RULE_ACCUMULATED)
+    a = Oracle(c, 1, 1, d, 1, rule=RULE_SCORES)
+    for t in range(T):
+        o.decode_step(q[t], k[t], v[t])
+        a.decode_step(q[t], k[t], v[t])
+    assert list(o.positions(0, 0) + 1) == [1, 41, 49, 53, 57, 59, 61, 63]
+    assert list(a.positions(0, 0)) != list(o.positions(0, 0))
 
 
 # ---------------------------------------------------------------------------------------------
