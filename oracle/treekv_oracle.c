@@ -55,14 +55,14 @@
  *     numeric contract follows the paper's "bf16 precision" set-up: the rotated q and k are computed in fp32 as
  *     x1' = fma(x1, cos, -(x2 sin)), x2' = fma(x2, cos, x1 sin) and rounded to the cache's element type before
  *     the fp64 dot product (no rounding for an fp32 cache).
- *   - accumulated criterion (Section 4.1 "Importance Score": "accumulated and normalized attention weights" were
- *     also tried; only the first has an evident definition): TKVO_RULE_ACCUMULATED compares S instead of
- *     S-bar = S / C in Algorithm 1's branch, and block means of S in the one-shot prefill.  Pinned by a dictionary
- *     restatement and by the closed form under uniform attention (older token = larger sum = keep-left ladder).
- *   PARITY UNPINNED: the grouped-query, chunked-prefill, protected-token, one-shot and in-cache-position readings are not fixed by anything the paper
- *   prints; the tests constrain them (m=1 equals a decode step, mass
- *   conservation, score-free rules give identical retained sets) but cannot
- *   pin them to the paper.
+ *   - accumulated criterion (Section 4.1 "Importance Score" reports that criteria other than the average were
+ *     tried, among them the accumulated weight, the only one with an evident definition): TKVO_RULE_ACCUMULATED
+ *     compares S instead of S-bar = S / C in Algorithm 1's branch, and block means of S in the one-shot
+ *     prefill.  Pinned by a dictionary restatement and by the closed form under uniform attention (the older
+ *     token has the larger sum, so the left member always survives: the keep-left ladder).
+ *   PARITY UNPINNED: the grouped-query, chunked-prefill, protected-token, one-shot and in-cache-position
+ *   readings are not fixed by anything the paper prints; the tests constrain them (m=1 equals a decode step,
+ *   mass conservation, score-free rules give identical retained sets) but cannot pin them to the paper.
  */
 #include <math.h>
 #include <stdint.h>
@@ -72,8 +72,8 @@
 #define TKVO_RULE_SCORES 0     /* Algorithm 1 */
 #define TKVO_RULE_KEEP_LEFT 1  /* Section 5.4 ablation: always keep slot idx */
 #define TKVO_RULE_EVICT_LEFT 2 /* what an exact tie does: always evict slot idx */
-#define TKVO_RULE_ACCUMULATED 3 /* Section 4.1 "Importance Score" names accumulated attention weights as a criterion
-                                   the authors also tried: Algorithm 1 with S in place of S-bar = S / C */
+#define TKVO_RULE_ACCUMULATED 3 /* Section 4.1 "Importance Score": the accumulated attention weight, a criterion the
+                                   authors also tried: Algorithm 1 with S in place of S-bar = S / C */
 
 #define TKVO_IDX_CYCLE 0   /* idx <- (idx mod c) + 1   (prose of Section 4.1) */
 #define TKVO_IDX_LITERAL 1 /* idx <- (idx+1) mod c + 1 (Algorithm 1 as printed) */
