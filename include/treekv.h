@@ -62,8 +62,16 @@ typedef enum { TREEKV_F32 = 0, TREEKV_BF16 = 1 } treekv_dtype;
 
 /* Eviction rule.  SCORES is Algorithm 1.  KEEP_LEFT is the ablation of Section 5.4 (always keep the
  * left token of the scope).  EVICT_LEFT is what an exact tie does under Algorithm 1's strict '>'.
- * The two score-free rules make the retained set a function of the schedule alone. */
-typedef enum { TREEKV_RULE_SCORES = 0, TREEKV_RULE_KEEP_LEFT = 1, TREEKV_RULE_EVICT_LEFT = 2 } treekv_rule;
+ * The two score-free rules make the retained set a function of the schedule alone.  ACCUMULATED is Algorithm 1
+ * with the accumulated attention weight S in place of the averaged weight S / C - a criterion Section 4.1
+ * ("Importance Score") reports as tried and found worse than the average; in the one-shot prefill a block's
+ * importance is then the mean of its tokens' S.  treekv_scores reports S / C under every rule. */
+typedef enum {
+    TREEKV_RULE_SCORES = 0,
+    TREEKV_RULE_KEEP_LEFT = 1,
+    TREEKV_RULE_EVICT_LEFT = 2,
+    TREEKV_RULE_ACCUMULATED = 3
+} treekv_rule;
 
 /* Options for treekv_set_option. */
 typedef enum {

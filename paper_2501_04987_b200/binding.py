@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libtreekv.so")
 
 TREEKV_OK = 0
 TREEKV_F32, TREEKV_BF16 = 0, 1
-RULE_SCORES, RULE_KEEP_LEFT, RULE_EVICT_LEFT = 0, 1, 2
+RULE_SCORES, RULE_KEEP_LEFT, RULE_EVICT_LEFT, RULE_ACCUMULATED = 0, 1, 2, 3
 OPT_DECODE_SPLIT, OPT_PREFILL_PATH, OPT_DECODE_PATH, OPT_PREFILL_APPEND, OPT_EVICTION_STREAM = 0, 1, 2, 3, 4
 OPT_PREFILL_KEY_SPLIT = 5
 

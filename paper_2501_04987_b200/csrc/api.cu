@@ -573,7 +573,8 @@ int64_t treekv_tokens_seen(const treekv_ctx* ctx, int b) {
 
 treekv_status treekv_set_rule(treekv_ctx* ctx, treekv_rule rule) {
     if (!ctx) return TREEKV_ERR_INVALID_ARG;
-    if (rule != TREEKV_RULE_SCORES && rule != TREEKV_RULE_KEEP_LEFT && rule != TREEKV_RULE_EVICT_LEFT)
+    if (rule != TREEKV_RULE_SCORES && rule != TREEKV_RULE_KEEP_LEFT && rule != TREEKV_RULE_EVICT_LEFT &&
+        rule != TREEKV_RULE_ACCUMULATED)
         return TREEKV_ERR_INVALID_ARG;
     ctx->cv.rule = (int)rule;
     return TREEKV_OK;

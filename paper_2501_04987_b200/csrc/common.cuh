@@ -151,14 +151,15 @@ __device__ inline uint4 ld_plain(const void* p) { return *reinterpret_cast<const
 // tokens older than the observation window were only scored from the window's first query (w0) on.
 __host__ __device__ inline int score_count(int n_seen, int pos, int w0) { return n_seen - (pos > w0 ? pos : w0); }
 
-// Algorithm 1's comparison on the averaged scores; returns true when the right member of the pair is evicted.
+// Algorithm 1's comparison on the averaged scores (on the accumulated ones under TREEKV_RULE_ACCUMULATED); returns true when the right member of the pair is evicted.
 // Also reports whether the decision was a near-tie (relative gap below kNearTieRel).
 __device__ inline bool pair_evicts_right(float S_l, int C_l, float S_r, int C_r, int rule, bool* near_tie) {
     *near_tie = false;
     if (rule == TREEKV_RULE_KEEP_LEFT) return true;
     if (rule == TREEKV_RULE_EVICT_LEFT) return false;
-    const float a = __fdiv_rn(S_l, (float)C_l);
-    const float b = __fdiv_rn(S_r, (float)C_r);
+    const bool acc = rule == TREEKV_RULE_ACCUMULATED;  // the sums themselves instead of the averages
+    const float a = acc ? S_l : __fdiv_rn(S_l, (float)C_l);
+    const float b = acc ? S_r : __fdiv_rn(S_r, (float)C_r);
     const float mx = fmaxf(fabsf(a), fabsf(b));
     *near_tie = !(fabsf(a - b) >= kNearTieRel * mx);
     return a > b;  // strict: ties and NaN evict the left (older) slot

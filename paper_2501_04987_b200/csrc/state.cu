@@ -509,11 +509,12 @@ oneshot_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens, int
     const int chunks = cv.d * (int)sizeof(T) / 16;
     int* dec = reinterpret_cast<int*>(scratch);  // [pairs of the segment] 1 = the right block goes
     const float inv_bs = 1.0f / (float)bs;
-    auto block_score = [&](int brow) {  // mean of S / C over the block's tokens, summed in a fixed order
+    const bool accumulated = cv.rule == TREEKV_RULE_ACCUMULATED;
+    auto block_score = [&](int brow) {  // mean of S / C (of S: accumulated rule) over the block's tokens, in a fixed order
         float a = 0.f;
         for (int t = lane; t < bs; t += 32) {
             const int row = brow * bs + t;
-            a += __fdiv_rn(Sc[row], (float)score_count(m, Pc[row], wstart));
+            a += accumulated ? Sc[row] : __fdiv_rn(Sc[row], (float)score_count(m, Pc[row], wstart));
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);

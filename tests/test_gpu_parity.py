@@ -268,6 +268,43 @@ def test_score_free_rules_match_closed_structure(gpu, rule):
         assert np.array_equal(pa, orc.retained_positions()[0])
 
 
+@pytest.mark.parametrize("dtype,d,g,path", [("bf16", 128, 4, 0), ("bf16", 128, 1, 3), ("f32", 64, 2, 0), ("bf16", 64, 8, 0)])
+def test_accumulated_criterion(gpu, dtype, d, g, path):
+    """Section 4.1 "Importance Score": the accumulated attention weight S as the criterion instead of S / C.  Chunked
+    prefill (tensor-core and CUDA-core kernels), decode (both kernels) and a one-shot block prefill in lock-step with
+    the oracle under the same rule; on these inputs the rule retains other tokens than the average does."""
+    from lockstep import step_oneshot
+    from oracle import RULE_ACCUMULATED, Oracle
+
+    w = W.parity_slice(W.CONFIGS["cfg4"], layers=1, batch=2, n_heads=2 * g, n_kv_heads=2, head_dim=d, dtype=dtype, budget=96,
+                       chunk=128)
+    kv = gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, d, dtype, 2, 128)
+    kv.set_rule(gpu.RULE_ACCUMULATED)
+    if path:
+        kv.set_option(gpu.OPT_PREFILL_PATH, path)
+    orc = Oracle(w.budget, w.n_heads, w.n_kv_heads, d, 2, rule=RULE_ACCUMULATED)
+    avg = Oracle(w.budget, w.n_heads, w.n_kv_heads, d, 2)
+    rep = Report()
+    q, k, v = W.tokens(w, 0, 0, 128)
+    qt, kt, vt = (x.transpose(1, 0, 2, 3) for x in (q, k, v))
+    step_oneshot(kv, orc, qt, kt, vt, 8, dtype, rep, lens=[128, 64])
+    avg.prefill_oneshot(qt, kt, vt, 8, [128, 64])
+    seen = [128, 64]
+    for lens in ([128, 128], [77, 128], [128, 0]):
+        qc, kc, vc = W.tokens_at(w, 0, seen, 128)
+        step_prefill(kv, orc, qc.transpose(1, 0, 2, 3), kc.transpose(1, 0, 2, 3), vc.transpose(1, 0, 2, 3), dtype, rep,
+                     chunk_lens=lens)
+        avg.prefill_chunk(qc.transpose(1, 0, 2, 3), kc.transpose(1, 0, 2, 3), vc.transpose(1, 0, 2, 3), lens)
+        seen = [a + b for a, b in zip(seen, lens)]
+    for _ in range(w.budget + 30):
+        qd, kd, vd = W.tokens_at(w, 0, seen, 1)
+        step_decode(kv, orc, qd[0], kd[0], vd[0], dtype, rep)
+        avg.decode_step(qd[0], kd[0], vd[0])
+        seen = [a + 1 for a in seen]
+    assert kv.stats()["device_error"] == 0 and rep.decisions > 0
+    assert not np.array_equal(orc.retained_positions()[0], avg.retained_positions()[0])
+
+
 def test_inactive_sequences_are_untouched(gpu):
     import torch
 

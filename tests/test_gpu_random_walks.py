@@ -1,10 +1,10 @@
 """GPU parity on random walks through the C ABI: every seed draws a cache geometry (dtype, head_dim, group size, batch,
-budget, chunk capacity), optional protected tokens and in-cache positions, kernel options, and a sequence of calls
-that mixes decode steps under changing active sets with ragged chunks (zero lengths included) and, where the
-geometry allows it, a one-shot block prefill as the first call.  The CUDA library runs in lock-step with the fp64
-oracle and is held to the usual bars after every call: retained positions exactly up to counted near-ties, outputs
-within 2e-2 (bf16) / 1e-4 (fp32), averaged scores within 1e-3.  The fixed cases of the other files aim at known
-corners; this one looks for the corners nobody thought of.
+budget, chunk capacity), optional protected tokens, in-cache positions and the accumulated criterion, kernel options,
+and a sequence of calls that mixes decode steps under changing active sets with ragged chunks (zero lengths
+included) and, where the geometry allows it, a one-shot block prefill as the first call.  The CUDA library runs in
+lock-step with the fp64 oracle and is held to the usual bars after every call: retained positions exactly up to
+counted near-ties, outputs within 2e-2 (bf16) / 1e-4 (fp32), averaged scores within 1e-3.  The fixed cases of the
+other files aim at known corners; this one looks for the corners nobody thought of.
 """
 import numpy as np
 import pytest
@@ -60,11 +60,12 @@ def _chunk_lens(rng, batch, max_chunk):
 @pytest.mark.parametrize("seed", range(64))
 def test_random_walk(gpu, seed):
     import torch
-    from oracle import Oracle
+    from oracle import RULE_ACCUMULATED, RULE_SCORES, Oracle
 
     rng = np.random.default_rng(977 + seed)
     dtype, d, hkv, g, batch, budget, max_chunk = _draw_geometry(rng)
     positions = rng.random() < 0.35
+    accumulated = rng.random() < 0.25   # Section 4.1 "Importance Score": S instead of S / C as the criterion
     ns = nr = 0
     if budget >= 4 and rng.random() < 0.4:
         ns = int(rng.integers(0, min(6, budget - 2) + 1))
@@ -72,7 +73,9 @@ def test_random_walk(gpu, seed):
     w = W.parity_slice(W.CONFIGS["cfg4"], layers=1, batch=batch, n_heads=g * hkv, n_kv_heads=hkv, head_dim=d, dtype=dtype,
                        budget=budget, chunk=max_chunk, rotate=not positions, seed=31000 + seed)
     kv = gpu.TreeKV(budget, g * hkv, hkv, d, dtype, batch, max_chunk)
-    orc = Oracle(budget, g * hkv, hkv, d, batch, n_sink=ns, n_recent=nr)
+    orc = Oracle(budget, g * hkv, hkv, d, batch, n_sink=ns, n_recent=nr, rule=RULE_ACCUMULATED if accumulated else RULE_SCORES)
+    if accumulated:
+        kv.set_rule(gpu.RULE_ACCUMULATED)
     if ns or nr:
         kv.set_protection(ns, nr)
     if positions:
@@ -95,8 +98,8 @@ def test_random_walk(gpu, seed):
               gpu.OPT_PREFILL_APPEND, gpu.OPT_EVICTION_STREAM):   # the path first: setting it resets the split
         if o in opts:
             kv.set_option(o, opts[o])
-    label = "seed %d: %s d=%d Hkv=%d g=%d B=%d c=%d max_chunk=%d ns=%d nr=%d positions=%d opts=%s" % (
-        seed, dtype, d, hkv, g, batch, budget, max_chunk, ns, nr, positions, opts)
+    label = "seed %d: %s d=%d Hkv=%d g=%d B=%d c=%d max_chunk=%d ns=%d nr=%d positions=%d accumulated=%d opts=%s" % (
+        seed, dtype, d, hkv, g, batch, budget, max_chunk, ns, nr, positions, accumulated, opts)
     print(label)
     rep = Report()
     seen = [0] * batch
