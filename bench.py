@@ -69,20 +69,20 @@ def measured_peaks():
 # profiles/, valid for the named workload's per-layer shape and only while the kernel's sources are the ones that
 # were profiled: a changed source file makes the entry stale and the reported traffic null.
 NCU_TRAFFIC = {
-    ('decode_mma_kernel', 'cfg4'): {"bytes_per_launch": 278167552, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
-        "sha1": "68d62dd60bbcd00707594a51ac84df544e179320", "profile": "profiles/decode_mma_cfg4_1layer.md"},
-    ('decode_mma_kernel', 'cfg2'): {"bytes_per_launch": 141089792, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
-        "sha1": "68d62dd60bbcd00707594a51ac84df544e179320", "profile": "profiles/decode_mma_cfg2_1layer.md"},
-    ('decode_mma_kernel', 'cfg5'): {"bytes_per_launch": 69239808, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
-        "sha1": "68d62dd60bbcd00707594a51ac84df544e179320", "profile": "profiles/decode_mma_cfg5_1layer.md"},
-    ('decode_mma_kernel', 'cfg3'): {"bytes_per_launch": 33949696, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
-        "sha1": "68d62dd60bbcd00707594a51ac84df544e179320", "profile": "profiles/decode_mma_cfg3_1layer.md"},
-    ('prefill_tc2_kernel', 'cfg5'): {"bytes_per_launch": 165677568, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
-        "sha1": "caa9d345bc96b97cebbf7872a73829f91129dac1", "profile": "profiles/prefill_tc2_cfg5_1layer.md"},
-    ('prefill_tc2_kernel', 'cfg4'): {"bytes_per_launch": 1167068928, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
-        "sha1": "caa9d345bc96b97cebbf7872a73829f91129dac1", "profile": "profiles/prefill_tc2_cfg4_1layer.md"},
-    ('prefill_tc_kernel', 'cfg3'): {"bytes_per_launch": 46872064, "sources": ['prefill_tc.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
-        "sha1": "8d92180bea87292fdd37121f278e962a3d3ccdc4", "profile": "profiles/prefill_tc_cfg3_2layers.md"},
+    ('decode_mma_kernel', 'cfg4'): {"bytes_per_launch": 276873216, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
+        "sha1": "7760273f6afd79fd142d87e0070cdb22723b8994", "profile": "profiles/decode_mma_cfg4_1layer.md"},
+    ('decode_mma_kernel', 'cfg2'): {"bytes_per_launch": 140841472, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
+        "sha1": "7760273f6afd79fd142d87e0070cdb22723b8994", "profile": "profiles/decode_mma_cfg2_1layer.md"},
+    ('decode_mma_kernel', 'cfg5'): {"bytes_per_launch": 68887808, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
+        "sha1": "7760273f6afd79fd142d87e0070cdb22723b8994", "profile": "profiles/decode_mma_cfg5_1layer.md"},
+    ('decode_mma_kernel', 'cfg3'): {"bytes_per_launch": 33938944, "sources": ['decode_mma.cu', 'common.cuh', 'tma.cuh'],
+        "sha1": "7760273f6afd79fd142d87e0070cdb22723b8994", "profile": "profiles/decode_mma_cfg3_1layer.md"},
+    ('prefill_tc2_kernel', 'cfg5'): {"bytes_per_launch": 165460992, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
+        "sha1": "2005cb6e2d6cc6f07ec484540ac8d3c80dec117e", "profile": "profiles/prefill_tc2_cfg5_1layer.md"},
+    ('prefill_tc2_kernel', 'cfg4'): {"bytes_per_launch": 1166141696, "sources": ['prefill_tc2.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
+        "sha1": "2005cb6e2d6cc6f07ec484540ac8d3c80dec117e", "profile": "profiles/prefill_tc2_cfg4_1layer.md"},
+    ('prefill_tc_kernel', 'cfg3'): {"bytes_per_launch": 46809600, "sources": ['prefill_tc.cu', 'prefill_tc_common.cuh', 'tma.cuh', 'common.cuh'],
+        "sha1": "c1b30800d0c447cec9ead6770a2a08397de9b4f1", "profile": "profiles/prefill_tc_cfg3_2layers.md"},
 }
 
 
