@@ -302,9 +302,11 @@ treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, 
                 if (rem > 0 && 2 * rem <= sms && pairs > rem) n_whole = (int)((pairs - rem) / 2);
             }
         }
+        ctx->attn_blocks = two ? (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + 2 * kQTileRows - 1) / (2 * kQTileRows)) : tiles;
         e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, *tmKeys, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, n_whole, s)
                 : launch_prefill_tc(ctx->cv, ps, tmQ, *tmKeys, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, s);
     } else {
+        ctx->attn_blocks = 0;
         e = launch_prefill_simt(ctx->cv, ctx->dt, ps, dev_q, dev_out, lens, chunk_stride, max_m, s);
     }
     return e == cudaSuccess ? TREEKV_OK : cuda_fail(ctx, e);
@@ -368,7 +370,15 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
     if (ctx->side) {
         e = cudaEventRecord(ctx->ev_attn, s);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->side, ctx->ev_attn, 0);
-        if (e == cudaSuccess) e = launch_chunk_update_evict(ctx->cv, ctx->dt, ctx->ps, lens, true, ctx->side);
+        // Beside the next attention kernel (typically the next layer's chunk, with the grid this one had): when that
+        // grid leaves SMs free, the eviction takes no more blocks than those SMs - an eviction block and an attention
+        // block do not fit on one SM, and blocks that got there first would hold up part of the attention's only wave.
+        int max_blocks = 0;
+        if (ctx->attn_blocks > 0 && ctx->attn_blocks < ctx->sm_count) {
+            const int units = ctx->cv.B * ctx->cv.Hkv;
+            max_blocks = std::max((int)(ctx->sm_count - ctx->attn_blocks), std::max(1, units / 4));
+        }
+        if (e == cudaSuccess) e = launch_chunk_update_evict_beside(ctx->cv, ctx->dt, ctx->ps, lens, max_blocks, ctx->side);
         if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_state, ctx->side);
         ctx->side_pending = true;  // also after a failure half-way: a later call then still orders itself behind `side`
     } else {

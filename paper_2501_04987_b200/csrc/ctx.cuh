@@ -28,6 +28,7 @@ struct treekv_ctx {
     cudaEvent_t ev_attn, ev_state;
     bool side_pending;  // a kernel on `side` may still be running that the caller's stream has not been told to wait for
     int sm_count;
+    long attn_blocks;  // thread blocks of the last chunk-attention launch (0: a kernel whose grid is not counted)
     int device;  // ordinal of the device that was current at creation: the workspace lives there
     // host-side record
     int64_t n_seen[treekv::kMaxBatch];
@@ -37,6 +38,9 @@ struct treekv_ctx {
 };
 
 namespace treekv {
+// chunk score update + eviction as blocks of 1024 threads, at most max_blocks of them (0 = one per unit): state.cu
+cudaError_t launch_chunk_update_evict_beside(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps,
+                                             const ChunkLens& lens, int max_blocks, cudaStream_t stream);
 // Orders `stream` behind the context's eviction stream, if a kernel there has not been waited for yet.  Every entry
 // point that enqueues work on the cache calls this first.
 inline cudaError_t join_eviction_stream(treekv_ctx* ctx, cudaStream_t stream) {

@@ -4,6 +4,7 @@
 #include <cooperative_groups.h>
 
 #include "common.cuh"
+#include "ctx.cuh"
 
 namespace treekv {
 
@@ -336,10 +337,12 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     auto unit_sync = [&]() { if (kEvictCluster == 1) __syncthreads(); else cluster.sync(); };
-    const int unit = blockIdx.y;
+    // a block (cluster) takes the units blockIdx.y, blockIdx.y + gridDim.y, ...: one each unless the launch asked for
+    // fewer blocks than units
+    for (int unit = blockIdx.y; unit < cv.B * cv.Hkv; unit += gridDim.y) {
     const int b = unit / cv.Hkv;
     const int m = lens.m[b];
-    if (m == 0) return;  // the whole cluster shares the unit
+    if (m == 0) continue;  // the whole cluster shares the unit
     const int rank = (int)cluster.block_rank();
     const int G = cv.Hq / cv.Hkv;
     const int N = cv.n_seen[unit];
@@ -422,13 +425,15 @@ chunk_update_evict_kernel(CacheView cv, PrefillScratch ps, ChunkLens lens) {
         }
         if (seg + 1 < nseg) unit_sync();  // the next segment's pairs read rows this one wrote
     }
+    }
 }
 
 template <typename T, int CL>
 static cudaError_t launch_chunk_update_evict_t(const CacheView& cv, const PrefillScratch& ps, const ChunkLens& lens,
-                                               cudaStream_t stream) {
+                                               int max_blocks, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(CL, cv.B * cv.Hkv);
+    const int units = cv.B * cv.Hkv;
+    cfg.gridDim = dim3(CL, max_blocks > 0 && max_blocks < units ? max_blocks : units);
     cfg.blockDim = dim3(evict_threads(CL));
     cfg.stream = stream;  // plain stream order behind the attention kernel; the kernel after it may be scheduled early
     cudaLaunchAttribute attr[1];
@@ -443,11 +448,17 @@ static cudaError_t launch_chunk_update_evict_t(const CacheView& cv, const Prefil
 
 cudaError_t launch_chunk_update_evict(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps, const ChunkLens& lens,
                                       bool small_footprint, cudaStream_t stream) {
-    if (dt == TREEKV_F32)
-        return small_footprint ? launch_chunk_update_evict_t<float, 1>(cv, ps, lens, stream)
-                               : launch_chunk_update_evict_t<float, 4>(cv, ps, lens, stream);
-    return small_footprint ? launch_chunk_update_evict_t<__nv_bfloat16, 1>(cv, ps, lens, stream)
-                           : launch_chunk_update_evict_t<__nv_bfloat16, 4>(cv, ps, lens, stream);
+    return small_footprint ? launch_chunk_update_evict_beside(cv, dt, ps, lens, 0, stream)
+                           : (dt == TREEKV_F32 ? launch_chunk_update_evict_t<float, 4>(cv, ps, lens, 0, stream)
+                                               : launch_chunk_update_evict_t<__nv_bfloat16, 4>(cv, ps, lens, 0, stream));
+}
+
+// The form that runs beside another kernel (eviction stream): one block of 1024 threads per unit, at most max_blocks
+// blocks (0 = one per unit), each then taking several units in turn.
+cudaError_t launch_chunk_update_evict_beside(const CacheView& cv, treekv_dtype dt, const PrefillScratch& ps,
+                                             const ChunkLens& lens, int max_blocks, cudaStream_t stream) {
+    return dt == TREEKV_F32 ? launch_chunk_update_evict_t<float, 1>(cv, ps, lens, max_blocks, stream)
+                            : launch_chunk_update_evict_t<__nv_bfloat16, 1>(cv, ps, lens, max_blocks, stream);
 }
 
 // ---------------------------------------------------------------------------------------------------------

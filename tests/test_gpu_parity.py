@@ -476,6 +476,31 @@ def test_eviction_stream_gives_the_same_bits_and_follows_the_oracle(gpu):
     assert kv.stats()["device_error"] == 0
 
 
+def test_eviction_beside_an_attention_grid_that_leaves_few_sms_free(gpu):
+    """An attention grid just below the machine (32 units x 4 query tiles = 128 thread blocks on 148 SMs) leaves 20 SMs
+    to the eviction kernel of the previous layer, which is then launched with 20 blocks for its 32 units: some blocks
+    take two units in turn.  Same bits as on one stream, and in lock-step with the oracle, ragged and inactive
+    sequences included."""
+    import torch
+
+    w = W.parity_slice(W.CONFIGS["cfg4"], layers=1, batch=2, n_heads=32, n_kv_heads=16, budget=192, chunk=256)
+    if torch.cuda.get_device_properties(0).multi_processor_count <= 128:
+        pytest.skip("the case needs more than 128 SMs")
+    kv, orc = _pair(gpu, w)
+    ref = gpu.TreeKV(w.budget, w.n_heads, w.n_kv_heads, w.head_dim, w.dtype, w.batch, w.chunk)
+    kv.set_option(gpu.OPT_EVICTION_STREAM, 1)
+    rep = Report()
+    seen = [0, 0]
+    for lens in ([256, 256], [256, 256], [256, 131], [256, 0], [256, 256]):
+        q, k, v = W.tokens_at(w, 0, seen, 256)
+        q, k, v = (x.transpose(1, 0, 2, 3) for x in (q, k, v))
+        step_prefill(kv, orc, q, k, v, w.dtype, rep, chunk_lens=lens)
+        ref.prefill_chunk(*(torch.from_numpy(np.ascontiguousarray(x)).cuda().bfloat16() for x in (q, k, v)), chunk_lens=lens)
+        seen = [a + b for a, b in zip(seen, lens)]
+        assert torch.equal(kv.scores(), ref.scores()) and torch.equal(kv.retained_positions()[0], ref.retained_positions()[0])
+    assert kv.stats()["device_error"] == 0 and rep.decisions > 0
+
+
 @pytest.mark.parametrize("pinned", [True, False])
 def test_host_entry_points_match_device_entry_points(gpu, pinned):
     """Page-locked host tensors are read by the decode kernel directly; pageable ones go through staging copies."""
