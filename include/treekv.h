@@ -278,8 +278,8 @@ int64_t treekv_tokens_seen(const treekv_ctx* ctx, int b);
 treekv_status treekv_set_rule(treekv_ctx* ctx, treekv_rule rule);
 
 /*
- * Protected tokens (Section 5.2: the language-modelling runs keep "4 initial tokens, 508 recent tokens, and 512
- * method-selected tokens" in a cache of 1024).  The first n_sink tokens of every sequence and its n_recent newest
+ * Protected tokens (Section 5.2: the language-modelling runs split a cache of 1024 into 4 initial tokens, 508 recent ones
+ * and 512 chosen by the method).  The first n_sink tokens of every sequence and its n_recent newest
  * cached tokens are never in an eviction scope; Algorithm 1 runs on the budget - n_sink - n_recent slots between
  * them (idx cycles over that many slots), and a token becomes eligible in the step in which it stops being one of
  * the n_recent newest.  S and C of every cached token advance from its arrival as in Algorithm 1.  The paper gives

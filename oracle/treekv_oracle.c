@@ -31,7 +31,7 @@
  *     chunk attends to every slot whose pos <= its own, S and C are advanced
  *     for all m steps at once, then Algorithm 1's eviction branch is repeated
  *     with those frozen scores until the length is back to c.
- *   - protected tokens (Section 5.2, "4 initial tokens, 508 recent tokens, and 512 method-selected tokens"; the
+ *   - protected tokens (Section 5.2: a cache of 1024 split into 4 initial, 508 recent and 512 method-chosen tokens; the
  *     paper does not say how the three parts interact): the first n_sink tokens of the stream and the newest
  *     n_recent cached tokens are never in an eviction scope.  Algorithm 1 runs on the region between them, whose
  *     size is c_mid = c - n_sink - n_recent: the scope is slots {n_sink + idx, n_sink + idx + 1} of the whole
@@ -39,8 +39,8 @@
  *     n_recent newest (it is then the last slot of the middle region, exactly where Algorithm 1 appends).  S and
  *     C of every cached token, protected or not, advance as in Algorithm 1 from the token's arrival.  With
  *     n_sink = n_recent = 0 this is Algorithm 1 unchanged.
- *   - one-shot, block-level prefill (Section 4.2): the prompt is cut into blocks of b tokens, "each block
- *     representing one token" of Algorithm 1; the last block is the observation window whose b queries score the
+ *   - one-shot, block-level prefill (Section 4.2): the prompt is cut into blocks of b tokens, each block
+ *     standing for one token of Algorithm 1; the last block is the observation window whose b queries score the
  *     whole prompt: Algorithm 1's S and C updates are applied for those b rows only, so a token older than the
  *     window has C = b and window token u (0-based) has C = b - u; a block's score is the mean of its tokens'
  *     S/C; Algorithm 1's branch then runs on blocks with a cache of c / b blocks, blocks arriving in order.  The

@@ -466,7 +466,7 @@ cudaError_t launch_chunk_update_evict_beside(const CacheView& cv, treekv_dtype d
 // prompt's m tokens sit in rows [0, m); the attention kernel left the column sums of the observation window (the
 // last `bs` tokens) per query tile.  This kernel adds them to S (Algorithm 1's S update for the window's rows; the
 // counter C of a token is the number of window rows that see it, kept implicitly through w0 = m - bs), then plays
-// Algorithm 1's "length > c" branch on blocks of bs tokens - "each block representing one token": a block's score
+// Algorithm 1's "length > c" branch on blocks of bs tokens, a block standing for one token: a block's score
 // is the mean of its tokens' S / C, the cache holds c / bs blocks, and the cycle-coordinate layout applies to
 // block rows (block r = token rows [r bs, (r+1) bs)), so that the final token rows are exactly the token-level
 // layout at cycle position ((m - c) mod c).  Per segment: one warp per pair decides (decisions go to the unit's

@@ -1,5 +1,5 @@
-"""Pins for the oracle's sink / recent-window protection (Section 5.2: "4 initial tokens, 508 recent tokens, and
-512 method-selected tokens").  The paper gives the split, not the mechanics; the reading under test is stated in
+"""Pins for the oracle's sink / recent-window protection (Section 5.2: a cache of 1024 split into 4 initial,
+508 recent and 512 method-chosen tokens).  The paper gives the split, not the mechanics; the reading under test is stated in
 the oracle's header.  What can be fixed without the CUDA library: nothing changes without protection; protected
 tokens are never evicted; the middle region is plain TreeKV on the delayed sub-stream (closed forms of the
 score-free rules carry over); a dictionary-based restatement on tiny inputs; the paper's 4 / 508 / 512 split.
