@@ -373,10 +373,12 @@ treekv_status treekv_prefill_chunk(treekv_ctx* ctx, const void* dev_q, const voi
         // Beside the next attention kernel (typically the next layer's chunk, with the grid this one had): when that
         // grid leaves SMs free, the eviction takes no more blocks than those SMs - an eviction block and an attention
         // block do not fit on one SM, and blocks that got there first would hold up part of the attention's only wave.
+        // With fewer free SMs than a quarter of the units the blocks would run long enough to be in the way for longer
+        // than a full launch is: then every unit gets its block.
         int max_blocks = 0;
         if (ctx->attn_blocks > 0 && ctx->attn_blocks < ctx->sm_count) {
-            const int units = ctx->cv.B * ctx->cv.Hkv;
-            max_blocks = std::max((int)(ctx->sm_count - ctx->attn_blocks), std::max(1, units / 4));
+            const int units = ctx->cv.B * ctx->cv.Hkv, free_sms = (int)(ctx->sm_count - ctx->attn_blocks);
+            if (free_sms < units && 4 * free_sms >= units) max_blocks = free_sms;
         }
         if (e == cudaSuccess) e = launch_chunk_update_evict_beside(ctx->cv, ctx->dt, ctx->ps, lens, max_blocks, ctx->side);
         if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_state, ctx->side);
