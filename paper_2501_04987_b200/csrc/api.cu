@@ -302,7 +302,11 @@ treekv_status launch_chunk_attention(treekv_ctx* ctx, const PrefillScratch& ps, 
                 if (rem > 0 && 2 * rem <= sms && pairs > rem) n_whole = (int)((pairs - rem) / 2);
             }
         }
-        ctx->attn_blocks = two ? (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + 2 * kQTileRows - 1) / (2 * kQTileRows)) : tiles;
+        ctx->attn_blocks = tiles;
+        if (two) {  // one block per tile pair; with key splitting two per cluster: whole-pair clusters, then one cluster per pair
+            const long pairs = (long)ctx->cv.B * ctx->cv.Hkv * ((max_m * ctx->G + 2 * kQTileRows - 1) / (2 * kQTileRows));
+            ctx->attn_blocks = n_whole < 0 ? pairs : 2 * (n_whole + std::max(0L, pairs - 2L * n_whole));
+        }
         e = two ? launch_prefill_tc2(ctx->cv, ps, tmQ, *tmKeys, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, n_whole, s)
                 : launch_prefill_tc(ctx->cv, ps, tmQ, *tmKeys, ctx->tmV, ct, dev_out, lens, chunk_stride, max_m, s);
     } else {
